@@ -1,0 +1,267 @@
+"""CPU oracle for the SurfaceLogicKV prefill KV-compression step.  TEST INFRASTRUCTURE ONLY.
+
+Plain, slow, fp64 numpy written from the paper; it shares no code with the CUDA library and must never
+be imported by the product path (only tests, the smoke check and the bench's CPU-baseline leg use it).
+A numpy matmul / stable sort serves as a step where the definition is a matrix product / an ordering;
+there is no blocking, fusion or reordering beyond what the definitions state.
+
+What follows which passage of the paper:
+  alloc_paper_literal   Algorithm 2 (and Eq. 6) exactly as printed, with its line-8 rounding.
+  alloc_budgets         Algorithm 2's weights (0.01 + L_i) * S_ij, normalised so the dynamic parts sum to
+                        the dynamic pool exactly (largest-remainder rounding) -- the paper concedes that its
+                        own formula "does not strictly conform to mathematical normalization" (Sec. 3.3).
+  window_votes          Eq. 7 / Algorithm 3 line 6: softmax over the history keys of Q_window H^T / sqrt(d_k)
+                        (Eq. 3-4 fix the scale and the softmax axis), then -- the paper does not say how the
+                        w rows are reduced -- summed over the window rows and averaged over a GQA group.
+  pool                  not in the paper (it defers to prior work): max / mean over an odd window, stride 1.
+  select_topk           Eq. 8 / Algorithm 3 lines 7-8: the C - window best history entries.
+  compress              Algorithm 3 as a whole: early-out, window always kept, Concat(history', window).
+  behavior_scores       Algorithm 1 (SF_sc, LG_sc, INF_sc of one attention row).
+
+Pins (tests/test_oracle_*.py): brute-force attention from Eq. 4 in pure Python loops, votes summing to w,
+closed forms for equal keys / one dominant key, permutation equivariance, box response of max pooling,
+exhaustive pure-Python sort for selection, Hamilton apportionment in exact rationals, the closed form
+sum of Algorithm 2's literal dynamic parts, the (b_c, beta) <-> (fixed, total) mapping at the paper's
+beta = 1.351, Algorithm 1 against the harmonic-mean identity and the consistency of Tables 6-8.
+Parity unpinned: the *choices* the paper leaves open (pool type, softmax over history only vs. all causal
+keys, global vs. within-layer head normaliser) are readings, each behind a flag; no printed value fixes them.
+"""
+from __future__ import annotations
+
+import math
+from typing import List, Sequence, Tuple
+
+import numpy as np
+
+LAYER_FLOOR = 0.01          # Sec. 3.3: minimum layer budget
+
+
+class OracleError(ValueError):
+    def __init__(self, code: str, msg: str = ""):
+        super().__init__(f"{code}: {msg}")
+        self.code = code
+
+
+# ----------------------------------------------------------------------------------------------
+# Stage 2: budgets
+# ----------------------------------------------------------------------------------------------
+def paper_fixed_and_pool(b_c: float, beta: float, n_layers: int, n_heads: int) -> Tuple[float, float]:
+    """Algorithm 2 lines 1-2: b_fixed = b_c (1 - 1/beta), B_total = (b_c / beta) L H."""
+    return b_c * (1.0 - 1.0 / beta), (b_c / beta) * n_layers * n_heads
+
+
+def alloc_paper_literal(b_c: float, beta: float, inf: np.ndarray, rounded: bool = True) -> np.ndarray:
+    """Algorithm 2 as printed.  inf[i][j] = INF_sc of head j in layer i.  Returns C[i][j]."""
+    inf = np.asarray(inf, dtype=np.float64)
+    L, H = inf.shape
+    b_fixed, B_total = paper_fixed_and_pool(b_c, beta, L, H)
+    L_alpha = [sum(float(inf[i][j]) for j in range(H)) for i in range(L)]        # line 3
+    L_s = sum(L_alpha)                                                           # line 4
+    out = np.zeros((L, H), dtype=np.float64)
+    for i in range(L):
+        L_ih = L_alpha[i] / L_s                                                  # line 5
+        for j in range(H):
+            S_jh = float(inf[i][j]) / L_s                                        # line 5
+            b_dyn = B_total * (LAYER_FLOOR + L_ih) * S_jh                        # line 6
+            b = b_fixed + b_dyn                                                  # line 7
+            out[i][j] = math.floor(max(0.0, b) + 0.5) if rounded else b          # line 8
+    return out.astype(np.int64) if rounded else out
+
+
+def alloc_budgets(inf: np.ndarray, fixed: int, total: int) -> np.ndarray:
+    """Integer budgets C[i][j] >= fixed with sum exactly `total` (Algorithm 2's weights, normalised).
+
+    Every floating-point operation is a separately rounded fp64 operation in the order written, sums run
+    in index order: the CUDA kernel must reproduce the result bit for bit.
+    """
+    inf32 = np.asarray(inf, dtype=np.float32)
+    if inf32.ndim != 2:
+        raise OracleError("BAD_SHAPE", "inf must be [n_layers, n_heads]")
+    L, H = inf32.shape
+    N = L * H
+    D = int(total) - N * int(fixed)
+    if fixed < 0 or D < 0:
+        raise OracleError("BUDGET_SUM", "total < n_heads_total * fixed")
+    x = inf32.astype(np.float64)
+    if not np.all(np.isfinite(x)) or np.any(x < 0):
+        raise OracleError("NEG_INF_SC", "INF_sc must be finite and >= 0")
+
+    La = [0.0] * L
+    for i in range(L):
+        acc = 0.0
+        for j in range(H):
+            acc = acc + float(x[i][j])
+        La[i] = acc
+    Ls = 0.0
+    for i in range(L):
+        Ls = Ls + La[i]
+
+    wgt = [1.0] * N
+    if Ls > 0.0:
+        for i in range(L):
+            lw = LAYER_FLOOR + La[i] / Ls                    # 0.01 + L_{i,h}
+            for j in range(H):
+                wgt[i * H + j] = lw * (float(x[i][j]) / Ls)  # * S_{j,h}
+    W = 0.0
+    for a in range(N):
+        W = W + wgt[a]
+    if not (W > 0.0):                                        # everything underflowed: uniform
+        wgt = [1.0] * N
+        W = float(N)
+
+    f = [0] * N
+    r = [0.0] * N
+    for a in range(N):
+        q = (float(D) * wgt[a]) / W
+        fl = math.floor(q)
+        f[a] = int(fl)
+        r[a] = q - fl
+    R = D - sum(f)
+    if R >= N:                                               # cannot happen in exact arithmetic
+        for a in range(N):
+            f[a] += R // N
+        R = R % N
+    if R > 0:
+        order = sorted(range(N), key=lambda a: (-r[a], a))  # largest remainder, ties -> lower index
+        for a in order[:R]:
+            f[a] += 1
+    while R < 0:                                             # rounding pushed the floors above D
+        cand = [a for a in range(N) if f[a] > 0]
+        order = sorted(cand, key=lambda a: (r[a], -a))       # smallest remainder, ties -> higher index
+        take = order[:min(-R, len(order))]
+        for a in take:
+            f[a] -= 1
+        R += len(take)
+    return (np.array(f, dtype=np.int64) + int(fixed)).reshape(L, H)
+
+
+# ----------------------------------------------------------------------------------------------
+# Stage 1: Algorithm 1
+# ----------------------------------------------------------------------------------------------
+def behavior_scores(W: np.ndarray, needle_idx: Sequence[int], topk_idx: Sequence[int]) -> Tuple[float, float, float]:
+    """Algorithm 1: (SF_sc, LG_sc, INF_sc) of one attention-weight row W; a 0/0 ratio counts as 0."""
+    W = np.asarray(W, dtype=np.float64)
+    Nset, Tset = set(int(i) for i in needle_idx), set(int(i) for i in topk_idx)
+    WO = sum(float(W[i]) for i in sorted(Nset & Tset))
+    WD = sum(float(W[i]) for i in sorted(Tset - Nset))
+    TNW = sum(float(W[i]) for i in sorted(Nset))
+    WS = max(0.0, TNW - WO)
+    SF = WO / (WO + WD) if (WO + WD) > 0 else 0.0
+    LG = WO / (WO + WS) if (WO + WS) > 0 else 0.0
+    INF = 2.0 * SF * LG / (SF + LG) if (SF + LG) > 0 else 0.0
+    return SF, LG, INF
+
+
+# ----------------------------------------------------------------------------------------------
+# Prefill: scores -> pool -> select -> gather
+# ----------------------------------------------------------------------------------------------
+def window_votes(q_win: np.ndarray, k: np.ndarray, cu_seqlens: Sequence[int], window: int,
+                 domain: str = "history") -> List[np.ndarray]:
+    """Per sequence: vote[g][j] = (1/G) sum_{h in group g} sum_{i in window} A^h_ij, fp64 [n_kv_heads, n_hist].
+
+    q_win [n_seqs, window, n_q_heads, d] holds the queries of each sequence's last `window` tokens,
+    k [total_tokens, n_kv_heads, d] the keys.  A^h = softmax_j(q_i . k_j / sqrt(d)) over the history keys
+    j < n_hist = len - window (domain="history", Eq. 7 / Algorithm 3 line 6), or over all keys a window query
+    may see causally (domain="all_causal": history plus window keys up to the query's own position), the
+    window columns being dropped afterwards.
+    """
+    q_win = np.asarray(q_win, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    B, w, Hq, d = q_win.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    assert w == window and Hq == G * Hkv
+    out = []
+    for s in range(B):
+        t0, t1 = int(cu_seqlens[s]), int(cu_seqlens[s + 1])
+        n_hist = max(t1 - t0 - w, 0)
+        vote = np.zeros((Hkv, n_hist), dtype=np.float64)
+        if n_hist > 0:
+            for g in range(Hkv):
+                Hist = k[t0:t0 + n_hist, g, :]                               # [n_hist, d]
+                for h in range(g * G, (g + 1) * G):
+                    Qw = q_win[s, :, h, :]                                   # [w, d]
+                    S = (Qw @ Hist.T) / math.sqrt(d)                         # Eq. 3
+                    if domain == "history":
+                        m = S.max(axis=1, keepdims=True)
+                        E = np.exp(S - m)
+                        A = E / E.sum(axis=1, keepdims=True)                 # Eq. 4, keys = history
+                    elif domain == "all_causal":
+                        Kw = k[t0 + n_hist:t1, g, :]                         # [w, d] window keys
+                        Sw = (Qw @ Kw.T) / math.sqrt(d)
+                        Sw = np.where(np.tril(np.ones((w, w), dtype=bool)), Sw, -np.inf)
+                        full = np.concatenate([S, Sw], axis=1)
+                        m = full.max(axis=1, keepdims=True)
+                        E = np.exp(full - m)
+                        A = (E / E.sum(axis=1, keepdims=True))[:, :n_hist]
+                    else:
+                        raise ValueError(domain)
+                    vote[g] += A.sum(axis=0)                                 # sum over the window rows
+                vote[g] /= G                                                 # mean over the query group
+        out.append(vote)
+    return out
+
+
+def pool(vote: np.ndarray, kernel: int, mode: str = "max") -> np.ndarray:
+    """Stride-1 pooling along the last axis over [j - kernel//2, j + kernel//2] clipped to the array
+    (max), or zero-padded mean (avg: sum over the clipped range divided by `kernel`)."""
+    assert kernel >= 1 and kernel % 2 == 1
+    vote = np.asarray(vote, dtype=np.float64)
+    n = vote.shape[-1]
+    r = kernel // 2
+    out = np.empty_like(vote)
+    for j in range(n):
+        lo, hi = max(0, j - r), min(n - 1, j + r)
+        seg = vote[..., lo:hi + 1]
+        out[..., j] = seg.max(axis=-1) if mode == "max" else seg.sum(axis=-1) / kernel
+    return out
+
+
+def kept_counts(seq_len: int, budget: int, window: int) -> Tuple[int, int]:
+    """(kept history rows, kept window rows) of one head: Algorithm 3 lines 1-4 and 7.
+
+    Everything is kept when the length does not exceed the budget; the window is always kept (so a budget
+    below the window acts as the window); otherwise C_H = C - window history rows survive.
+    """
+    kept = min(seq_len, max(int(budget), window))
+    n_win = min(seq_len, window)
+    return kept - n_win, n_win
+
+
+def select_topk(scores: np.ndarray, k: int) -> np.ndarray:
+    """Indices of the k largest scores, ties -> lower index, returned ascending (Eq. 8 / Alg. 3 line 8)."""
+    scores = np.asarray(scores)
+    order = np.argsort(-scores, kind="stable")                 # stable: equal scores keep index order
+    return np.sort(order[:k]).astype(np.int64)
+
+
+def compress(q_win, k, v, cu_seqlens, budgets, window: int, pool_kernel: int, pool_mode: str = "max",
+             domain: str = "history"):
+    """Algorithm 3 for every (sequence, KV head) segment.
+
+    Returns dict: pooled (list per sequence of [n_kv_heads, n_hist] fp64), kept_idx (list per segment, positions
+    within the sequence, selected history ascending then the window), offsets [n_seg+1], k_out / v_out (rows
+    gathered from the inputs, same dtype as given).  Segment id = s * n_kv_heads + h.
+    """
+    k_arr, v_arr = np.asarray(k), np.asarray(v)
+    Hkv = k_arr.shape[1]
+    B = len(cu_seqlens) - 1
+    votes = window_votes(q_win, k_arr, cu_seqlens, window, domain)
+    pooled = [pool(vt, pool_kernel, pool_mode) for vt in votes]
+    kept_idx, offsets, k_rows, v_rows = [], [0], [], []
+    for s in range(B):
+        t0, t1 = int(cu_seqlens[s]), int(cu_seqlens[s + 1])
+        n = t1 - t0
+        for h in range(Hkv):
+            n_keep_hist, n_win = kept_counts(n, int(budgets[h]), window)
+            hist = select_topk(pooled[s][h], n_keep_hist)
+            idx = np.concatenate([hist, np.arange(n - n_win, n, dtype=np.int64)])
+            kept_idx.append(idx)
+            offsets.append(offsets[-1] + len(idx))
+            k_rows.append(k_arr[t0 + idx, h, :])
+            v_rows.append(v_arr[t0 + idx, h, :])
+    d = k_arr.shape[2]
+    k_out = np.concatenate(k_rows, axis=0) if k_rows else np.zeros((0, d), k_arr.dtype)
+    v_out = np.concatenate(v_rows, axis=0) if v_rows else np.zeros((0, d), v_arr.dtype)
+    return {"pooled": pooled, "kept_idx": kept_idx, "offsets": np.array(offsets, dtype=np.int64),
+            "k_out": k_out, "v_out": v_out}
