@@ -1,0 +1,182 @@
+/*
+ * slkv.h -- C ABI of the SurfaceLogicKV prefill KV-cache compression library (CUDA, sm_100a).
+ *
+ * One call per step of the paper's method:
+ *   slkv_alloc_budgets   Stage 2, per-head KV budgets from the INF_sc table     (Sec. 3.3, Eq. 6, Algorithm 2)
+ *   slkv_score           relevance of every history key to the query window     (Sec. 3.4, Eq. 7, Alg. 3 l.4-6)
+ *   slkv_compress        score -> top-(C - window) history rows + window, gather (Sec. 3.4, Eq. 8, Algorithm 3)
+ *   slkv_compress_host   the same, from/to host buffers (copies included)
+ *
+ * Conventions
+ *   - "dev" pointers are device memory of the current CUDA device, "host" pointers are host memory.
+ *   - The caller owns every buffer.  The library allocates no device memory; scratch comes from the
+ *     caller's `workspace` (size from slkv_workspace_bytes) and must stay untouched until the enqueued
+ *     work has finished.  Nothing is freed or retained by the library.
+ *   - All device work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     No call synchronises the device except slkv_compress_host, which returns after its results are
+ *     in the host buffers.
+ *   - Every function returns SLKV_OK (0) or a negative slkv_status.  Argument errors are found on the
+ *     host before anything is enqueued.  Errors only visible in device data (a negative INF_sc, an
+ *     output capacity that turns out too small) are written to the optional device word `status`
+ *     (untouched when nothing is wrong -- zero it first), never raised as a device fault.
+ *
+ * Tensor layouts (element = float for SLKV_F32, bfloat16 for SLKV_BF16; head_dim contiguous)
+ *   K, V   packed varlen, token-major: element (t, h, p) at t*stride_tok + h*stride_head + p,
+ *          t in [0, total_tokens), sequences delimited by cu_seqlens[n_seqs+1] (cu[0] = 0).
+ *   Q_win  the queries of each sequence's last `window` tokens: element (s, i, h, p) at
+ *          s*q_stride_seq + i*q_stride_row + h*q_stride_head + p; row i is token len_s - window + i.
+ *          (Rows are unused for sequences not longer than the window.)
+ *   GQA    query head h scores against KV head h / (n_q_heads / n_kv_heads).
+ *   pooled ragged float array: sequence s, KV head h, history position j (j < n_hist_s = max(len_s -
+ *          window, 0)) at  n_kv_heads * sum_{s'<s} n_hist_s'  +  h * n_hist_s  +  j.
+ *   packed output: segment seg = s*n_kv_heads + h owns rows offsets[seg] .. offsets[seg+1]-1 of k_out /
+ *          v_out / kept_idx; its rows are the selected history positions in ascending order followed by
+ *          the window positions; a row is head_dim contiguous elements.  kept_idx holds positions
+ *          within the sequence (0-based).
+ */
+#ifndef SLKV_H_
+#define SLKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum slkv_status {
+  SLKV_OK = 0,
+  SLKV_ERR_NULL_PTR = -1,       /* a required pointer is NULL */
+  SLKV_ERR_BAD_SHAPE = -2,      /* a size / count / stride is out of the supported range */
+  SLKV_ERR_BAD_DTYPE = -3,      /* dtype / mode enum not recognised or not supported by the chosen path */
+  SLKV_ERR_BAD_ALIGN = -4,      /* a pointer or stride breaks the 16-byte row alignment rule */
+  SLKV_ERR_BUDGET_SUM = -5,     /* total < n_layers*n_heads*fixed, or fixed < 0 */
+  SLKV_ERR_NEG_INF_SC = -6,     /* an INF_sc entry is negative or not finite (device status word) */
+  SLKV_ERR_CAPACITY = -7,       /* out_capacity_rows smaller than the rows to write */
+  SLKV_ERR_WORKSPACE = -8,      /* workspace NULL or smaller than slkv_workspace_bytes */
+  SLKV_ERR_CUDA = -9,           /* a CUDA runtime call failed (see slkv_last_cuda_error) */
+  SLKV_ERR_DEVICE_TIMEOUT = -10 /* a bounded device-side wait ran out (device status word) */
+} slkv_status;
+
+enum { SLKV_F32 = 0, SLKV_BF16 = 1 };                 /* slkv_params.dtype */
+enum { SLKV_POOL_MAX = 0, SLKV_POOL_AVG = 1 };        /* slkv_params.pool_mode */
+enum { SLKV_HISTORY = 0 };                            /* slkv_params.softmax_domain: softmax over history keys */
+enum { SLKV_PATH_AUTO = 0,                            /* slkv_params.score_path */
+       SLKV_PATH_SIMT = 1,                            /*   fp32 FMA kernels (any dtype, head_dim 64/128) */
+       SLKV_PATH_TENSOR = 2 };                        /*   tcgen05 + TMA kernels (bf16, head_dim 128) */
+
+/* Shapes and options shared by slkv_score / slkv_compress. Strides are in elements. */
+typedef struct slkv_params {
+  int32_t n_seqs;          /* >= 1 */
+  int32_t n_q_heads;       /* multiple of n_kv_heads */
+  int32_t n_kv_heads;
+  int32_t head_dim;        /* 64 or 128 */
+  int32_t window;          /* w >= 1: observation window (last w tokens), always kept */
+  int32_t pool_kernel;     /* odd >= 1 (1 = no pooling) */
+  int32_t dtype;           /* SLKV_F32 | SLKV_BF16: element type of Q_win, K, V and the packed outputs */
+  int32_t pool_mode;       /* SLKV_POOL_MAX | SLKV_POOL_AVG */
+  int32_t softmax_domain;  /* SLKV_HISTORY */
+  int32_t score_path;      /* SLKV_PATH_AUTO picks TENSOR when the shape allows it, else SIMT */
+  int64_t k_stride_tok, k_stride_head;
+  int64_t v_stride_tok, v_stride_head;
+  int64_t q_stride_seq, q_stride_row, q_stride_head;
+} slkv_params;
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* slkv_strerror(int status);
+
+/* Last CUDA runtime error code seen by a call that returned SLKV_ERR_CUDA on this thread (0 = none). */
+int slkv_last_cuda_error(void);
+
+/*
+ * Stage-2 budget allocation (Sec. 3.3, Eq. 6; Algorithm 2).
+ *   inf_sc   dev, float[n_layers*n_heads], row-major (layer, head); INF_sc >= 0, finite
+ *   fixed    fixed part every head receives (= b_c (1 - 1/beta) in the paper's notation)
+ *   total    sum of all budgets (= b_c * n_layers * n_heads); dynamic pool D = total - N*fixed >= 0
+ *   budgets  dev, out, int32[n_layers*n_heads]
+ *   status   dev, optional: set to SLKV_ERR_NEG_INF_SC (budgets then left unwritten)
+ * Head (i, j) receives fixed + its share of D in proportion to Algorithm 2's weight
+ * (0.01 + L_i/L_s) * (inf_ij/L_s), L_i the layer's INF_sc sum, L_s the grand sum; shares are rounded by
+ * largest remainder (ties: lower index first) so that the budgets sum to `total` exactly.  All-zero
+ * INF_sc gives uniform shares.  fp64 arithmetic in a fixed order: results are reproducible bit for bit.
+ * Limits: n_layers <= 1024, n_layers*n_heads <= 16384, total - N*fixed < 2^52, budgets < 2^31.
+ */
+int slkv_alloc_budgets(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
+                       int32_t* budgets, int32_t* status, void* stream);
+
+/* Bytes of workspace slkv_score / slkv_compress need for these shapes (0 on invalid arguments).
+ * cu_seqlens_host: host, int32[n_seqs+1]. */
+size_t slkv_workspace_bytes(const slkv_params* p, const int32_t* cu_seqlens_host);
+
+/* Number of floats in the ragged `pooled` array: n_kv_heads * sum_s max(len_s - window, 0) (-1 on error). */
+int64_t slkv_pooled_elems(const slkv_params* p, const int32_t* cu_seqlens_host);
+
+/* Upper bound of packed rows for any budgets: n_kv_heads * total_tokens (-1 on error). */
+int64_t slkv_packed_rows_upper_bound(const slkv_params* p, const int32_t* cu_seqlens_host);
+
+/*
+ * Relevance scores (Sec. 3.4, Eq. 7; Algorithm 3 lines 4-6; scale and softmax axis from Eq. 3-4).
+ * For every sequence s, KV head g and history key j < n_hist_s:
+ *     vote[j]   = (1/G) * sum_{query heads h of group g} sum_{window rows i} softmax_j(q_i . k_j / sqrt(head_dim))
+ *     pooled[j] = max (or zero-padded mean) of vote over [j - pool_kernel/2, j + pool_kernel/2] within the history
+ * with the softmax taken over the history keys only.  (The paper leaves the reduction over the window
+ * rows, the GQA reduction and the pooling to prior work; this is the reading used here.)
+ *   q_win, k         dev, layouts above
+ *   cu_seqlens_dev   dev, int32[n_seqs+1];  cu_seqlens_host: the same values on the host (sizes the launch)
+ *   pooled           dev, out, float[slkv_pooled_elems]
+ * Accuracy: fp32 accumulation; relative error of pooled <= 1e-3 of the exact value.
+ */
+int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+               const int32_t* cu_seqlens_host, float* pooled, void* workspace, size_t workspace_bytes,
+               void* stream);
+
+/*
+ * KV entry selection and gather for one layer (Sec. 3.4, Eq. 8; Algorithm 3).
+ * For each segment (s, h) with budget C = budgets[h]:  kept = min(len_s, max(C, window)) rows survive:
+ * everything if len_s <= C (Alg. 3 l.1-3), else the window rows plus the kept - window history positions
+ * with the largest pooled score (ties: lower position first), in ascending position order (l.7-10).
+ *   budgets            dev, int32[n_kv_heads]: this layer's row of slkv_alloc_budgets' output
+ *   k_out, v_out       dev, out, [out_capacity_rows, head_dim] elements of p->dtype
+ *   offsets            dev, out, int32[n_seqs*n_kv_heads + 1]
+ *   kept_idx           dev, out, int32[out_capacity_rows]
+ *   pooled_opt         dev, optional out, float[slkv_pooled_elems]: the scores the selection used
+ *   status             dev, optional: SLKV_ERR_CAPACITY if offsets[last] > out_capacity_rows (rows beyond
+ *                      the capacity are then not written; offsets are still complete)
+ * Gathered rows are bit copies of the input rows.
+ */
+int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const void* v,
+                  const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
+                  void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx,
+                  float* pooled_opt, int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of device arena slkv_compress_host needs (inputs, outputs and workspace; 0 on invalid arguments). */
+size_t slkv_compress_host_arena_bytes(const slkv_params* p, const int32_t* cu_seqlens_host,
+                                      int64_t out_capacity_rows);
+
+/*
+ * slkv_compress for callers whose tensors live in host memory (Algorithm 3, same semantics).
+ * q_win, k, v, budgets are HOST inputs (dense layouts: the strides in `p` must describe contiguous
+ * [n_seqs, window, n_q_heads, head_dim] and [total_tokens, n_kv_heads, head_dim] arrays); k_out, v_out,
+ * offsets, kept_idx are HOST outputs.  `arena` is caller-owned DEVICE memory of at least
+ * slkv_compress_host_arena_bytes, 256-byte aligned.  The call copies the inputs to the arena, runs the
+ * kernels, copies offsets, kept_idx and the packed rows back and waits for `stream` before returning, so
+ * the outputs are valid on return.  Pinned host buffers make the copies asynchronous and fast; pageable
+ * ones work.  Returns SLKV_ERR_CAPACITY if out_capacity_rows is too small (nothing is copied back then
+ * except offsets).  *rows_out (optional) receives offsets[last].
+ */
+int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, const void* v,
+                       const int32_t* cu_seqlens_host, const int32_t* budgets, void* k_out, void* v_out,
+                       int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx, int64_t* rows_out,
+                       void* arena, size_t arena_bytes, void* stream);
+
+/* Number of kernels the most recent slkv_score / slkv_compress / slkv_compress_host call on this
+ * thread enqueued (launch accounting for benchmarks). */
+int slkv_last_launch_count(void);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int slkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLKV_H_ */

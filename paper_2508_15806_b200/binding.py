@@ -1,0 +1,188 @@
+"""ctypes binding of libslkv.so: the same entry points as include/slkv.h, argument marshalling only.
+
+Tensors are torch tensors (device memory and streams come from torch); every step of the method runs in
+the library's kernels.  There is no fallback: if the shared library is missing, lib() raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libslkv.so")
+
+SLKV_OK = 0
+ERR = {"NULL_PTR": -1, "BAD_SHAPE": -2, "BAD_DTYPE": -3, "BAD_ALIGN": -4, "BUDGET_SUM": -5, "NEG_INF_SC": -6,
+       "CAPACITY": -7, "WORKSPACE": -8, "CUDA": -9, "DEVICE_TIMEOUT": -10}
+SLKV_F32, SLKV_BF16 = 0, 1
+SLKV_POOL_MAX, SLKV_POOL_AVG = 0, 1
+SLKV_HISTORY = 0
+SLKV_PATH_AUTO, SLKV_PATH_SIMT, SLKV_PATH_TENSOR = 0, 1, 2
+
+
+class SlkvParams(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_seqs", "n_q_heads", "n_kv_heads", "head_dim", "window", "pool_kernel",
+                                         "dtype", "pool_mode", "softmax_domain", "score_path")] + \
+               [(n, C.c_int64) for n in ("k_stride_tok", "k_stride_head", "v_stride_tok", "v_stride_head",
+                                         "q_stride_seq", "q_stride_row", "q_stride_head")]
+
+
+class SlkvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().slkv_strerror(code).decode()
+        if code == ERR["CUDA"]:
+            msg += f" (cudaError {lib().slkv_last_cuda_error()})"
+        super().__init__(f"{where}: {msg}")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded shared library (loads it on first use; raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2508_15806_b200.build` "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32p, i64, i32, sz = C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_size_t
+        pp = C.POINTER(SlkvParams)
+        L.slkv_strerror.restype = C.c_char_p
+        L.slkv_strerror.argtypes = [C.c_int]
+        L.slkv_last_cuda_error.restype = C.c_int
+        L.slkv_last_launch_count.restype = C.c_int
+        L.slkv_version.restype = C.c_int
+        L.slkv_alloc_budgets.restype = C.c_int
+        L.slkv_alloc_budgets.argtypes = [vp, i32, i32, i32, i64, vp, vp, vp]
+        L.slkv_workspace_bytes.restype = sz
+        L.slkv_workspace_bytes.argtypes = [pp, i32p]
+        L.slkv_pooled_elems.restype = i64
+        L.slkv_pooled_elems.argtypes = [pp, i32p]
+        L.slkv_packed_rows_upper_bound.restype = i64
+        L.slkv_packed_rows_upper_bound.argtypes = [pp, i32p]
+        L.slkv_score.restype = C.c_int
+        L.slkv_score.argtypes = [pp, vp, vp, vp, i32p, vp, vp, sz, vp]
+        L.slkv_compress.restype = C.c_int
+        L.slkv_compress.argtypes = [pp, vp, vp, vp, vp, i32p, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+        L.slkv_compress_host_arena_bytes.restype = sz
+        L.slkv_compress_host_arena_bytes.argtypes = [pp, i32p, i64]
+        L.slkv_compress_host.restype = C.c_int
+        L.slkv_compress_host.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, i64, vp, vp, C.POINTER(C.c_int64),
+                                         vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _cu_host(cu_seqlens: Sequence[int]):
+    arr = (C.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
+    return arr
+
+
+def make_params(q_win: torch.Tensor, k: torch.Tensor, v: Optional[torch.Tensor], window: int, pool_kernel: int,
+                pool_mode: int = SLKV_POOL_MAX, score_path: int = SLKV_PATH_AUTO) -> SlkvParams:
+    """Shapes and strides from the tensors: q_win [n_seqs, w, Hq, d], k / v [T, Hkv, d] (last dim contiguous)."""
+    assert q_win.dim() == 4 and k.dim() == 3 and q_win.stride(3) == 1 and k.stride(2) == 1
+    if v is None:
+        v = k
+    dt = {torch.float32: SLKV_F32, torch.bfloat16: SLKV_BF16}[k.dtype]
+    assert q_win.dtype == k.dtype == v.dtype
+    return SlkvParams(n_seqs=q_win.shape[0], n_q_heads=q_win.shape[2], n_kv_heads=k.shape[1], head_dim=k.shape[2],
+                      window=window, pool_kernel=pool_kernel, dtype=dt, pool_mode=pool_mode,
+                      softmax_domain=SLKV_HISTORY, score_path=score_path,
+                      k_stride_tok=k.stride(0), k_stride_head=k.stride(1),
+                      v_stride_tok=v.stride(0), v_stride_head=v.stride(1),
+                      q_stride_seq=q_win.stride(0), q_stride_row=q_win.stride(1), q_stride_head=q_win.stride(2))
+
+
+def slkv_version() -> int:
+    return lib().slkv_version()
+
+
+def slkv_last_launch_count() -> int:
+    return lib().slkv_last_launch_count()
+
+
+def slkv_alloc_budgets(inf_sc: torch.Tensor, fixed: int, total: int, budgets: Optional[torch.Tensor] = None,
+                       status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """inf_sc: CUDA float32 [n_layers, n_heads] -> CUDA int32 budgets of the same shape."""
+    assert inf_sc.is_cuda and inf_sc.dtype == torch.float32 and inf_sc.dim() == 2 and inf_sc.is_contiguous()
+    if budgets is None:
+        budgets = torch.empty(inf_sc.shape, dtype=torch.int32, device=inf_sc.device)
+    rc = lib().slkv_alloc_budgets(inf_sc.data_ptr(), inf_sc.shape[0], inf_sc.shape[1], int(fixed), int(total),
+                                  budgets.data_ptr(), _ptr(status), _stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_alloc_budgets")
+    return budgets
+
+
+def slkv_workspace_bytes(params: SlkvParams, cu_seqlens: Sequence[int]) -> int:
+    return int(lib().slkv_workspace_bytes(C.byref(params), _cu_host(cu_seqlens)))
+
+
+def slkv_pooled_elems(params: SlkvParams, cu_seqlens: Sequence[int]) -> int:
+    return int(lib().slkv_pooled_elems(C.byref(params), _cu_host(cu_seqlens)))
+
+
+def slkv_packed_rows_upper_bound(params: SlkvParams, cu_seqlens: Sequence[int]) -> int:
+    return int(lib().slkv_packed_rows_upper_bound(C.byref(params), _cu_host(cu_seqlens)))
+
+
+def new_workspace(params: SlkvParams, cu_seqlens: Sequence[int], device) -> torch.Tensor:
+    n = slkv_workspace_bytes(params, cu_seqlens)
+    if n == 0:
+        raise SlkvError(ERR["BAD_SHAPE"], "slkv_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def slkv_score(params: SlkvParams, q_win: torch.Tensor, k: torch.Tensor, cu_dev: torch.Tensor,
+               cu_seqlens: Sequence[int], pooled: torch.Tensor, workspace: torch.Tensor, stream=None) -> torch.Tensor:
+    rc = lib().slkv_score(C.byref(params), q_win.data_ptr(), k.data_ptr(), cu_dev.data_ptr(), _cu_host(cu_seqlens),
+                          pooled.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_score")
+    return pooled
+
+
+def slkv_compress(params: SlkvParams, q_win, k, v, cu_dev, cu_seqlens: Sequence[int], budgets, k_out, v_out,
+                  offsets, kept_idx, workspace, pooled: Optional[torch.Tensor] = None,
+                  status: Optional[torch.Tensor] = None, stream=None) -> None:
+    rc = lib().slkv_compress(C.byref(params), q_win.data_ptr(), k.data_ptr(), v.data_ptr(), cu_dev.data_ptr(),
+                             _cu_host(cu_seqlens), budgets.data_ptr(), k_out.data_ptr(), v_out.data_ptr(),
+                             k_out.shape[0], offsets.data_ptr(), kept_idx.data_ptr(), _ptr(pooled), _ptr(status),
+                             workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_compress")
+
+
+def slkv_compress_host_arena_bytes(params: SlkvParams, cu_seqlens: Sequence[int], capacity_rows: int) -> int:
+    return int(lib().slkv_compress_host_arena_bytes(C.byref(params), _cu_host(cu_seqlens), int(capacity_rows)))
+
+
+def slkv_compress_host(params: SlkvParams, q_win, k, v, cu_seqlens: Sequence[int], budgets, k_out, v_out, offsets,
+                       kept_idx, arena: torch.Tensor, stream=None) -> int:
+    """All tensors except `arena` are HOST tensors (pinned for speed); returns the number of packed rows."""
+    for t in (q_win, k, v, budgets, k_out, v_out, offsets, kept_idx):
+        assert not t.is_cuda and t.is_contiguous()
+    assert arena.is_cuda
+    rows = C.c_int64(0)
+    rc = lib().slkv_compress_host(C.byref(params), q_win.data_ptr(), k.data_ptr(), v.data_ptr(), _cu_host(cu_seqlens),
+                                  budgets.data_ptr(), k_out.data_ptr(), v_out.data_ptr(), k_out.shape[0],
+                                  offsets.data_ptr(), kept_idx.data_ptr(), C.byref(rows), arena.data_ptr(),
+                                  arena.numel(), _stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_compress_host")
+    return int(rows.value)

@@ -1,0 +1,358 @@
+// extern "C" entry points of libslkv: argument validation, workspace carve-up, launch sequencing.
+// No step of the method runs here; every step is a kernel in the other translation units.
+#include <cstring>
+
+#include "slkv_internal.cuh"
+
+namespace slkv {
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+thread_local int g_last_launches = 0;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+constexpr int kMinChunkKeys = 256;     // no score path uses smaller chunks (sizes the partial buffers)
+constexpr int kMaxWindow = 256;
+constexpr size_t kSimtSmemLimit = 192 * 1024;
+
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return SLKV_ERR_CUDA;
+}
+
+struct Layout {
+  size_t hist_off, vote, pooled, part_m, part_z, flags, total;
+};
+
+// Validates p and cu_seqlens_host and fills the host-known fields of `pb`.
+int describe(const slkv_params* p, const int32_t* cu_host, Problem* pb) {
+  if (!p || !cu_host) return SLKV_ERR_NULL_PTR;
+  if (p->dtype != SLKV_F32 && p->dtype != SLKV_BF16) return SLKV_ERR_BAD_DTYPE;
+  if (p->pool_mode != SLKV_POOL_MAX && p->pool_mode != SLKV_POOL_AVG) return SLKV_ERR_BAD_DTYPE;
+  if (p->softmax_domain != SLKV_HISTORY) return SLKV_ERR_BAD_DTYPE;
+  if (p->score_path < SLKV_PATH_AUTO || p->score_path > SLKV_PATH_TENSOR) return SLKV_ERR_BAD_DTYPE;
+  if (p->n_seqs < 1 || p->n_seqs > (1 << 20)) return SLKV_ERR_BAD_SHAPE;
+  if (p->n_kv_heads < 1 || p->n_kv_heads > 65535 || p->n_q_heads < p->n_kv_heads ||
+      p->n_q_heads % p->n_kv_heads != 0)
+    return SLKV_ERR_BAD_SHAPE;
+  if (p->head_dim != 64 && p->head_dim != 128) return SLKV_ERR_BAD_SHAPE;
+  if (p->window < 1 || p->window > kMaxWindow) return SLKV_ERR_BAD_SHAPE;
+  if (p->pool_kernel < 1 || p->pool_kernel % 2 == 0 || p->pool_kernel > 1025) return SLKV_ERR_BAD_SHAPE;
+  const int elem = p->dtype == SLKV_F32 ? 4 : 2;
+  const int64_t row = p->head_dim;
+  if (p->k_stride_head < row || p->v_stride_head < row || p->q_stride_head < row ||
+      p->k_stride_tok < row || p->v_stride_tok < row || p->q_stride_row < row || p->q_stride_seq < row)
+    return SLKV_ERR_BAD_SHAPE;
+  const int64_t strides[] = {p->k_stride_tok, p->k_stride_head, p->v_stride_tok, p->v_stride_head,
+                             p->q_stride_seq, p->q_stride_row, p->q_stride_head};
+  for (int64_t s : strides)
+    if ((s * elem) % 16 != 0) return SLKV_ERR_BAD_ALIGN;
+  if (cu_host[0] != 0) return SLKV_ERR_BAD_SHAPE;
+  int64_t total_hist = 0;
+  int max_hist = 0;
+  for (int s = 0; s < p->n_seqs; ++s) {
+    int64_t len = (int64_t)cu_host[s + 1] - cu_host[s];
+    if (len < 0) return SLKV_ERR_BAD_SHAPE;
+    int64_t nh = len > p->window ? len - p->window : 0;
+    total_hist += nh;
+    if (nh > max_hist) max_hist = (int)nh;
+  }
+  const int64_t T = cu_host[p->n_seqs];
+  if ((int64_t)p->n_kv_heads * T >= (1ll << 31)) return SLKV_ERR_BAD_SHAPE;
+  std::memset(pb, 0, sizeof(*pb));
+  pb->p = *p;
+  pb->G = p->n_q_heads / p->n_kv_heads;
+  pb->R = pb->G * p->window;
+  pb->elem = elem;
+  pb->max_hist = max_hist;
+  pb->total_tokens = T;
+  pb->total_hist = total_hist;
+  pb->n_seg = p->n_seqs * p->n_kv_heads;
+  if (pb->n_seg > 65535 * 16) return SLKV_ERR_BAD_SHAPE;
+  if (pb->R > 1024) return SLKV_ERR_BAD_SHAPE;
+  return SLKV_OK;
+}
+
+Layout layout_of(const Problem& pb) {
+  Layout L;
+  size_t o = 0;
+  L.hist_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int64_t));
+  const size_t votes = (size_t)pb.p.n_kv_heads * (size_t)pb.total_hist * sizeof(float);
+  L.vote = o; o = align_up(o + votes);
+  L.pooled = o; o = align_up(o + votes);
+  const size_t nchunks = (size_t)(pb.max_hist + kMinChunkKeys - 1) / kMinChunkKeys + 1;
+  const size_t parts = (size_t)pb.n_seg * pb.R * nchunks * sizeof(float);
+  L.part_m = o; o = align_up(o + parts);
+  L.part_z = o; o = align_up(o + parts);
+  L.flags = o; o = align_up(o + 8 * sizeof(int32_t));
+  L.total = o;
+  return L;
+}
+
+// Picks the score path; SLKV_ERR_* when the requested one cannot take the shape.
+int resolve_path(const Problem& pb, int* path) {
+  int want = pb.p.score_path;
+  const bool tensor_ok = tensor_path_supported(pb.p);
+  if (want == SLKV_PATH_AUTO) want = tensor_ok ? SLKV_PATH_TENSOR : SLKV_PATH_SIMT;
+  if (want == SLKV_PATH_TENSOR && !tensor_ok) return SLKV_ERR_BAD_DTYPE;
+  if (want == SLKV_PATH_SIMT && simt_smem_bytes(pb) > kSimtSmemLimit) return SLKV_ERR_BAD_SHAPE;
+  *path = want;
+  return SLKV_OK;
+}
+
+int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path) {
+  if (!ws) return SLKV_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(ws) % kAlign != 0) return SLKV_ERR_BAD_ALIGN;
+  Layout L = layout_of(*pb);
+  if (ws_bytes < L.total) return SLKV_ERR_WORKSPACE;
+  unsigned char* b = static_cast<unsigned char*>(ws);
+  pb->hist_off = reinterpret_cast<int64_t*>(b + L.hist_off);
+  pb->vote = reinterpret_cast<float*>(b + L.vote);
+  pb->pooled_ws = reinterpret_cast<float*>(b + L.pooled);
+  pb->part_m = reinterpret_cast<float*>(b + L.part_m);
+  pb->part_z = reinterpret_cast<float*>(b + L.part_z);
+  pb->dev_flags = reinterpret_cast<int32_t*>(b + L.flags);
+  pb->chunk_keys = path == SLKV_PATH_TENSOR ? tensor_chunk_keys(*pb) : simt_chunk_keys();
+  pb->n_chunks = (pb->max_hist + pb->chunk_keys - 1) / pb->chunk_keys;
+  if (pb->n_chunks < 1) pb->n_chunks = 1;
+  return SLKV_OK;
+}
+
+bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
+// score -> pooled (device pointers resolved); shared by slkv_score and slkv_compress
+int enqueue_score(const Problem& pb, int path, float* pooled, cudaStream_t st, int* launches) {
+  cudaError_t e = path == SLKV_PATH_TENSOR ? launch_score_tensor(pb, st, launches)
+                                           : launch_score_simt(pb, st, launches);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_pool(pb, pooled, st, launches);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return SLKV_OK;
+}
+
+int compress_impl(const slkv_params* p, const void* q_win, const void* k, const void* v, const int32_t* cu_dev,
+                  const int32_t* cu_host, const int32_t* budgets, void* k_out, void* v_out, int64_t capacity,
+                  int32_t* offsets, int32_t* kept_idx, float* pooled_opt, int32_t* status, void* ws,
+                  size_t ws_bytes, cudaStream_t st) {
+  g_last_launches = 0;
+  if (!q_win || !k || !v || !cu_dev || !budgets || !k_out || !v_out || !offsets || !kept_idx)
+    return SLKV_ERR_NULL_PTR;
+  Problem pb;
+  int rc = describe(p, cu_host, &pb);
+  if (rc != SLKV_OK) return rc;
+  if (capacity < 0) return SLKV_ERR_CAPACITY;
+  if (!aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
+    return SLKV_ERR_BAD_ALIGN;
+  int path = 0;
+  rc = resolve_path(pb, &path);
+  if (rc != SLKV_OK) return rc;
+  rc = bind_workspace(&pb, ws, ws_bytes, path);
+  if (rc != SLKV_OK) return rc;
+  pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
+  int launches = 0;
+  cudaError_t e = launch_setup(pb, budgets, offsets, capacity, status, st, &launches);
+  if (e != cudaSuccess) return cuda_fail(e);
+  float* pooled = pooled_opt ? pooled_opt : pb.pooled_ws;
+  rc = enqueue_score(pb, path, pooled, st, &launches);
+  if (rc != SLKV_OK) return rc;
+  e = launch_select(pb, pooled, budgets, offsets, kept_idx, capacity, st, &launches);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_gather(pb, offsets, kept_idx, k_out, v_out, capacity, st, &launches);
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_last_launches = launches;
+  return SLKV_OK;
+}
+
+}  // namespace
+}  // namespace slkv
+
+using namespace slkv;
+
+extern "C" {
+
+const char* slkv_strerror(int status) {
+  switch (status) {
+    case SLKV_OK: return "SLKV_OK";
+    case SLKV_ERR_NULL_PTR: return "SLKV_ERR_NULL_PTR: a required pointer is NULL";
+    case SLKV_ERR_BAD_SHAPE: return "SLKV_ERR_BAD_SHAPE: size, count or stride out of range";
+    case SLKV_ERR_BAD_DTYPE: return "SLKV_ERR_BAD_DTYPE: unknown or unsupported dtype / mode / path";
+    case SLKV_ERR_BAD_ALIGN: return "SLKV_ERR_BAD_ALIGN: pointer or stride not 16-byte aligned";
+    case SLKV_ERR_BUDGET_SUM: return "SLKV_ERR_BUDGET_SUM: total smaller than heads * fixed";
+    case SLKV_ERR_NEG_INF_SC: return "SLKV_ERR_NEG_INF_SC: INF_sc negative or not finite";
+    case SLKV_ERR_CAPACITY: return "SLKV_ERR_CAPACITY: packed output capacity too small";
+    case SLKV_ERR_WORKSPACE: return "SLKV_ERR_WORKSPACE: workspace missing or too small";
+    case SLKV_ERR_CUDA: return "SLKV_ERR_CUDA: a CUDA runtime call failed";
+    case SLKV_ERR_DEVICE_TIMEOUT: return "SLKV_ERR_DEVICE_TIMEOUT: a bounded device-side wait ran out";
+    default: return "unknown slkv status";
+  }
+}
+
+int slkv_last_cuda_error(void) { return g_last_cuda_error; }
+int slkv_last_launch_count(void) { return g_last_launches; }
+int slkv_version(void) { return 100; }
+
+int slkv_alloc_budgets(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
+                       int32_t* budgets, int32_t* status, void* stream) {
+  if (!inf_sc || !budgets) return SLKV_ERR_NULL_PTR;
+  if (n_layers < 1 || n_heads < 1 || n_layers > 1024 || (int64_t)n_layers * n_heads > 16384)
+    return SLKV_ERR_BAD_SHAPE;
+  if (fixed < 0 || total < (int64_t)n_layers * n_heads * fixed) return SLKV_ERR_BUDGET_SUM;
+  if (total > 0x7fffffffll) return SLKV_ERR_BAD_SHAPE;
+  cudaError_t e = launch_alloc(inf_sc, n_layers, n_heads, fixed, total, budgets, status, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return SLKV_OK;
+}
+
+size_t slkv_workspace_bytes(const slkv_params* p, const int32_t* cu_seqlens_host) {
+  Problem pb;
+  if (describe(p, cu_seqlens_host, &pb) != SLKV_OK) return 0;
+  return layout_of(pb).total;
+}
+
+int64_t slkv_pooled_elems(const slkv_params* p, const int32_t* cu_seqlens_host) {
+  Problem pb;
+  if (describe(p, cu_seqlens_host, &pb) != SLKV_OK) return -1;
+  return (int64_t)pb.p.n_kv_heads * pb.total_hist;
+}
+
+int64_t slkv_packed_rows_upper_bound(const slkv_params* p, const int32_t* cu_seqlens_host) {
+  Problem pb;
+  if (describe(p, cu_seqlens_host, &pb) != SLKV_OK) return -1;
+  return (int64_t)pb.p.n_kv_heads * pb.total_tokens;
+}
+
+int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+               const int32_t* cu_seqlens_host, float* pooled, void* workspace, size_t workspace_bytes,
+               void* stream) {
+  g_last_launches = 0;
+  if (!q_win || !k || !cu_seqlens_dev || !pooled) return SLKV_ERR_NULL_PTR;
+  Problem pb;
+  int rc = describe(p, cu_seqlens_host, &pb);
+  if (rc != SLKV_OK) return rc;
+  if (!aligned16(q_win) || !aligned16(k)) return SLKV_ERR_BAD_ALIGN;
+  int path = 0;
+  rc = resolve_path(pb, &path);
+  if (rc != SLKV_OK) return rc;
+  rc = bind_workspace(&pb, workspace, workspace_bytes, path);
+  if (rc != SLKV_OK) return rc;
+  pb.cu = cu_seqlens_dev; pb.q = q_win; pb.k = k; pb.v = nullptr;
+  cudaStream_t st = (cudaStream_t)stream;
+  int launches = 0;
+  cudaError_t e = launch_setup(pb, nullptr, nullptr, 0, nullptr, st, &launches);
+  if (e != cudaSuccess) return cuda_fail(e);
+  rc = enqueue_score(pb, path, pooled, st, &launches);
+  if (rc != SLKV_OK) return rc;
+  g_last_launches = launches;
+  return SLKV_OK;
+}
+
+int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const void* v,
+                  const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
+                  void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx,
+                  float* pooled_opt, int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
+  return compress_impl(p, q_win, k, v, cu_seqlens_dev, cu_seqlens_host, budgets, k_out, v_out, out_capacity_rows,
+                       offsets, kept_idx, pooled_opt, status, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+// ---- host-buffer variant ---------------------------------------------------------------------------
+namespace {
+struct HostArena {
+  size_t q, k, v, cu, budgets, k_out, v_out, offsets, kept, status, ws, total;
+};
+bool host_arena_layout(const Problem& pb, int64_t capacity, HostArena* A) {
+  const slkv_params& p = pb.p;
+  const size_t e = pb.elem, d = p.head_dim;
+  size_t o = 0;
+  A->q = o; o = align_up(o + (size_t)p.n_seqs * p.window * p.n_q_heads * d * e);
+  A->k = o; o = align_up(o + (size_t)pb.total_tokens * p.n_kv_heads * d * e);
+  A->v = o; o = align_up(o + (size_t)pb.total_tokens * p.n_kv_heads * d * e);
+  A->cu = o; o = align_up(o + (size_t)(p.n_seqs + 1) * 4);
+  A->budgets = o; o = align_up(o + (size_t)p.n_kv_heads * 4);
+  A->k_out = o; o = align_up(o + (size_t)capacity * d * e);
+  A->v_out = o; o = align_up(o + (size_t)capacity * d * e);
+  A->offsets = o; o = align_up(o + (size_t)(pb.n_seg + 1) * 4);
+  A->kept = o; o = align_up(o + (size_t)capacity * 4);
+  A->status = o; o = align_up(o + 4);
+  A->ws = o; o = align_up(o + layout_of(pb).total);
+  A->total = o;
+  return true;
+}
+bool dense_strides(const slkv_params& p) {
+  const int64_t d = p.head_dim;
+  return p.k_stride_head == d && p.k_stride_tok == d * p.n_kv_heads && p.v_stride_head == d &&
+         p.v_stride_tok == d * p.n_kv_heads && p.q_stride_head == d && p.q_stride_row == d * p.n_q_heads &&
+         p.q_stride_seq == d * p.n_q_heads * p.window;
+}
+}  // namespace
+
+size_t slkv_compress_host_arena_bytes(const slkv_params* p, const int32_t* cu_seqlens_host,
+                                      int64_t out_capacity_rows) {
+  Problem pb;
+  if (describe(p, cu_seqlens_host, &pb) != SLKV_OK || out_capacity_rows < 0) return 0;
+  HostArena A;
+  host_arena_layout(pb, out_capacity_rows, &A);
+  return A.total;
+}
+
+int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, const void* v,
+                       const int32_t* cu_seqlens_host, const int32_t* budgets, void* k_out, void* v_out,
+                       int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx, int64_t* rows_out,
+                       void* arena, size_t arena_bytes, void* stream) {
+  g_last_launches = 0;
+  if (!q_win || !k || !v || !budgets || !k_out || !v_out || !offsets || !kept_idx || !arena)
+    return SLKV_ERR_NULL_PTR;
+  Problem pb;
+  int rc = describe(p, cu_seqlens_host, &pb);
+  if (rc != SLKV_OK) return rc;
+  if (!dense_strides(*p)) return SLKV_ERR_BAD_SHAPE;
+  if (out_capacity_rows < 0) return SLKV_ERR_CAPACITY;
+  if (reinterpret_cast<uintptr_t>(arena) % kAlign != 0) return SLKV_ERR_BAD_ALIGN;
+  HostArena A;
+  host_arena_layout(pb, out_capacity_rows, &A);
+  if (arena_bytes < A.total) return SLKV_ERR_WORKSPACE;
+  // rows that will be written, known on the host because the budgets are (Algorithm 3 l.1-4, l.7)
+  int64_t rows = 0;
+  for (int s = 0; s < p->n_seqs; ++s) {
+    const int64_t len = cu_seqlens_host[s + 1] - cu_seqlens_host[s];
+    for (int h = 0; h < p->n_kv_heads; ++h) {
+      int64_t c = budgets[h] > p->window ? budgets[h] : p->window;
+      rows += len < c ? len : c;
+    }
+  }
+  if (rows_out) *rows_out = rows;
+  if (rows > out_capacity_rows) return SLKV_ERR_CAPACITY;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned char* b = static_cast<unsigned char*>(arena);
+  const size_t e = pb.elem, d = p->head_dim;
+  cudaError_t ce;
+#define SLKV_CP(dst, src, n, kind)                                  \
+  do {                                                              \
+    if ((n) > 0) {                                                  \
+      ce = cudaMemcpyAsync((dst), (src), (n), (kind), st);          \
+      if (ce != cudaSuccess) return cuda_fail(ce);                  \
+    }                                                               \
+  } while (0)
+  SLKV_CP(b + A.q, q_win, (size_t)p->n_seqs * p->window * p->n_q_heads * d * e, cudaMemcpyHostToDevice);
+  SLKV_CP(b + A.k, k, (size_t)pb.total_tokens * p->n_kv_heads * d * e, cudaMemcpyHostToDevice);
+  SLKV_CP(b + A.v, v, (size_t)pb.total_tokens * p->n_kv_heads * d * e, cudaMemcpyHostToDevice);
+  SLKV_CP(b + A.cu, cu_seqlens_host, (size_t)(p->n_seqs + 1) * 4, cudaMemcpyHostToDevice);
+  SLKV_CP(b + A.budgets, budgets, (size_t)p->n_kv_heads * 4, cudaMemcpyHostToDevice);
+  rc = compress_impl(p, b + A.q, b + A.k, b + A.v, reinterpret_cast<int32_t*>(b + A.cu), cu_seqlens_host,
+                     reinterpret_cast<int32_t*>(b + A.budgets), b + A.k_out, b + A.v_out, out_capacity_rows,
+                     reinterpret_cast<int32_t*>(b + A.offsets), reinterpret_cast<int32_t*>(b + A.kept), nullptr,
+                     nullptr, b + A.ws, arena_bytes - A.ws, st);
+  if (rc != SLKV_OK) return rc;
+  SLKV_CP(offsets, b + A.offsets, (size_t)(pb.n_seg + 1) * 4, cudaMemcpyDeviceToHost);
+  SLKV_CP(kept_idx, b + A.kept, (size_t)rows * 4, cudaMemcpyDeviceToHost);
+  SLKV_CP(k_out, b + A.k_out, (size_t)rows * d * e, cudaMemcpyDeviceToHost);
+  SLKV_CP(v_out, b + A.v_out, (size_t)rows * d * e, cudaMemcpyDeviceToHost);
+#undef SLKV_CP
+  ce = cudaStreamSynchronize(st);
+  if (ce != cudaSuccess) return cuda_fail(ce);
+  return SLKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,58 @@
+// Internal declarations shared by the translation units of libslkv (not part of the public ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "slkv.h"
+
+namespace slkv {
+
+constexpr double kLayerFloor = 0.01;   // minimum layer budget (Sec. 3.3)
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Everything a score / select / gather launch needs, resolved by the host entry points.
+struct Problem {
+  slkv_params p;
+  int G;                  // query heads per KV head
+  int R;                  // score rows per KV head = G * window
+  int elem;               // bytes per element
+  int max_hist;           // max_s n_hist_s
+  int64_t total_tokens;
+  int64_t total_hist;     // sum_s n_hist_s
+  int n_seg;              // n_seqs * n_kv_heads
+  const int32_t* cu;      // dev
+  const void* q;          // dev
+  const void* k;          // dev
+  const void* v;          // dev
+  // workspace carve-up (dev)
+  int64_t* hist_off;      // [n_seqs+1] exclusive prefix of n_hist_s
+  float* vote;            // [n_kv_heads * total_hist] ragged, same layout as pooled
+  float* part_m;          // [n_seg][R][n_chunks] partial row maxima (log2 domain)
+  float* part_z;          // [n_seg][R][n_chunks] partial row sums
+  int n_chunks;           // chunks per segment (stride of part_*), per score path
+  int chunk_keys;         // keys per chunk
+  float* pooled_ws;       // [n_kv_heads * total_hist] used when the caller wants no pooled output
+  int32_t* dev_flags;     // [8] scratch words (timeouts etc.)
+};
+
+// host-side launchers; each returns a cudaError_t and adds to *launches
+cudaError_t launch_alloc(const float* inf, int n_layers, int n_heads, int fixed, long long total, int32_t* budgets,
+                         int32_t* status, cudaStream_t st);
+cudaError_t launch_setup(const Problem& pb, const int32_t* budgets, int32_t* offsets, int64_t capacity,
+                         int32_t* status, cudaStream_t st, int* launches);
+int simt_chunk_keys();
+size_t simt_smem_bytes(const Problem& pb);
+cudaError_t launch_score_simt(const Problem& pb, cudaStream_t st, int* launches);
+bool tensor_path_supported(const slkv_params& p);
+int tensor_chunk_keys(const Problem& pb);
+cudaError_t launch_score_tensor(const Problem& pb, cudaStream_t st, int* launches);
+cudaError_t launch_pool(const Problem& pb, float* pooled, cudaStream_t st, int* launches);
+cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t* budgets, const int32_t* offsets,
+                          int32_t* kept_idx, int64_t capacity, cudaStream_t st, int* launches);
+cudaError_t launch_gather(const Problem& pb, const int32_t* offsets, const int32_t* kept_idx, void* k_out,
+                          void* v_out, int64_t capacity, cudaStream_t st, int* launches);
+
+}  // namespace slkv

@@ -1,0 +1,212 @@
+// Window relevance scores with fp32 FMA arithmetic (Sec. 3.4, Eq. 7; Algorithm 3 l.6; Eq. 3-4).
+//
+// Serves the fp32 configuration and every shape the tensor-core kernels do not take.  One thread owns
+// one history key (its row of K lives in registers), the G*w query rows of the KV head's group sit in
+// shared memory, and a CTA walks a chunk of key tiles:
+//   pass 1  per query row: running max and sum of 2^(s - max) over the chunk's keys -> part_m / part_z
+//   pass 2  merges the chunks' partials into the row's log-sum-exp, then per key
+//           vote[j] = (1/G) sum_rows 2^(s_rj - lse_r)      (s in log2 units: s = q.k * log2(e)/sqrt(d))
+// The w x n_hist probability matrix never exists in memory.
+#include "slkv_internal.cuh"
+
+namespace slkv {
+namespace {
+
+constexpr int kThreads = 128;          // keys per tile
+constexpr int kTilesPerChunk = 8;      // key tiles a CTA walks
+constexpr int kRowBatch = 8;           // query rows reduced together in pass 1
+
+template <typename T> struct Vec;      // 16-byte vector of T
+template <> struct Vec<float> { static constexpr int N = 4; };
+template <> struct Vec<__nv_bfloat16> { static constexpr int N = 8; };
+
+__device__ __forceinline__ void unpack(const uint4& u, float (&f)[4], float) {
+  f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+}
+__device__ __forceinline__ void unpack(const uint4& u, float (&f)[8], __nv_bfloat16) {
+  // a bf16 is the high half of an fp32
+  f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+  f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+  f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
+  f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+}
+
+template <typename T, int D>
+__device__ __forceinline__ float dot_row(const T* __restrict__ qrow /*smem*/, const float (&kreg)[D]) {
+  constexpr int VN = Vec<T>::N;
+  float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+  for (int c = 0; c < D / VN; ++c) {
+    uint4 u = *reinterpret_cast<const uint4*>(qrow + c * VN);
+    float f[VN];
+    unpack(u, f, T());
+#pragma unroll
+    for (int e = 0; e < VN; e += 2) {
+      acc0 = fmaf(f[e], kreg[c * VN + e], acc0);
+      acc1 = fmaf(f[e + 1], kreg[c * VN + e + 1], acc1);
+    }
+  }
+  return acc0 + acc1;
+}
+
+template <typename T, int D, int PASS>
+__global__ void __launch_bounds__(kThreads)
+k_score_simt(const T* __restrict__ q, const T* __restrict__ k, const int32_t* __restrict__ cu,
+             const int64_t* __restrict__ hist_off, float* __restrict__ part_m, float* __restrict__ part_z,
+             float* __restrict__ vote, int n_kv_heads, int G, int window, int n_chunks, long long k_stride_tok,
+             long long k_stride_head, long long q_stride_seq, long long q_stride_row, long long q_stride_head,
+             float scale_log2) {
+  constexpr int VN = Vec<T>::N;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int R = G * window;
+  T* qs = reinterpret_cast<T*>(smem_raw);                               // [R][D]
+  float* fbuf = reinterpret_cast<float*>(smem_raw + (size_t)R * D * sizeof(T));
+  float* run_m = fbuf;                                                  // [R]  (pass 2: lse per row)
+  float* run_z = fbuf + R;                                              // [R]
+  float* wred = fbuf + 2 * R;                                           // [2][kRowBatch][4]
+
+  const int chunk = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int t0 = cu[s];
+  const int n_hist = max(cu[s + 1] - t0 - window, 0);
+  const int key0 = chunk * (kThreads * kTilesPerChunk);
+  if (key0 >= n_hist) return;
+  const int seg = s * n_kv_heads + g;
+
+  // the group's query rows: row r = hh*window + i  <->  query head g*G + hh, window row i
+  for (int idx = tid; idx < R * (D / VN); idx += kThreads) {
+    int r = idx / (D / VN), c = idx - r * (D / VN);
+    int hh = r / window, i = r - hh * window;
+    const T* src = q + s * q_stride_seq + i * q_stride_row + (long long)(g * G + hh) * q_stride_head + c * VN;
+    *reinterpret_cast<uint4*>(qs + r * D + c * VN) = *reinterpret_cast<const uint4*>(src);
+  }
+  if (PASS == 1) {
+    for (int r = tid; r < R; r += kThreads) { run_m[r] = -INFINITY; run_z[r] = 0.f; }
+  } else {
+    const int nc = (n_hist + kThreads * kTilesPerChunk - 1) / (kThreads * kTilesPerChunk);
+    for (int r = tid; r < R; r += kThreads) {
+      const float* pm = part_m + ((long long)seg * R + r) * n_chunks;
+      const float* pz = part_z + ((long long)seg * R + r) * n_chunks;
+      float M = -INFINITY;
+      for (int c = 0; c < nc; ++c) M = fmaxf(M, pm[c]);
+      float Z = 0.f;
+      for (int c = 0; c < nc; ++c) Z += pz[c] * exp2f(pm[c] - M);
+      run_m[r] = M + log2f(Z);
+    }
+  }
+  __syncthreads();
+
+  for (int tile = 0; tile < kTilesPerChunk; ++tile) {
+    const int j = key0 + tile * kThreads + tid;
+    if (key0 + tile * kThreads >= n_hist) break;
+    const bool valid = j < n_hist;
+    float kreg[D];
+    {
+      const T* krow = k + (long long)(t0 + (valid ? j : 0)) * k_stride_tok + (long long)g * k_stride_head;
+#pragma unroll
+      for (int c = 0; c < D / VN; ++c) {
+        uint4 u = *reinterpret_cast<const uint4*>(krow + c * VN);
+        float f[VN];
+        unpack(u, f, T());
+#pragma unroll
+        for (int e = 0; e < VN; ++e) kreg[c * VN + e] = f[e];
+      }
+    }
+    if (PASS == 1) {
+      for (int r0 = 0; r0 < R; r0 += kRowBatch) {
+        float sv[kRowBatch], bm[kRowBatch];
+#pragma unroll
+        for (int b = 0; b < kRowBatch; ++b) {
+          int r = min(r0 + b, R - 1);
+          float d = dot_row<T, D>(qs + r * D, kreg) * scale_log2;
+          sv[b] = valid ? d : -INFINITY;
+          float m = sv[b];
+          for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+          if (lane == 0) wred[b * 4 + wid] = m;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int b = 0; b < kRowBatch; ++b) {
+          bm[b] = fmaxf(fmaxf(wred[b * 4], wred[b * 4 + 1]), fmaxf(wred[b * 4 + 2], wred[b * 4 + 3]));
+          float e = exp2f(sv[b] - bm[b]);
+          for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+          if (lane == 0) wred[kRowBatch * 4 + b * 4 + wid] = e;
+        }
+        __syncthreads();
+        if (tid < kRowBatch && r0 + tid < R) {
+          const int r = r0 + tid;
+          const float* ws = wred + kRowBatch * 4 + tid * 4;
+          float bs = (ws[0] + ws[1]) + (ws[2] + ws[3]);
+          const float* wm = wred + tid * 4;                 // the batch's warp maxima are still in place
+          float tm = fmaxf(fmaxf(wm[0], wm[1]), fmaxf(wm[2], wm[3]));
+          float om = run_m[r], nm = fmaxf(om, tm);
+          run_z[r] = run_z[r] * exp2f(om - nm) + bs * exp2f(tm - nm);
+          run_m[r] = nm;
+        }
+        __syncthreads();
+      }
+    } else {
+      float acc = 0.f;
+      for (int r = 0; r < R; ++r) acc += exp2f(dot_row<T, D>(qs + r * D, kreg) * scale_log2 - run_m[r]);
+      if (valid) vote[hist_off[s] * n_kv_heads + (long long)g * n_hist + j] = acc / (float)G;
+    }
+  }
+  if (PASS == 1) {
+    __syncthreads();
+    for (int r = tid; r < R; r += kThreads) {
+      part_m[((long long)seg * R + r) * n_chunks + chunk] = run_m[r];
+      part_z[((long long)seg * R + r) * n_chunks + chunk] = run_z[r];
+    }
+  }
+}
+
+template <typename T, int D>
+cudaError_t launch_both(const Problem& pb, cudaStream_t st, int* launches) {
+  const size_t smem = simt_smem_bytes(pb);
+  static thread_local int configured_dev = -1;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (configured_dev != dev) {
+    e = cudaFuncSetAttribute(k_score_simt<T, D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_score_simt<T, D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    configured_dev = dev;
+  }
+  const int chunk_keys = kThreads * kTilesPerChunk;
+  dim3 grid((pb.max_hist + chunk_keys - 1) / chunk_keys, pb.p.n_kv_heads, pb.p.n_seqs);
+  const float scale_log2 = kLog2e / sqrtf((float)pb.p.head_dim);
+  const slkv_params& p = pb.p;
+  k_score_simt<T, D, 1><<<grid, kThreads, smem, st>>>(
+      (const T*)pb.q, (const T*)pb.k, pb.cu, pb.hist_off, pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G,
+      p.window, pb.n_chunks, p.k_stride_tok, p.k_stride_head, p.q_stride_seq, p.q_stride_row, p.q_stride_head,
+      scale_log2);
+  ++*launches;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  k_score_simt<T, D, 2><<<grid, kThreads, smem, st>>>(
+      (const T*)pb.q, (const T*)pb.k, pb.cu, pb.hist_off, pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G,
+      p.window, pb.n_chunks, p.k_stride_tok, p.k_stride_head, p.q_stride_seq, p.q_stride_row, p.q_stride_head,
+      scale_log2);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+int simt_chunk_keys() { return kThreads * kTilesPerChunk; }
+
+size_t simt_smem_bytes(const Problem& pb) {
+  return (size_t)pb.R * pb.p.head_dim * pb.elem + (size_t)(2 * pb.R + 2 * kRowBatch * 4) * sizeof(float);
+}
+
+cudaError_t launch_score_simt(const Problem& pb, cudaStream_t st, int* launches) {
+  if (pb.max_hist <= 0) return cudaSuccess;
+  const bool bf = pb.p.dtype == SLKV_BF16;
+  if (pb.p.head_dim == 64)
+    return bf ? launch_both<__nv_bfloat16, 64>(pb, st, launches) : launch_both<float, 64>(pb, st, launches);
+  return bf ? launch_both<__nv_bfloat16, 128>(pb, st, launches) : launch_both<float, 128>(pb, st, launches);
+}
+
+}  // namespace slkv
