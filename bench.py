@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the prefill KV-compression step:  python bench.py [--gpus N] [--steps K] [--warmup W]
+
+One step = the whole hot path (window scores -> pooling -> per-head top-k -> packed K/V gather) for every
+layer of the workload, budgets precomputed once by slkv_alloc_budgets (they are per model, not per step).
+Workload at N=1: the 32k-context Llama-3-8B-shaped configuration (32 layers, 32 query / 8 KV heads,
+head_dim 128, window 32, pool 7, average budget 512 per KV head), synthetic seeded inputs resident in HBM.
+Every layer has its own Q/K/V (4.3 GB in total, far larger than L2), so K is really streamed from HBM.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2508_15806_b200 import synth  # noqa: E402
+
+METRIC = "context tokens compressed per second per layer"
+UNIT = "tokens/s/layer"
+WORKLOAD_INDEX = 2          # configs[2]: the 32k-context, 32-layer configuration the target is quoted on
+TOTAL_INDEX = 1             # average budget 512 per KV head
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ---------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons of the bench's GPU through NVML while the timed loops run."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            props = torch.cuda.get_device_properties(device_index)
+            try:
+                bus = "%08x:%02x:%02x.0" % (props.pci_domain_id, props.pci_bus_id, props.pci_device_id)
+                self.h = pynvml.nvmlDeviceGetHandleByPciBusId(bus.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.nv = pynvml
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._stop.clear()
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        if self._thr is not None:
+            self._stop.set()
+            self._thr.join()
+            self._thr = None
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------------------------------
+def rows_of_layer(lens, budgets_row, window):
+    return sum(min(n, max(int(c), window)) for n in lens for c in budgets_row)
+
+
+def run_cuda(args):
+    from paper_2508_15806_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()
+
+    wl = synth.workloads()[WORKLOAD_INDEX]
+    if args.layers:
+        wl = synth.small_variant(wl, wl.seq_lens, n_layers=args.layers,
+                                 totals=[t // 32 * args.layers for t in wl.totals])
+    if world > 1:
+        wl.seed = wl.seed + 1000 * rank          # weak scaling: every rank compresses its own sequence
+    total = wl.totals[TOTAL_INDEX]
+    cu = wl.cu_seqlens
+    T, nl, hkv, d, w = wl.total_tokens, wl.n_layers, wl.n_kv_heads, wl.head_dim, wl.window
+    e = wl.elem_size
+
+    # budgets: once per model, on the GPU
+    inf = synth.inf_sc(wl).to(dev)
+    budgets = B.slkv_alloc_budgets(inf, wl.fixed, total)
+    torch.cuda.synchronize()
+    budgets_host = budgets.cpu()
+    assert int(budgets_host.sum()) == total
+
+    layers = []
+    cu_dev = torch.tensor(cu, dtype=torch.int32, device=dev)
+    params = None
+    for l in range(nl):
+        x = synth.layer_inputs(wl, l, device=dev)
+        if params is None:
+            params = B.make_params(x.q_win, x.k, x.v, w, wl.pool_kernel)
+        rows = rows_of_layer(wl.seq_lens, budgets_host[l].tolist(), w)
+        layers.append({"q": x.q_win, "k": x.k, "v": x.v, "rows": rows, "bud": budgets[l].contiguous(),
+                       "k_out": torch.empty(rows, d, dtype=wl.torch_dtype, device=dev),
+                       "v_out": torch.empty(rows, d, dtype=wl.torch_dtype, device=dev),
+                       "offsets": torch.empty(len(wl.seq_lens) * hkv + 1, dtype=torch.int32, device=dev),
+                       "kept": torch.empty(rows, dtype=torch.int32, device=dev)})
+    ws = B.new_workspace(params, cu, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    launches_per_step = 0
+
+    def step():
+        nonlocal launches_per_step
+        n = 0
+        for L in layers:
+            B.slkv_compress(params, L["q"], L["k"], L["v"], cu_dev, cu, L["bud"], L["k_out"], L["v_out"],
+                            L["offsets"], L["kept"], ws, None, status, stream)
+            n += B.slkv_last_launch_count()
+        launches_per_step = n
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(n_steps, fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        a.record(stream)
+        for _ in range(n_steps):
+            fn()
+        b.record(stream)
+        barrier()
+        ms = a.elapsed_time(b)
+        if dist is not None:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "device status word set during warm-up"
+    steps = args.steps
+    if steps is None:                                   # aim at ~3 s of timed work
+        one = timed(1, step)
+        steps = int(min(2000, max(10, 3000.0 / max(one, 1e-3))))
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_total = timed(steps, step)
+    # same steps again with an event pair around every kernel: attributes the time to kernels
+    B.slkv_profile_enable(True)
+    barrier()
+    prof_steps = min(steps, 50)
+    for _ in range(prof_steps):
+        step()
+    torch.cuda.synchronize()
+    per_kernel = B.slkv_profile_collect()
+    B.slkv_profile_enable(False)
+    sampler.stop()
+    assert int(status.item()) == 0
+
+    ms_per_step = ms_total / steps
+    t_layer_us = ms_per_step * 1e3 / nl
+    value = world * T * nl / (ms_per_step * 1e-3)      # = world * T / t_layer: tokens per second per layer
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies in the timed region)
+    e2e = None
+    if not args.no_e2e:
+        cap = max(L["rows"] for L in layers)
+        arena = torch.empty(B.slkv_compress_host_arena_bytes(params, cu, cap), dtype=torch.uint8, device=dev)
+        n_host = min(nl, args.e2e_layers)
+        host = []
+        for L in layers[:n_host]:
+            host.append({"q": L["q"].cpu().pin_memory(), "k": L["k"].cpu().pin_memory(), "v": L["v"].cpu().pin_memory(),
+                         "bud": L["bud"].cpu(), "rows": L["rows"]})
+        k_out_h = torch.empty(cap, d, dtype=wl.torch_dtype).pin_memory()
+        v_out_h = torch.empty(cap, d, dtype=wl.torch_dtype).pin_memory()
+        off_h = torch.empty(len(wl.seq_lens) * hkv + 1, dtype=torch.int32).pin_memory()
+        kept_h = torch.empty(cap, dtype=torch.int32).pin_memory()
+
+        def e2e_step():
+            for l in range(nl):
+                Hh = host[l % n_host]
+                B.slkv_compress_host(params, Hh["q"], Hh["k"], Hh["v"], cu, Hh["bud"], k_out_h, v_out_h, off_h,
+                                     kept_h, arena, stream)
+
+        e2e_step()
+        e2e_steps = max(1, min(steps, args.e2e_steps))
+        barrier()
+        t0 = time.perf_counter()
+        ev_ms = timed(e2e_steps, e2e_step)
+        wall_ms = (time.perf_counter() - t0) * 1e3
+        e2e_ms = max(ev_ms, 0.0)
+        h2d = sum((Hh["q"].numel() + Hh["k"].numel() + Hh["v"].numel()) * e + (len(cu) + hkv) * 4
+                  for Hh in (host[l % n_host] for l in range(nl)))
+        d2h = sum(host[l % n_host]["rows"] * (2 * d * e + 4) + (len(wl.seq_lens) * hkv + 1) * 4 for l in range(nl))
+        e2e = {"value": world * T * nl / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
+               "host_layers_cycled": n_host, "wall_ms": wall_ms,
+               "api": "slkv_compress_host (pinned host buffers in, packed rows + offsets + indices out)"}
+        del arena
+
+    # ---- roofline of the dominant kernel and of the whole layer
+    peaks = measured_peaks()
+    n_hist = sum(max(n - w, 0) for n in wl.seq_lens)
+    q_bytes = len(wl.seq_lens) * w * wl.n_q_heads * d * e
+    k_scan = hkv * n_hist * d * e
+    rows_avg = sum(L["rows"] for L in layers) / nl
+    alg = {"k_score_lse": k_scan + q_bytes, "k_score_vote": k_scan + q_bytes + 4 * hkv * n_hist,
+           "k_pool": 8 * hkv * n_hist, "k_select": 4 * hkv * n_hist + 4 * rows_avg,
+           "k_gather": 4 * rows_avg * d * e + 4 * rows_avg, "k_setup": 0}
+    kern = {}
+    prof_total = sum(ms for ms, _ in per_kernel.values()) or 1.0
+    for name, (ms, cnt) in per_kernel.items():
+        kern[name] = {"launches_per_step": cnt / prof_steps, "avg_us": ms * 1e3 / cnt, "share": ms / prof_total}
+    top = max(per_kernel, key=lambda n: per_kernel[n][0])
+    top_us = kern[top]["avg_us"]
+    achieved = alg[top] / (top_us * 1e-6) / 1e9
+    layer_bytes = k_scan + q_bytes + 4 * rows_avg * d * e
+    flops_layer = 2 * 2.0 * wl.n_q_heads * w * n_hist * d           # two softmax passes
+    exps_layer = 2.0 * wl.n_q_heads * w * n_hist
+    clocks = sampler.summary()
+    f_sm = (clocks["sm_mhz"] or 1965.0) * 1e6
+    ceilings = {"t_hbm_us": layer_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                "t_tensor_us": flops_layer / (peaks["bf16_tflops"] * 1e12) * 1e6,
+                "t_ex2_us": exps_layer / (148 * 16 * f_sm) * 1e6}
+    roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "alg_bytes_per_launch": alg[top], "avg_launch_us": top_us,
+                "layer": {"alg_bytes": layer_bytes, "us": t_layer_us,
+                          "achieved": layer_bytes / (t_layer_us * 1e-6) / 1e9,
+                          "frac": layer_bytes / (t_layer_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                          "frac_of_8TBs_nominal": layer_bytes / (t_layer_us * 1e-6) / 8e12},
+                "ceilings": ceilings}
+    traffic_file = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(traffic_file):
+        try:
+            tr = json.load(open(traffic_file)).get(top)
+            if tr:
+                roofline["traffic"] = tr["bytes_per_key_row"] * hkv * n_hist
+                roofline["traffic_source"] = tr["source"]
+        except Exception:
+            pass
+
+    # ---- the oracle on the host cores (rank 0, N=1 only): a reported baseline, not a target
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle(wl, [(L["q"], L["k"], L["v"], budgets_host[i].tolist()) for i, L in enumerate(layers)],
+                                   budget_s=args.cpu_budget_s)
+
+    if rank == 0:
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+               "ms_per_step": ms_per_step, "us_per_layer": t_layer_us, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+               "config": {"workload": wl.name, "n_layers": nl, "n_q_heads": wl.n_q_heads, "n_kv_heads": hkv,
+                          "head_dim": d, "seq_lens": wl.seq_lens, "window": w, "pool_kernel": wl.pool_kernel,
+                          "avg_budget_per_kv_head": total // (nl * hkv), "fixed": wl.fixed, "parallelism":
+                          f"dp{world} (one sequence batch per GPU, no collective)",
+                          "l2": "inputs larger than L2: every layer has its own Q/K/V (%.1f GB per step)" %
+                                (nl * (2 * T * hkv * d * e) / 1e9)},
+               "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * steps,
+               "gpu_launches_per_step": launches_per_step, "kernels": kern, "roofline": roofline,
+               "cpu_baseline": cpu_baseline}
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------------
+# the oracle arm
+# ---------------------------------------------------------------------------------------------------
+def oracle_layer(wl, q, k, v, budgets_row):
+    import numpy as np
+    from oracle import slkv_oracle as O
+    f64 = lambda t: t.cpu().to(torch.float32).numpy().astype(np.float64)
+    f32 = lambda t: t.cpu().to(torch.float32).numpy()
+    return O.compress(f64(q), f32(k), f32(v), wl.cu_seqlens, budgets_row, wl.window, wl.pool_kernel)
+
+
+def time_oracle(wl, layer_inputs, budget_s=20.0):
+    """Times the oracle, as it stands, on a bounded sample of layers; returns the cpu_baseline object."""
+    times = []
+    t_begin = time.perf_counter()
+    for (q, k, v, bud) in layer_inputs:
+        qh, kh, vh = q.cpu(), k.cpu(), v.cpu()
+        t0 = time.perf_counter()
+        oracle_layer(wl, qh, kh, vh, bud)
+        times.append(time.perf_counter() - t0)
+        if time.perf_counter() - t_begin > budget_s:
+            break
+    t_layer = sum(times) / len(times)
+    return {"value": wl.total_tokens / t_layer, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "host_cores": os.cpu_count(), "s_per_layer": t_layer,
+            "sample": f"layers 0..{len(times) - 1} of {wl.name} ({len(times)} of {wl.n_layers} layers, full length, "
+                      f"all heads; numpy fp64, BLAS threads = cores)"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import slkv_oracle as O
+    wl = synth.workloads()[WORKLOAD_INDEX]
+    total = wl.totals[TOTAL_INDEX]
+    budgets = O.alloc_budgets(synth.inf_sc(wl).numpy(), wl.fixed, total)
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    n_samples = 2
+    inputs = []
+    for l in range(n_samples):
+        x = synth.layer_inputs(wl, l, device=gen_dev)
+        inputs.append((x.q_win.cpu(), x.k.cpu(), x.v.cpu(), budgets[l].tolist()))
+    warmup, steps = max(args.warmup, 1), (args.steps or 10)
+    # one step = the oracle on one layer (a 1/32 sample of the 32-layer step); bounded to a few minutes
+    t0 = time.perf_counter()
+    oracle_layer(wl, *inputs[0])
+    one = time.perf_counter() - t0
+    steps = max(1, min(steps, int(150.0 / max(one, 1e-3))))
+    warmup = max(1, min(warmup, int(30.0 / max(one, 1e-3))))
+    for i in range(warmup):
+        oracle_layer(wl, *inputs[i % n_samples])
+    t0 = time.perf_counter()
+    for i in range(steps):
+        oracle_layer(wl, *inputs[i % n_samples])
+    t_layer = (time.perf_counter() - t0) / steps
+    value = wl.total_tokens / t_layer
+    sample = f"one step = one layer of {wl.name} (layers 0,1 alternating; 1/32 of the 32-layer step), full length"
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+           "steps": steps, "warmup": warmup, "ms_per_step": t_layer * 1e3, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": wl.name, "n_layers": wl.n_layers, "n_q_heads": wl.n_q_heads,
+                      "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "seq_lens": wl.seq_lens,
+                      "window": wl.window, "pool_kernel": wl.pool_kernel,
+                      "avg_budget_per_kv_head": total // (wl.n_layers * wl.n_kv_heads), "fixed": wl.fixed},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                            "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="use fewer layers (profiling captures only)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-layers", type=int, default=8, help="distinct layers kept in pinned host memory")
+    ap.add_argument("--cpu-budget-s", type=float, default=20.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

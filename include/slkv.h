@@ -99,7 +99,7 @@ int slkv_last_cuda_error(void);
  * (0.01 + L_i/L_s) * (inf_ij/L_s), L_i the layer's INF_sc sum, L_s the grand sum; shares are rounded by
  * largest remainder (ties: lower index first) so that the budgets sum to `total` exactly.  All-zero
  * INF_sc gives uniform shares.  fp64 arithmetic in a fixed order: results are reproducible bit for bit.
- * Limits: n_layers <= 1024, n_layers*n_heads <= 16384, total - N*fixed < 2^52, budgets < 2^31.
+ * Limits: n_layers <= 1024, n_layers*n_heads <= 16384, total < 2^31 (else SLKV_ERR_BAD_SHAPE).
  */
 int slkv_alloc_budgets(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
                        int32_t* budgets, int32_t* status, void* stream);
@@ -172,6 +172,19 @@ int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, c
 /* Number of kernels the most recent slkv_score / slkv_compress / slkv_compress_host call on this
  * thread enqueued (launch accounting for benchmarks). */
 int slkv_last_launch_count(void);
+
+/*
+ * Per-kernel timing for benchmarks (no counterpart in the paper).  While enabled on the calling thread,
+ * every kernel the library enqueues is bracketed by a CUDA event pair on its stream (events are created
+ * on demand and reused; this adds host work per launch, so headline timings are taken with it off).
+ * slkv_profile_collect waits for the recorded events, adds each kernel's elapsed milliseconds and launch
+ * count into total_ms[id] / launches[id] (arrays of n_kernels entries, overwritten) and forgets the records.
+ * Kernel ids run from 0 to slkv_kernel_count()-1; slkv_kernel_name gives their names.
+ */
+int slkv_profile_enable(int on);
+int slkv_profile_collect(float* total_ms, int32_t* launches, int32_t n_kernels);
+const char* slkv_kernel_name(int kernel_id);
+int slkv_kernel_count(void);
 
 /* Library version, major*10000 + minor*100 + patch. */
 int slkv_version(void);

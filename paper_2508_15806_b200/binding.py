@@ -74,6 +74,13 @@ def lib() -> C.CDLL:
         L.slkv_compress_host.restype = C.c_int
         L.slkv_compress_host.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, i64, vp, vp, C.POINTER(C.c_int64),
                                          vp, sz, vp]
+        L.slkv_profile_enable.restype = C.c_int
+        L.slkv_profile_enable.argtypes = [C.c_int]
+        L.slkv_profile_collect.restype = C.c_int
+        L.slkv_profile_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int32), C.c_int32]
+        L.slkv_kernel_name.restype = C.c_char_p
+        L.slkv_kernel_name.argtypes = [C.c_int]
+        L.slkv_kernel_count.restype = C.c_int
         _lib = L
     return _lib
 
@@ -186,3 +193,18 @@ def slkv_compress_host(params: SlkvParams, q_win, k, v, cu_seqlens: Sequence[int
     if rc != SLKV_OK:
         raise SlkvError(rc, "slkv_compress_host")
     return int(rows.value)
+
+
+def slkv_profile_enable(on: bool) -> None:
+    lib().slkv_profile_enable(1 if on else 0)
+
+
+def slkv_profile_collect() -> dict:
+    """{kernel name: (total milliseconds, launches)} since the last collect, for kernels that ran."""
+    n = lib().slkv_kernel_count()
+    ms = (C.c_float * n)()
+    cnt = (C.c_int32 * n)()
+    rc = lib().slkv_profile_collect(ms, cnt, n)
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_profile_collect")
+    return {lib().slkv_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i] > 0}

@@ -153,6 +153,8 @@ cudaError_t launch_alloc(const float* inf, int n_layers, int n_heads, int fixed,
     if (e != cudaSuccess) return e;
     configured_dev = dev;
   }
+  int launches = 0;
+  LaunchScope scope(KID_ALLOC, st, &launches);
   k_alloc<<<1, kAllocThreads, smem, st>>>(inf, n_layers, n_heads, fixed, total, budgets, status);
   return cudaGetLastError();
 }

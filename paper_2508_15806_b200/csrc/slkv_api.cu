@@ -1,6 +1,7 @@
 // extern "C" entry points of libslkv: argument validation, workspace carve-up, launch sequencing.
 // No step of the method runs here; every step is a kernel in the other translation units.
 #include <cstring>
+#include <vector>
 
 #include "slkv_internal.cuh"
 
@@ -9,6 +10,23 @@ namespace {
 
 thread_local int g_last_cuda_error = 0;
 thread_local int g_last_launches = 0;
+
+// ---- per-kernel timing (off by default) -----------------------------------------------------------
+struct TimedLaunch { int kid; cudaEvent_t a, b; };
+thread_local bool g_prof_on = false;
+thread_local std::vector<TimedLaunch>* g_prof = nullptr;      // records of the current thread
+thread_local std::vector<cudaEvent_t>* g_prof_free = nullptr;
+
+cudaEvent_t prof_event() {
+  if (g_prof_free && !g_prof_free->empty()) {
+    cudaEvent_t e = g_prof_free->back();
+    g_prof_free->pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+  return e;
+}
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -166,6 +184,21 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
 }
 
 }  // namespace
+
+LaunchScope::LaunchScope(int kid, cudaStream_t st, int* launches) : kid_(kid), st_(st), slot_(-1) {
+  ++*launches;
+  if (!g_prof_on) return;
+  if (!g_prof) g_prof = new std::vector<TimedLaunch>();
+  TimedLaunch t{kid, prof_event(), prof_event()};
+  if (!t.a || !t.b) return;
+  cudaEventRecord(t.a, st);
+  g_prof->push_back(t);
+  slot_ = (int)g_prof->size() - 1;
+}
+LaunchScope::~LaunchScope() {
+  if (slot_ >= 0) cudaEventRecord((*g_prof)[slot_].b, st_);
+}
+
 }  // namespace slkv
 
 using namespace slkv;
@@ -188,6 +221,38 @@ const char* slkv_strerror(int status) {
     default: return "unknown slkv status";
   }
 }
+
+int slkv_profile_enable(int on) {
+  g_prof_on = on != 0;
+  return SLKV_OK;
+}
+
+int slkv_profile_collect(float* total_ms, int32_t* launches, int32_t n_kernels) {
+  if (!total_ms || !launches) return SLKV_ERR_NULL_PTR;
+  for (int i = 0; i < n_kernels; ++i) { total_ms[i] = 0.f; launches[i] = 0; }
+  if (!g_prof) return SLKV_OK;
+  if (!g_prof_free) g_prof_free = new std::vector<cudaEvent_t>();
+  int rc = SLKV_OK;
+  for (TimedLaunch& t : *g_prof) {
+    float ms = 0.f;
+    cudaError_t e = cudaEventSynchronize(t.b);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, t.a, t.b);
+    if (e != cudaSuccess) rc = cuda_fail(e);
+    else if (t.kid < n_kernels) { total_ms[t.kid] += ms; launches[t.kid] += 1; }
+    g_prof_free->push_back(t.a);
+    g_prof_free->push_back(t.b);
+  }
+  g_prof->clear();
+  return rc;
+}
+
+const char* slkv_kernel_name(int kernel_id) {
+  static const char* names[KID_COUNT] = {"k_setup", "k_score_lse", "k_score_vote", "k_pool", "k_select",
+                                         "k_gather", "k_alloc"};
+  return (kernel_id >= 0 && kernel_id < KID_COUNT) ? names[kernel_id] : "";
+}
+
+int slkv_kernel_count(void) { return KID_COUNT; }
 
 int slkv_last_cuda_error(void) { return g_last_cuda_error; }
 int slkv_last_launch_count(void) { return g_last_launches; }

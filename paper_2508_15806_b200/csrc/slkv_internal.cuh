@@ -38,6 +38,17 @@ struct Problem {
   int32_t* dev_flags;     // [8] scratch words (timeouts etc.)
 };
 
+// kernel ids for launch accounting / per-kernel timing
+enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_COUNT };
+
+// Brackets one kernel launch: counts it and, when per-kernel timing is on for this thread, records a
+// CUDA event pair around it on the launch stream.
+struct LaunchScope {
+  LaunchScope(int kid, cudaStream_t st, int* launches);
+  ~LaunchScope();
+  int kid_; cudaStream_t st_; int slot_;
+};
+
 // host-side launchers; each returns a cudaError_t and adds to *launches
 cudaError_t launch_alloc(const float* inf, int n_layers, int n_heads, int fixed, long long total, int32_t* budgets,
                          int32_t* status, cudaStream_t st);

@@ -178,18 +178,20 @@ cudaError_t launch_both(const Problem& pb, cudaStream_t st, int* launches) {
   dim3 grid((pb.max_hist + chunk_keys - 1) / chunk_keys, pb.p.n_kv_heads, pb.p.n_seqs);
   const float scale_log2 = kLog2e / sqrtf((float)pb.p.head_dim);
   const slkv_params& p = pb.p;
-  k_score_simt<T, D, 1><<<grid, kThreads, smem, st>>>(
-      (const T*)pb.q, (const T*)pb.k, pb.cu, pb.hist_off, pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G,
-      p.window, pb.n_chunks, p.k_stride_tok, p.k_stride_head, p.q_stride_seq, p.q_stride_row, p.q_stride_head,
-      scale_log2);
-  ++*launches;
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  {
+    LaunchScope scope(KID_SCORE_LSE, st, launches);
+    k_score_simt<T, D, 1><<<grid, kThreads, smem, st>>>(
+        (const T*)pb.q, (const T*)pb.k, pb.cu, pb.hist_off, pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G,
+        p.window, pb.n_chunks, p.k_stride_tok, p.k_stride_head, p.q_stride_seq, p.q_stride_row, p.q_stride_head,
+        scale_log2);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  LaunchScope scope(KID_SCORE_VOTE, st, launches);
   k_score_simt<T, D, 2><<<grid, kThreads, smem, st>>>(
       (const T*)pb.q, (const T*)pb.k, pb.cu, pb.hist_off, pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G,
       p.window, pb.n_chunks, p.k_stride_tok, p.k_stride_head, p.q_stride_seq, p.q_stride_row, p.q_stride_head,
       scale_log2);
-  ++*launches;
   return cudaGetLastError();
 }
 

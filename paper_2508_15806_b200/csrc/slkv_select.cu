@@ -204,26 +204,26 @@ k_gather(const unsigned char* __restrict__ k, const unsigned char* __restrict__ 
 
 cudaError_t launch_setup(const Problem& pb, const int32_t* budgets, int32_t* offsets, int64_t capacity,
                          int32_t* status, cudaStream_t st, int* launches) {
+  LaunchScope scope(KID_SETUP, st, launches);
   k_setup<<<1, kScanThreads, 0, st>>>(pb.cu, pb.p.n_seqs, pb.p.n_kv_heads, pb.p.window, budgets, pb.hist_off,
                                       offsets, (long long)capacity, status);
-  ++*launches;
   return cudaGetLastError();
 }
 
 cudaError_t launch_pool(const Problem& pb, float* pooled, cudaStream_t st, int* launches) {
   if (pb.max_hist <= 0) return cudaSuccess;
   dim3 grid((pb.max_hist + 255) / 256, pb.p.n_kv_heads, pb.p.n_seqs);
+  LaunchScope scope(KID_POOL, st, launches);
   k_pool<<<grid, 256, 0, st>>>(pb.vote, pooled, pb.cu, pb.hist_off, pb.p.n_kv_heads, pb.p.window,
                                pb.p.pool_kernel, pb.p.pool_mode);
-  ++*launches;
   return cudaGetLastError();
 }
 
 cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t capacity, cudaStream_t st, int* launches) {
+  LaunchScope scope(KID_SELECT, st, launches);
   k_select<<<pb.n_seg, kScanThreads, 0, st>>>(pooled, pb.cu, pb.hist_off, budgets, offsets, kept_idx,
                                               pb.p.n_kv_heads, pb.p.window, (long long)capacity);
-  ++*launches;
   return cudaGetLastError();
 }
 
@@ -236,11 +236,11 @@ cudaError_t launch_gather(const Problem& pb, const int32_t* offsets, const int32
   if (max_rows <= 0) return cudaSuccess;
   long long want = (max_rows + rows_per_cta - 1) / rows_per_cta;
   int grid = (int)(want < 148 * 16 ? want : 148 * 16);
+  LaunchScope scope(KID_GATHER, st, launches);
   k_gather<<<grid, 256, 0, st>>>((const unsigned char*)pb.k, (const unsigned char*)pb.v, (unsigned char*)k_out,
                                  (unsigned char*)v_out, pb.cu, offsets, kept_idx, pb.n_seg, pb.p.n_kv_heads,
                                  row_bytes, pb.p.k_stride_tok * pb.elem, pb.p.k_stride_head * pb.elem,
                                  pb.p.v_stride_tok * pb.elem, pb.p.v_stride_head * pb.elem, (long long)capacity);
-  ++*launches;
   return cudaGetLastError();
 }
 
