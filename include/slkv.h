@@ -124,11 +124,13 @@ int64_t slkv_packed_rows_upper_bound(const slkv_params* p, const int32_t* cu_seq
  *   q_win, k         dev, layouts above
  *   cu_seqlens_dev   dev, int32[n_seqs+1];  cu_seqlens_host: the same values on the host (sizes the launch)
  *   pooled           dev, out, float[slkv_pooled_elems]
+ *   status           dev, optional: SLKV_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel ran out
+ *                    (pooled is then incomplete)
  * Accuracy: fp32 accumulation; relative error of pooled <= 1e-3 of the exact value.
  */
 int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
-               const int32_t* cu_seqlens_host, float* pooled, void* workspace, size_t workspace_bytes,
-               void* stream);
+               const int32_t* cu_seqlens_host, float* pooled, int32_t* status, void* workspace,
+               size_t workspace_bytes, void* stream);
 
 /*
  * KV entry selection and gather for one layer (Sec. 3.4, Eq. 8; Algorithm 3).

@@ -66,7 +66,7 @@ def lib() -> C.CDLL:
         L.slkv_packed_rows_upper_bound.restype = i64
         L.slkv_packed_rows_upper_bound.argtypes = [pp, i32p]
         L.slkv_score.restype = C.c_int
-        L.slkv_score.argtypes = [pp, vp, vp, vp, i32p, vp, vp, sz, vp]
+        L.slkv_score.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, sz, vp]
         L.slkv_compress.restype = C.c_int
         L.slkv_compress.argtypes = [pp, vp, vp, vp, vp, i32p, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
         L.slkv_compress_host_arena_bytes.restype = sz
@@ -156,9 +156,10 @@ def new_workspace(params: SlkvParams, cu_seqlens: Sequence[int], device) -> torc
 
 
 def slkv_score(params: SlkvParams, q_win: torch.Tensor, k: torch.Tensor, cu_dev: torch.Tensor,
-               cu_seqlens: Sequence[int], pooled: torch.Tensor, workspace: torch.Tensor, stream=None) -> torch.Tensor:
+               cu_seqlens: Sequence[int], pooled: torch.Tensor, workspace: torch.Tensor,
+               status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     rc = lib().slkv_score(C.byref(params), q_win.data_ptr(), k.data_ptr(), cu_dev.data_ptr(), _cu_host(cu_seqlens),
-                          pooled.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(stream))
+                          pooled.data_ptr(), _ptr(status), workspace.data_ptr(), workspace.numel(), _stream(stream))
     if rc != SLKV_OK:
         raise SlkvError(rc, "slkv_score")
     return pooled

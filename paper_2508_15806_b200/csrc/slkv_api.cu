@@ -31,7 +31,7 @@ cudaEvent_t prof_event() {
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-constexpr int kMinChunkKeys = 256;     // no score path uses smaller chunks (sizes the partial buffers)
+constexpr int kMinChunkKeys = 128;     // no score path uses smaller chunks (sizes the partial buffers)
 constexpr int kMaxWindow = 256;
 constexpr size_t kSimtSmemLimit = 192 * 1024;
 
@@ -41,7 +41,7 @@ int cuda_fail(cudaError_t e) {
 }
 
 struct Layout {
-  size_t hist_off, vote, pooled, part_m, part_z, flags, total;
+  size_t hist_off, tile_off, vote, pooled, part_m, part_z, flags, total;
 };
 
 // Validates p and cu_seqlens_host and fills the host-known fields of `pb`.
@@ -97,10 +97,11 @@ Layout layout_of(const Problem& pb) {
   Layout L;
   size_t o = 0;
   L.hist_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int64_t));
+  L.tile_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int32_t));
   const size_t votes = (size_t)pb.p.n_kv_heads * (size_t)pb.total_hist * sizeof(float);
   L.vote = o; o = align_up(o + votes);
   L.pooled = o; o = align_up(o + votes);
-  const size_t nchunks = (size_t)(pb.max_hist + kMinChunkKeys - 1) / kMinChunkKeys + 1;
+  const size_t nchunks = (size_t)(pb.max_hist + kMinChunkKeys - 1) / kMinChunkKeys + 2;
   const size_t parts = (size_t)pb.n_seg * pb.R * nchunks * sizeof(float);
   L.part_m = o; o = align_up(o + parts);
   L.part_z = o; o = align_up(o + parts);
@@ -127,13 +128,15 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path) {
   if (ws_bytes < L.total) return SLKV_ERR_WORKSPACE;
   unsigned char* b = static_cast<unsigned char*>(ws);
   pb->hist_off = reinterpret_cast<int64_t*>(b + L.hist_off);
+  pb->tile_off = reinterpret_cast<int32_t*>(b + L.tile_off);
   pb->vote = reinterpret_cast<float*>(b + L.vote);
   pb->pooled_ws = reinterpret_cast<float*>(b + L.pooled);
   pb->part_m = reinterpret_cast<float*>(b + L.part_m);
   pb->part_z = reinterpret_cast<float*>(b + L.part_z);
   pb->dev_flags = reinterpret_cast<int32_t*>(b + L.flags);
-  pb->chunk_keys = path == SLKV_PATH_TENSOR ? tensor_chunk_keys(*pb) : simt_chunk_keys();
-  pb->n_chunks = (pb->max_hist + pb->chunk_keys - 1) / pb->chunk_keys;
+  pb->chunk_keys = path == SLKV_PATH_TENSOR ? 128 : simt_chunk_keys();
+  pb->n_chunks = path == SLKV_PATH_TENSOR ? tensor_slot_stride(*pb)
+                                          : (pb->max_hist + pb->chunk_keys - 1) / pb->chunk_keys;
   if (pb->n_chunks < 1) pb->n_chunks = 1;
   return SLKV_OK;
 }
@@ -141,8 +144,9 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path) {
 bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
 
 // score -> pooled (device pointers resolved); shared by slkv_score and slkv_compress
-int enqueue_score(const Problem& pb, int path, float* pooled, cudaStream_t st, int* launches) {
-  cudaError_t e = path == SLKV_PATH_TENSOR ? launch_score_tensor(pb, st, launches)
+int enqueue_score(const Problem& pb, int path, const int32_t* cu_host, float* pooled, int32_t* status,
+                  cudaStream_t st, int* launches) {
+  cudaError_t e = path == SLKV_PATH_TENSOR ? launch_score_tensor(pb, cu_host, status, st, launches)
                                            : launch_score_simt(pb, st, launches);
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_pool(pb, pooled, st, launches);
@@ -173,7 +177,7 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
   cudaError_t e = launch_setup(pb, budgets, offsets, capacity, status, st, &launches);
   if (e != cudaSuccess) return cuda_fail(e);
   float* pooled = pooled_opt ? pooled_opt : pb.pooled_ws;
-  rc = enqueue_score(pb, path, pooled, st, &launches);
+  rc = enqueue_score(pb, path, cu_host, pooled, status, st, &launches);
   if (rc != SLKV_OK) return rc;
   e = launch_select(pb, pooled, budgets, offsets, kept_idx, capacity, st, &launches);
   if (e != cudaSuccess) return cuda_fail(e);
@@ -289,8 +293,8 @@ int64_t slkv_packed_rows_upper_bound(const slkv_params* p, const int32_t* cu_seq
 }
 
 int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
-               const int32_t* cu_seqlens_host, float* pooled, void* workspace, size_t workspace_bytes,
-               void* stream) {
+               const int32_t* cu_seqlens_host, float* pooled, int32_t* status, void* workspace,
+               size_t workspace_bytes, void* stream) {
   g_last_launches = 0;
   if (!q_win || !k || !cu_seqlens_dev || !pooled) return SLKV_ERR_NULL_PTR;
   Problem pb;
@@ -307,7 +311,7 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
   int launches = 0;
   cudaError_t e = launch_setup(pb, nullptr, nullptr, 0, nullptr, st, &launches);
   if (e != cudaSuccess) return cuda_fail(e);
-  rc = enqueue_score(pb, path, pooled, st, &launches);
+  rc = enqueue_score(pb, path, cu_seqlens_host, pooled, status, st, &launches);
   if (rc != SLKV_OK) return rc;
   g_last_launches = launches;
   return SLKV_OK;

@@ -29,6 +29,7 @@ struct Problem {
   const void* v;          // dev
   // workspace carve-up (dev)
   int64_t* hist_off;      // [n_seqs+1] exclusive prefix of n_hist_s
+  int32_t* tile_off;      // [n_seqs+1] exclusive prefix of ceil(n_hist_s / 128)
   float* vote;            // [n_kv_heads * total_hist] ragged, same layout as pooled
   float* part_m;          // [n_seg][R][n_chunks] partial row maxima (log2 domain)
   float* part_z;          // [n_seg][R][n_chunks] partial row sums
@@ -58,8 +59,9 @@ int simt_chunk_keys();
 size_t simt_smem_bytes(const Problem& pb);
 cudaError_t launch_score_simt(const Problem& pb, cudaStream_t st, int* launches);
 bool tensor_path_supported(const slkv_params& p);
-int tensor_chunk_keys(const Problem& pb);
-cudaError_t launch_score_tensor(const Problem& pb, cudaStream_t st, int* launches);
+int tensor_slot_stride(const Problem& pb);
+cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, cudaStream_t st,
+                                int* launches);
 cudaError_t launch_pool(const Problem& pb, float* pooled, cudaStream_t st, int* launches);
 cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t capacity, cudaStream_t st, int* launches);

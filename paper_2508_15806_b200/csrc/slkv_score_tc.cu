@@ -1,8 +1,544 @@
-// Tensor-core score path (tcgen05 + TMA).  Placeholder until the kernels land: reports "unsupported".
+// Window relevance scores on the 5th-generation tensor cores (Sec. 3.4, Eq. 7; Algorithm 3 l.6; Eq. 3-4).
+//
+// bf16, head_dim 128.  Two persistent kernels share one schedule: the history keys of all (sequence,
+// KV head) segments form one list of 128-key tiles, split evenly over one CTA per SM.
+//   pass 1 (row statistics)  S = Q K^T per tile with the G*w query rows as the M dimension, so that a
+//           TMEM lane -- one thread -- owns a query row: running max and sum of 2^(s - max) stay in
+//           registers; per CTA and segment one (max, sum) pair per row goes to global memory.
+//   pass 2 (votes)           S^T = K Q^T per tile with the keys as the M dimension, so that a thread owns
+//           a key: vote[j] = (1/G) sum_rows 2^(s_rj - lse_r) is a thread-local sum and a coalesced store.
+// Warp roles: warp 0 issues TMA loads (128-byte-swizzled K-major tiles, no multicast), warp 1 issues
+// tcgen05.mma into TMEM accumulators and commits to mbarriers, warps 4..11 (two warpgroups, alternating
+// tiles) read TMEM with tcgen05.ld and do the softmax arithmetic in fp32.
+// Every mbarrier wait is bounded by a wall-clock limit; when one runs out the CTA raises
+// SLKV_ERR_DEVICE_TIMEOUT in the status word, stops waiting everywhere, releases TMEM and returns.
+#include <cuda.h>
+
 #include "slkv_internal.cuh"
 
 namespace slkv {
-bool tensor_path_supported(const slkv_params&) { return false; }
-int tensor_chunk_keys(const Problem&) { return 1024; }
-cudaError_t launch_score_tensor(const Problem&, cudaStream_t, int*) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kTileKeys = 128;                 // keys per tile (MMA N in pass 1, M in pass 2)
+constexpr int kStages = 4;                     // K tiles in flight in shared memory
+constexpr int kHalfBytes = kTileKeys * 128;    // one 64-element (128-byte) half of a 128-row tile
+constexpr int kStageBytes = 2 * kHalfBytes;    // 32 KB
+constexpr int kThreads = 384;                  // warps 0-3: TMA, MMA, 2 idle; warps 4-11: epilogue
+constexpr int kEpiThreads = 256;
+constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per wait
+
+struct TcArgs {
+  const int32_t* cu;
+  const int64_t* hist_off;
+  const int32_t* tile_off;      // [n_seqs+1] exclusive prefix of ceil(n_hist_s / 128)
+  float* part_m;
+  float* part_z;
+  float* vote;
+  int32_t* status;
+  int n_seqs, n_kv_heads, G, window, R, MT, slot_stride, tiles_per_cta, total_tiles;
+  int q_head_inner, k_head_inner;   // tensor-map dimension order: 1 = the head axis comes before the row axis
+  float scale_log2;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase with the given parity.  false = gave up (limit reached or another thread did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = now_ns();
+  for (unsigned it = 1;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (now_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, int w,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
+
+// K-major, 128-byte-swizzled operand: rows 128 bytes apart, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// D fp32, A and B bf16, both K-major, M x N tile
+__device__ __forceinline__ uint32_t instr_desc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct Run { int s, g, t0, count, n_hist, seg_tile0, tiles_seg; };
+
+// The run of tiles starting at global tile `gt` that stays inside one segment and before `end`.
+__device__ __forceinline__ Run locate(const TcArgs& a, int gt, int end) {
+  int lo = 0, hi = a.n_seqs;                       // last s with Hkv*tile_off[s] <= gt
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (a.n_kv_heads * a.tile_off[mid] <= gt) lo = mid; else hi = mid;
+  }
+  Run r;
+  r.s = lo;
+  r.tiles_seg = a.tile_off[lo + 1] - a.tile_off[lo];
+  const int rel = gt - a.n_kv_heads * a.tile_off[lo];
+  r.g = rel / r.tiles_seg;
+  r.t0 = rel - r.g * r.tiles_seg;
+  r.seg_tile0 = gt - r.t0;
+  r.count = min(end - gt, r.tiles_seg - r.t0);
+  r.n_hist = max(a.cu[lo + 1] - a.cu[lo] - a.window, 0);
+  return r;
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const TcArgs a) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ __align__(8) unsigned long long bars[2 * kStages + 2 * 4 + 2];
+  __shared__ uint32_t tmem_base_sh;
+  __shared__ int abort_sh;
+  __shared__ __align__(16) float lse_sh[2][256];
+  __shared__ float stat_m[256], stat_z[256];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int MT = a.MT, R = a.R;
+  const int buf_cols = MT * 128;
+  const int n_bufs = 512 / buf_cols;                        // 4 or 2 TMEM accumulator buffers
+  const int q_half_bytes = MT * 128 * 128;                  // one 64-element half of the (padded) Q tile
+
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  const uint32_t q_smem = smem_u32(smem);
+  const uint32_t k_smem = q_smem + 2 * q_half_bytes;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int st) { return bar0 + 8u * st; };
+  auto empty_bar = [&](int st) { return bar0 + 8u * (kStages + st); };
+  auto accf_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
+  auto acce_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 4 + b); };
+  const uint32_t qfull_bar = bar0 + 8u * (2 * kStages + 8), qempty_bar = qfull_bar + 8u;
+  volatile int* abort_flag = &abort_sh;
+
+  const int begin = blockIdx.x * a.tiles_per_cta;
+  const int end = min(begin + a.tiles_per_cta, a.total_tiles);
+
+  if (tid == 0) {
+    abort_sh = 0;
+    for (int st = 0; st < kStages; ++st) { mbar_init(full_bar(st), 1); mbar_init(empty_bar(st), 1); }
+    for (int b = 0; b < 4; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
+    mbar_init(qfull_bar, 1);
+    mbar_init(qempty_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // rows of the Q tile beyond R are never written by TMA: keep them zero
+  for (int i = tid; i < 2 * q_half_bytes / 16; i += kThreads) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_sh;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int it = 0, run_idx = 0;
+      bool ok = true;
+      for (int gt = begin; gt < end && ok;) {
+        const Run r = locate(a, gt, end);
+        ok = mbar_wait(qempty_bar, (run_idx & 1) ^ 1, abort_flag);      // previous run's MMAs are done with Q
+        if (!ok) break;
+        mbar_expect_tx(qfull_bar, 2u * (uint32_t)R * 128u);
+        const int qy = a.q_head_inner ? r.g * a.G : 0, qz = a.q_head_inner ? 0 : r.g * a.G;
+        tma_load_4d(q_smem, &tm_q, 0, qy, qz, r.s, qfull_bar);
+        tma_load_4d(q_smem + q_half_bytes, &tm_q, 64, qy, qz, r.s, qfull_bar);
+        const int tok0 = a.cu[r.s];
+        for (int t = 0; t < r.count; ++t, ++it) {
+          const int st = it % kStages;
+          ok = mbar_wait(empty_bar(st), ((it / kStages) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(full_bar(st), kStageBytes);
+          const int tok = tok0 + (r.t0 + t) * kTileKeys;
+          const int ky = a.k_head_inner ? r.g : tok, kz = a.k_head_inner ? tok : r.g;
+          tma_load_3d(k_smem + st * kStageBytes, &tm_k, 0, ky, kz, full_bar(st));
+          tma_load_3d(k_smem + st * kStageBytes + kHalfBytes, &tm_k, 64, ky, kz, full_bar(st));
+        }
+        gt += r.count;
+        ++run_idx;
+      }
+      if (!ok) {
+        // give loads already in flight a bounded chance to land before the CTA's shared memory goes away
+        const unsigned long long t0 = now_ns();
+        for (int st = 0; st < kStages; ++st) {
+          const int last = it - 1 - ((it - 1 - st) % kStages + kStages) % kStages;   // last issue into stage st
+          if (it == 0 || last < 0) continue;
+          while (!mbar_try(full_bar(st), (last / kStages) & 1) && now_ns() - t0 < kWaitLimitNs) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = PASS == 1 ? instr_desc(128, kTileKeys) : instr_desc(kTileKeys, R);
+      int it = 0, run_idx = 0;
+      bool ok = true;
+      for (int gt = begin; gt < end && ok;) {
+        const Run r = locate(a, gt, end);
+        ok = mbar_wait(qfull_bar, run_idx & 1, abort_flag);
+        if (!ok) break;
+        for (int t = 0; t < r.count; ++t, ++it) {
+          const int st = it % kStages, b = it % n_bufs;
+          ok = mbar_wait(full_bar(st), (it / kStages) & 1, abort_flag) &&
+               mbar_wait(acce_bar(b), ((it / n_bufs) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t kst = k_smem + st * kStageBytes;
+          const uint32_t d0 = tmem_base + (uint32_t)(b * buf_cols);
+          if (PASS == 1) {
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+              for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                const uint32_t qoff = (uint32_t)(ks >> 2) * q_half_bytes + (uint32_t)(ks & 3) * 32u + mt * (128 * 128);
+                tc_mma(d0 + mt * 128, smem_desc(q_smem + qoff), smem_desc(kst + koff), idesc, ks > 0);
+              }
+          } else {
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+              const uint32_t qoff = (uint32_t)(ks >> 2) * q_half_bytes + (uint32_t)(ks & 3) * 32u;
+              tc_mma(d0, smem_desc(kst + koff), smem_desc(q_smem + qoff), idesc, ks > 0);
+            }
+          }
+          tc_commit(empty_bar(st));       // K stage free once these MMAs have read it
+          tc_commit(accf_bar(b));         // accumulator ready for the epilogue
+        }
+        tc_commit(qempty_bar);            // Q tile free once the run's MMAs are done
+        gt += r.count;
+        ++run_idx;
+      }
+    }
+  } else if (warp >= 4) {
+    // ---------------- epilogue: two warpgroups, alternating tiles ----------------
+    const int et = tid - 128;                   // 0..255
+    const int wg = et >> 7;                     // warpgroup 0 / 1
+    const int row = et & 127;                   // TMEM lane this thread reads
+    const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+    const float sc = a.scale_log2;
+    const float inv_g = 1.0f / (float)a.G;
+    int it = 0, run_idx = 0;
+    bool ok = true;
+    for (int gt = begin; gt < end;) {
+      const Run r = locate(a, gt, end);
+      const int seg = r.s * a.n_kv_heads + r.g;
+      const int first_cta = r.seg_tile0 / a.tiles_per_cta;
+      float m_run[2] = {-INFINITY, -INFINITY}, z_run[2] = {0.f, 0.f};
+      float* lse = lse_sh[run_idx & 1];
+      if (PASS == 2) {
+        // merge the per-CTA partials of this segment into the rows' log-sum-exp (log2 units)
+        const int n_slots = (r.seg_tile0 + r.tiles_seg - 1) / a.tiles_per_cta - first_cta + 1;
+        if (et < R) {
+          const float* pm = a.part_m + ((long long)seg * R + et) * a.slot_stride;
+          const float* pz = a.part_z + ((long long)seg * R + et) * a.slot_stride;
+          float M = -INFINITY;
+          for (int c = 0; c < n_slots; ++c) M = fmaxf(M, pm[c]);
+          float Z = 0.f;
+          for (int c = 0; c < n_slots; ++c) Z += pz[c] * exp2f(pm[c] - M);
+          lse[et] = M + log2f(Z);
+        }
+        epi_bar();
+      }
+      for (int t = 0; t < r.count; ++t, ++it) {
+        if ((it & 1) != wg) continue;
+        const int b = it % n_bufs;
+        if (ok) ok = mbar_wait(accf_bar(b), (it / n_bufs) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, ok) != 0;         // the TMEM loads below need the whole warp
+        if (!ok) continue;
+        tc_fence_after();
+        const int key0 = (r.t0 + t) * kTileKeys;
+        const uint32_t tb = tmem_base + lane_sel + (uint32_t)(b * buf_cols);
+        if (PASS == 1) {
+          const int n_valid = min(r.n_hist - key0, kTileKeys);
+          for (int mt = 0; mt < MT; ++mt) {
+            float m = m_run[mt], z = z_run[mt];
+#pragma unroll 1
+            for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
+              float v[32];
+              tc_ld32(tb + mt * 128 + c0, v);
+              if (n_valid < kTileKeys) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) if (c0 + e >= n_valid) v[e] = -INFINITY;
+              }
+              float cm = v[0];
+#pragma unroll
+              for (int e = 1; e < 32; ++e) cm = fmaxf(cm, v[e]);
+              const float mn = fmaxf(m, cm * sc);
+              if (mn > -INFINITY) {
+                z *= ex2(m - mn);
+                m = mn;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                  s0 += ex2(fmaf(v[e], sc, -m));
+                  s1 += ex2(fmaf(v[e + 1], sc, -m));
+                }
+                z += s0 + s1;
+              }
+            }
+            m_run[mt] = m; z_run[mt] = z;
+          }
+        } else {
+          float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll 1
+          for (int c0 = 0; c0 < R; c0 += 32) {
+            float v[32];
+            tc_ld32(tb + c0, v);
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+              const float4 l4 = *reinterpret_cast<const float4*>(lse + c0 + e);
+              acc0 += ex2(fmaf(v[e], sc, -l4.x));
+              acc1 += ex2(fmaf(v[e + 1], sc, -l4.y));
+              acc0 += ex2(fmaf(v[e + 2], sc, -l4.z));
+              acc1 += ex2(fmaf(v[e + 3], sc, -l4.w));
+            }
+          }
+          const int j = key0 + row;
+          if (j < r.n_hist) a.vote[a.hist_off[r.s] * a.n_kv_heads + (long long)r.g * r.n_hist + j] = (acc0 + acc1) * inv_g;
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(b));
+      }
+      if (PASS == 1) {
+        // combine the two warpgroups' statistics and publish this CTA's partial for the segment
+        const int slot = blockIdx.x - first_cta;
+        for (int mt = 0; mt < MT; ++mt) {
+          if (wg == 1) { stat_m[row] = m_run[mt]; stat_z[row] = z_run[mt]; }
+          epi_bar();
+          if (wg == 0) {
+            const int rr = mt * 128 + row;
+            if (rr < R) {
+              const float m1 = stat_m[row], z1 = stat_z[row];
+              const float M = fmaxf(m_run[mt], m1);
+              float Z = 0.f;
+              if (M > -INFINITY) Z = z_run[mt] * ex2(m_run[mt] - M) + z1 * ex2(m1 - M);
+              a.part_m[((long long)seg * R + rr) * a.slot_stride + slot] = M;
+              a.part_z[((long long)seg * R + rr) * a.slot_stride + slot] = Z;
+            }
+          }
+          epi_bar();
+        }
+      }
+      gt += r.count;
+      ++run_idx;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (abort_sh && tid == 0 && a.status) atomicExch(a.status, (int)SLKV_ERR_DEVICE_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// ---- host side ----------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+int sm_count() {
+  static thread_local int dev_cached = -1, n = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (dev != dev_cached) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 148;
+    dev_cached = dev;
+  }
+  return n;
+}
+
+struct Schedule { int total_tiles, tiles_per_cta, n_cta; };
+
+Schedule schedule_of(const Problem& pb, const int32_t* cu_host) {
+  long long tiles = 0;
+  for (int s = 0; s < pb.p.n_seqs; ++s) {
+    long long nh = (long long)cu_host[s + 1] - cu_host[s] - pb.p.window;
+    if (nh > 0) tiles += (nh + kTileKeys - 1) / kTileKeys;
+  }
+  Schedule sc;
+  sc.total_tiles = (int)(tiles * pb.p.n_kv_heads);
+  const int sms = sm_count();
+  sc.tiles_per_cta = sc.total_tiles > 0 ? (sc.total_tiles + sms - 1) / sms : 1;
+  sc.n_cta = sc.total_tiles > 0 ? (sc.total_tiles + sc.tiles_per_cta - 1) / sc.tiles_per_cta : 0;
+  return sc;
+}
+
+}  // namespace
+
+bool tensor_path_supported(const slkv_params& p) {
+  if (p.dtype != SLKV_BF16 || p.head_dim != 128) return false;
+  const int G = p.n_q_heads / p.n_kv_heads, R = G * p.window;
+  if (R % 32 != 0 || R > 256 || p.window > 256 || G > 256) return false;
+  return encode_fn() != nullptr;
+}
+
+int tensor_slot_stride(const Problem& pb) { return (pb.max_hist + kTileKeys - 1) / kTileKeys + 2; }
+
+cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, cudaStream_t st,
+                                int* launches) {
+  if (pb.max_hist <= 0) return cudaSuccess;
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  const slkv_params& p = pb.p;
+  const Schedule sc = schedule_of(pb, cu_host);
+  if (sc.n_cta == 0) return cudaSuccess;
+
+  // Tensor-map dimensions go from the smallest stride to the largest.  The order of the G*w query rows
+  // inside the Q tile follows from it (head-fastest or window-row-fastest); the scores do not depend on it.
+  const int q_head_inner = p.q_stride_head <= p.q_stride_row;
+  const int k_head_inner = p.k_stride_head <= p.k_stride_tok;
+  CUtensorMap tm_q, tm_k;
+  {
+    cuuint64_t dims[4] = {(cuuint64_t)p.head_dim, (cuuint64_t)p.window, (cuuint64_t)p.n_q_heads, (cuuint64_t)p.n_seqs};
+    cuuint64_t strides[3] = {(cuuint64_t)p.q_stride_row * 2, (cuuint64_t)p.q_stride_head * 2, (cuuint64_t)p.q_stride_seq * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)p.window, (cuuint32_t)pb.G, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (q_head_inner) {
+      cuuint64_t t = dims[1]; dims[1] = dims[2]; dims[2] = t;
+      t = strides[0]; strides[0] = strides[1]; strides[1] = t;
+      cuuint32_t b = box[1]; box[1] = box[2]; box[2] = b;
+    }
+    if (enc(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pb.q), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+  {
+    cuuint64_t dims[3] = {(cuuint64_t)p.head_dim, (cuuint64_t)p.n_kv_heads, (cuuint64_t)pb.total_tokens};
+    cuuint64_t strides[2] = {(cuuint64_t)p.k_stride_head * 2, (cuuint64_t)p.k_stride_tok * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)kTileKeys};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (!k_head_inner) {
+      cuuint64_t t = dims[1]; dims[1] = dims[2]; dims[2] = t;
+      t = strides[0]; strides[0] = strides[1]; strides[1] = t;
+      cuuint32_t b = box[1]; box[1] = box[2]; box[2] = b;
+    }
+    if (enc(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(pb.k), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorInvalidValue;
+  }
+
+  TcArgs a;
+  a.cu = pb.cu; a.hist_off = pb.hist_off; a.tile_off = pb.tile_off;
+  a.part_m = pb.part_m; a.part_z = pb.part_z; a.vote = pb.vote; a.status = status;
+  a.n_seqs = p.n_seqs; a.n_kv_heads = p.n_kv_heads; a.G = pb.G; a.window = p.window; a.R = pb.R;
+  a.MT = (pb.R + 127) / 128;
+  a.q_head_inner = q_head_inner; a.k_head_inner = k_head_inner;
+  a.slot_stride = pb.n_chunks;
+  a.tiles_per_cta = sc.tiles_per_cta; a.total_tiles = sc.total_tiles;
+  a.scale_log2 = kLog2e / sqrtf((float)p.head_dim);
+
+  const size_t smem = 1024 + (size_t)a.MT * 2 * 128 * 128 + (size_t)kStages * kStageBytes;
+  static thread_local int configured_dev = -1;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (configured_dev != dev) {
+    e = cudaFuncSetAttribute(k_score_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_score_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    configured_dev = dev;
+  }
+  {
+    LaunchScope scope(KID_SCORE_LSE, st, launches);
+    k_score_tc<1><<<sc.n_cta, kThreads, smem, st>>>(tm_q, tm_k, a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  LaunchScope scope(KID_SCORE_VOTE, st, launches);
+  k_score_tc<2><<<sc.n_cta, kThreads, smem, st>>>(tm_q, tm_k, a);
+  return cudaGetLastError();
+}
+
 }  // namespace slkv

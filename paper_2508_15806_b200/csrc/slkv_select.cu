@@ -38,11 +38,11 @@ __device__ __forceinline__ int kept_rows(int len, int budget, int window) {
 // seg = s*Hkv + h starts.
 __global__ void __launch_bounds__(kScanThreads, 1)
 k_setup(const int32_t* __restrict__ cu, int n_seqs, int n_kv_heads, int window, const int32_t* __restrict__ budgets,
-        int64_t* __restrict__ hist_off, int32_t* __restrict__ offsets, long long capacity,
-        int32_t* __restrict__ status) {
+        int64_t* __restrict__ hist_off, int32_t* __restrict__ tile_off, int32_t* __restrict__ offsets,
+        long long capacity, int32_t* __restrict__ status) {
   __shared__ long long wt[32];
   const int tid = threadIdx.x;
-  long long run = 0;
+  long long run = 0, run_tiles = 0;
   for (int s0 = 0; s0 < n_seqs; s0 += kScanThreads) {
     int s = s0 + tid;
     long long nh = 0;
@@ -50,8 +50,11 @@ k_setup(const int32_t* __restrict__ cu, int n_seqs, int n_kv_heads, int window, 
     long long tot, ex = block_excl_scan<long long>(nh, wt, &tot);
     if (s < n_seqs) hist_off[s] = run + ex;
     run += tot;
+    ex = block_excl_scan<long long>((nh + 127) >> 7, wt, &tot);     // 128-key tiles of the tensor-core path
+    if (s < n_seqs) tile_off[s] = (int32_t)(run_tiles + ex);
+    run_tiles += tot;
   }
-  if (tid == 0) hist_off[n_seqs] = run;
+  if (tid == 0) { hist_off[n_seqs] = run; tile_off[n_seqs] = (int32_t)run_tiles; }
   if (budgets == nullptr) return;
   const int n_seg = n_seqs * n_kv_heads;
   run = 0;
@@ -206,7 +209,7 @@ cudaError_t launch_setup(const Problem& pb, const int32_t* budgets, int32_t* off
                          int32_t* status, cudaStream_t st, int* launches) {
   LaunchScope scope(KID_SETUP, st, launches);
   k_setup<<<1, kScanThreads, 0, st>>>(pb.cu, pb.p.n_seqs, pb.p.n_kv_heads, pb.p.window, budgets, pb.hist_off,
-                                      offsets, (long long)capacity, status);
+                                      pb.tile_off, offsets, (long long)capacity, status);
   return cudaGetLastError();
 }
 

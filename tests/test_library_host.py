@@ -65,15 +65,15 @@ def test_bad_enums_and_alignment(L):
                      (dict(softmax_domain=1), "BAD_DTYPE"), (dict(score_path=9), "BAD_DTYPE"),
                      (dict(k_stride_tok=257), "BAD_ALIGN")]:
         p = params(**kw)
-        rc = L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, fake, 1 << 30, None)
+        rc = L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, None, fake, 1 << 30, None)
         assert rc == B.ERR[code], (kw, rc)
     p = params()
-    assert L.slkv_score(C.byref(p), None, fake, fake, cu, fake, fake, 1 << 30, None) == B.ERR["NULL_PTR"]
-    assert L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, None, 0, None) == B.ERR["WORKSPACE"]
-    assert L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, fake, 16, None) == B.ERR["WORKSPACE"]
-    assert L.slkv_score(C.byref(p), C.c_void_p(4100), fake, fake, cu, fake, fake, 1 << 30, None) == B.ERR["BAD_ALIGN"]
+    assert L.slkv_score(C.byref(p), None, fake, fake, cu, fake, None, fake, 1 << 30, None) == B.ERR["NULL_PTR"]
+    assert L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, None, None, 0, None) == B.ERR["WORKSPACE"]
+    assert L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, None, fake, 16, None) == B.ERR["WORKSPACE"]
+    assert L.slkv_score(C.byref(p), C.c_void_p(4100), fake, fake, cu, fake, None, fake, 1 << 30, None) == B.ERR["BAD_ALIGN"]
     bad_cu = (C.c_int32 * 2)(0, -5)
-    assert L.slkv_score(C.byref(p), fake, fake, fake, bad_cu, fake, fake, 1 << 30, None) == B.ERR["BAD_SHAPE"]
+    assert L.slkv_score(C.byref(p), fake, fake, fake, bad_cu, fake, None, fake, 1 << 30, None) == B.ERR["BAD_SHAPE"]
 
 
 def test_alloc_argument_errors(L):
