@@ -188,6 +188,16 @@ int slkv_profile_collect(float* total_ms, int32_t* launches, int32_t n_kernels);
 const char* slkv_kernel_name(int kernel_id);
 int slkv_kernel_count(void);
 
+/*
+ * Timeline tracing of the tensor-core score kernels (diagnostics; no counterpart in the paper).
+ * With a device buffer set on the calling thread, every CTA of the two score kernels stores %globaltimer
+ * nanosecond stamps into it: 64 uint64 slots per CTA, pass 1 first (n_cta * 64 entries), pass 2 after
+ * it.  Slots: 0 CTA start, 1 set-up done, 2 query tile landed, 3 first key tile landed, 4 CTA end,
+ * 8+2i / 9+2i start / end of the softmax arithmetic on the CTA's i-th tile (i < 28).  The buffer must hold
+ * 2 * n_cta * 64 * 8 bytes (n_cta <= number of SMs); smaller buffers switch tracing off.  NULL switches it off.
+ */
+int slkv_trace_set_buffer(void* dev_buf, size_t bytes);
+
 /* Library version, major*10000 + minor*100 + patch. */
 int slkv_version(void);
 

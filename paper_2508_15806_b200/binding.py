@@ -81,6 +81,8 @@ def lib() -> C.CDLL:
         L.slkv_kernel_name.restype = C.c_char_p
         L.slkv_kernel_name.argtypes = [C.c_int]
         L.slkv_kernel_count.restype = C.c_int
+        L.slkv_trace_set_buffer.restype = C.c_int
+        L.slkv_trace_set_buffer.argtypes = [C.c_void_p, C.c_size_t]
         _lib = L
     return _lib
 
@@ -209,3 +211,11 @@ def slkv_profile_collect() -> dict:
     if rc != SLKV_OK:
         raise SlkvError(rc, "slkv_profile_collect")
     return {lib().slkv_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i] > 0}
+
+
+def slkv_trace_set_buffer(buf: Optional[torch.Tensor]) -> None:
+    """buf: CUDA int64 tensor that receives the score kernels' timeline stamps, or None to switch tracing off."""
+    if buf is None:
+        lib().slkv_trace_set_buffer(None, 0)
+    else:
+        lib().slkv_trace_set_buffer(buf.data_ptr(), buf.numel() * buf.element_size())

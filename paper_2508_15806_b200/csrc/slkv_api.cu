@@ -143,13 +143,11 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path) {
 
 bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
 
-// score -> pooled (device pointers resolved); shared by slkv_score and slkv_compress
-int enqueue_score(const Problem& pb, int path, const int32_t* cu_host, float* pooled, int32_t* status,
-                  cudaStream_t st, int* launches) {
+// window votes of every history key (device pointers resolved)
+int enqueue_votes(const Problem& pb, int path, const int32_t* cu_host, int32_t* status, cudaStream_t st,
+                  int* launches) {
   cudaError_t e = path == SLKV_PATH_TENSOR ? launch_score_tensor(pb, cu_host, status, st, launches)
                                            : launch_score_simt(pb, st, launches);
-  if (e != cudaSuccess) return cuda_fail(e);
-  e = launch_pool(pb, pooled, st, launches);
   if (e != cudaSuccess) return cuda_fail(e);
   return SLKV_OK;
 }
@@ -174,13 +172,22 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
   if (rc != SLKV_OK) return rc;
   pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
   int launches = 0;
-  cudaError_t e = launch_setup(pb, budgets, offsets, capacity, status, st, &launches);
+  const bool clustered = select_cluster_supported(pb);
+  cudaError_t e = launch_setup(pb, clustered ? nullptr : budgets, offsets, capacity, status, st, &launches);
   if (e != cudaSuccess) return cuda_fail(e);
-  float* pooled = pooled_opt ? pooled_opt : pb.pooled_ws;
-  rc = enqueue_score(pb, path, cu_host, pooled, status, st, &launches);
+  rc = enqueue_votes(pb, path, cu_host, status, st, &launches);
   if (rc != SLKV_OK) return rc;
-  e = launch_select(pb, pooled, budgets, offsets, kept_idx, capacity, st, &launches);
-  if (e != cudaSuccess) return cuda_fail(e);
+  if (clustered) {
+    // pooling, offsets and selection in one cluster kernel
+    e = launch_select_cluster(pb, pooled_opt, budgets, offsets, kept_idx, capacity, status, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+  } else {
+    float* pooled = pooled_opt ? pooled_opt : pb.pooled_ws;
+    e = launch_pool(pb, pooled, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_select(pb, pooled, budgets, offsets, kept_idx, capacity, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   e = launch_gather(pb, offsets, kept_idx, k_out, v_out, capacity, st, &launches);
   if (e != cudaSuccess) return cuda_fail(e);
   g_last_launches = launches;
@@ -258,6 +265,11 @@ const char* slkv_kernel_name(int kernel_id) {
 
 int slkv_kernel_count(void) { return KID_COUNT; }
 
+int slkv_trace_set_buffer(void* dev_buf, size_t bytes) {
+  set_tensor_trace(dev_buf, dev_buf ? bytes : 0);
+  return SLKV_OK;
+}
+
 int slkv_last_cuda_error(void) { return g_last_cuda_error; }
 int slkv_last_launch_count(void) { return g_last_launches; }
 int slkv_version(void) { return 100; }
@@ -311,8 +323,10 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
   int launches = 0;
   cudaError_t e = launch_setup(pb, nullptr, nullptr, 0, nullptr, st, &launches);
   if (e != cudaSuccess) return cuda_fail(e);
-  rc = enqueue_score(pb, path, cu_seqlens_host, pooled, status, st, &launches);
+  rc = enqueue_votes(pb, path, cu_seqlens_host, status, st, &launches);
   if (rc != SLKV_OK) return rc;
+  e = launch_pool(pb, pooled, st, &launches);
+  if (e != cudaSuccess) return cuda_fail(e);
   g_last_launches = launches;
   return SLKV_OK;
 }

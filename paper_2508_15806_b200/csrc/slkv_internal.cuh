@@ -60,11 +60,16 @@ size_t simt_smem_bytes(const Problem& pb);
 cudaError_t launch_score_simt(const Problem& pb, cudaStream_t st, int* launches);
 bool tensor_path_supported(const slkv_params& p);
 int tensor_slot_stride(const Problem& pb);
+void set_tensor_trace(void* dev_buf, size_t bytes);
 cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, cudaStream_t st,
                                 int* launches);
 cudaError_t launch_pool(const Problem& pb, float* pooled, cudaStream_t st, int* launches);
 cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t capacity, cudaStream_t st, int* launches);
+bool select_cluster_supported(const Problem& pb);
+cudaError_t launch_select_cluster(const Problem& pb, float* pooled_out, const int32_t* budgets, int32_t* offsets,
+                                  int32_t* kept_idx, int64_t capacity, int32_t* status, cudaStream_t st,
+                                  int* launches);
 cudaError_t launch_gather(const Problem& pb, const int32_t* offsets, const int32_t* kept_idx, void* k_out,
                           void* v_out, int64_t capacity, cudaStream_t st, int* launches);
 

@@ -25,6 +25,8 @@ constexpr int kHalfBytes = kTileKeys * 128;    // one 64-element (128-byte) half
 constexpr int kStageBytes = 2 * kHalfBytes;    // 32 KB
 constexpr int kThreads = 384;                  // warps 0-3: TMA, MMA, 2 idle; warps 4-11: epilogue
 constexpr int kEpiThreads = 256;
+constexpr int kTraceSlots = 64;               // per CTA: 0 start, 1 set-up done, 2 Q landed, 3 first K landed,
+                                               // 4 end; 8+2i / 9+2i = epilogue of the CTA's i-th tile begins / ends
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per wait
 
 struct TcArgs {
@@ -35,6 +37,7 @@ struct TcArgs {
   float* part_z;
   float* vote;
   int32_t* status;
+  unsigned long long* trace;    // optional timeline buffer: kTraceSlots timestamps (ns) per CTA, or null
   int n_seqs, n_kv_heads, G, window, R, MT, slot_stride, tiles_per_cta, total_tiles;
   int q_head_inner, k_head_inner;   // tensor-map dimension order: 1 = the head axis comes before the row axis
   float scale_log2;
@@ -65,6 +68,9 @@ __device__ __forceinline__ unsigned long long now_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
+}
+__device__ __forceinline__ void trace_mark(const unsigned long long* base, int slot) {
+  if (base) const_cast<unsigned long long*>(base)[(size_t)blockIdx.x * kTraceSlots + slot] = now_ns();
 }
 // Waits for the phase with the given parity.  false = gave up (limit reached or another thread did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
@@ -103,8 +109,14 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Issues a TMEM load of 32 consecutive columns of this thread's lane; the registers are valid only after
+// tc_ld_wait on the same array.
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
       "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
@@ -113,14 +125,16 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
+// Waits for this thread's outstanding TMEM loads; naming the registers keeps their uses behind the wait.
+__device__ __forceinline__ void tc_ld_wait(uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+        "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+        "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+        "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
 }
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
@@ -135,23 +149,54 @@ __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
 
 struct Run { int s, g, t0, count, n_hist, seg_tile0, tiles_seg; };
 
-// The run of tiles starting at global tile `gt` that stays inside one segment and before `end`.
-__device__ __forceinline__ Run locate(const TcArgs& a, int gt, int end) {
-  int lo = 0, hi = a.n_seqs;                       // last s with Hkv*tile_off[s] <= gt
+// A run = consecutive tiles of one segment inside the CTA's range [begin, end).  Forward walks (pass 1)
+// name a run by its first tile, backward walks (pass 2) by its last one.
+template <bool REV>
+__device__ __forceinline__ Run locate(const TcArgs& a, int pos, int begin, int end) {
+  int lo = 0, hi = a.n_seqs;                       // last s with Hkv*tile_off[s] <= pos
   while (hi - lo > 1) {
     int mid = (lo + hi) >> 1;
-    if (a.n_kv_heads * a.tile_off[mid] <= gt) lo = mid; else hi = mid;
+    if (a.n_kv_heads * a.tile_off[mid] <= pos) lo = mid; else hi = mid;
   }
   Run r;
   r.s = lo;
   r.tiles_seg = a.tile_off[lo + 1] - a.tile_off[lo];
-  const int rel = gt - a.n_kv_heads * a.tile_off[lo];
+  const int rel = pos - a.n_kv_heads * a.tile_off[lo];
   r.g = rel / r.tiles_seg;
-  r.t0 = rel - r.g * r.tiles_seg;
-  r.seg_tile0 = gt - r.t0;
-  r.count = min(end - gt, r.tiles_seg - r.t0);
+  const int t = rel - r.g * r.tiles_seg;
+  r.seg_tile0 = pos - t;
+  if (REV) {
+    r.t0 = max(r.seg_tile0, begin) - r.seg_tile0;
+    r.count = t - r.t0 + 1;
+  } else {
+    r.t0 = t;
+    r.count = min(end - pos, r.tiles_seg - t);
+  }
   r.n_hist = max(a.cu[lo + 1] - a.cu[lo] - a.window, 0);
   return r;
+}
+
+// sum_e 2^(v_e * sc - m) over 32 accumulator values, four independent chains
+__device__ __forceinline__ float sum_ex2_32(const uint32_t (&r)[32], float sc, float m) {
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < 32; e += 4) {
+    s0 += ex2(fmaf(__uint_as_float(r[e]), sc, -m));
+    s1 += ex2(fmaf(__uint_as_float(r[e + 1]), sc, -m));
+    s2 += ex2(fmaf(__uint_as_float(r[e + 2]), sc, -m));
+    s3 += ex2(fmaf(__uint_as_float(r[e + 3]), sc, -m));
+  }
+  return (s0 + s1) + (s2 + s3);
+}
+__device__ __forceinline__ float max_32(const uint32_t (&r)[32], int n_valid_here) {
+  float t[32];
+#pragma unroll
+  for (int e = 0; e < 32; ++e) t[e] = e < n_valid_here ? __uint_as_float(r[e]) : -INFINITY;
+#pragma unroll
+  for (int w = 16; w >= 1; w >>= 1)
+#pragma unroll
+    for (int e = 0; e < w; ++e) t[e] = fmaxf(t[e], t[e + w]);
+  return t[0];
 }
 
 template <int PASS>
@@ -184,6 +229,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const int begin = blockIdx.x * a.tiles_per_cta;
   const int end = min(begin + a.tiles_per_cta, a.total_tiles);
 
+  if (tid == 0) trace_mark(a.trace, 0);
   if (tid == 0) {
     abort_sh = 0;
     for (int st = 0; st < kStages; ++st) { mbar_init(full_bar(st), 1); mbar_init(empty_bar(st), 1); }
@@ -203,14 +249,21 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_sh;
+  if (tid == 0) trace_mark(a.trace, 1);
+
+  constexpr bool REV = PASS == 2;      // pass 2 walks the CTA's tiles backwards: the last ones read are likeliest in L2
+  const int pos0 = REV ? end - 1 : begin;
+  auto more = [&](int pos) { return REV ? pos >= begin : pos < end; };
+  auto advance = [&](int pos, const Run& r) { return REV ? pos - r.count : pos + r.count; };
+  auto tile_of = [&](const Run& r, int i) { return r.t0 + (REV ? r.count - 1 - i : i); };
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       int it = 0, run_idx = 0;
       bool ok = true;
-      for (int gt = begin; gt < end && ok;) {
-        const Run r = locate(a, gt, end);
+      for (int pos = pos0; more(pos) && ok;) {
+        const Run r = locate<REV>(a, pos, begin, end);
         ok = mbar_wait(qempty_bar, (run_idx & 1) ^ 1, abort_flag);      // previous run's MMAs are done with Q
         if (!ok) break;
         mbar_expect_tx(qfull_bar, 2u * (uint32_t)R * 128u);
@@ -218,17 +271,17 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tma_load_4d(q_smem, &tm_q, 0, qy, qz, r.s, qfull_bar);
         tma_load_4d(q_smem + q_half_bytes, &tm_q, 64, qy, qz, r.s, qfull_bar);
         const int tok0 = a.cu[r.s];
-        for (int t = 0; t < r.count; ++t, ++it) {
+        for (int i = 0; i < r.count; ++i, ++it) {
           const int st = it % kStages;
           ok = mbar_wait(empty_bar(st), ((it / kStages) & 1) ^ 1, abort_flag);
           if (!ok) break;
           mbar_expect_tx(full_bar(st), kStageBytes);
-          const int tok = tok0 + (r.t0 + t) * kTileKeys;
+          const int tok = tok0 + tile_of(r, i) * kTileKeys;
           const int ky = a.k_head_inner ? r.g : tok, kz = a.k_head_inner ? tok : r.g;
           tma_load_3d(k_smem + st * kStageBytes, &tm_k, 0, ky, kz, full_bar(st));
           tma_load_3d(k_smem + st * kStageBytes + kHalfBytes, &tm_k, 64, ky, kz, full_bar(st));
         }
-        gt += r.count;
+        pos = advance(pos, r);
         ++run_idx;
       }
       if (!ok) {
@@ -247,15 +300,17 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const uint32_t idesc = PASS == 1 ? instr_desc(128, kTileKeys) : instr_desc(kTileKeys, R);
       int it = 0, run_idx = 0;
       bool ok = true;
-      for (int gt = begin; gt < end && ok;) {
-        const Run r = locate(a, gt, end);
+      for (int pos = pos0; more(pos) && ok;) {
+        const Run r = locate<REV>(a, pos, begin, end);
         ok = mbar_wait(qfull_bar, run_idx & 1, abort_flag);
         if (!ok) break;
-        for (int t = 0; t < r.count; ++t, ++it) {
+        if (run_idx == 0) trace_mark(a.trace, 2);
+        for (int i = 0; i < r.count; ++i, ++it) {
           const int st = it % kStages, b = it % n_bufs;
           ok = mbar_wait(full_bar(st), (it / kStages) & 1, abort_flag) &&
                mbar_wait(acce_bar(b), ((it / n_bufs) & 1) ^ 1, abort_flag);
           if (!ok) break;
+          if (it == 0) trace_mark(a.trace, 3);
           tc_fence_after();
           const uint32_t kst = k_smem + st * kStageBytes;
           const uint32_t d0 = tmem_base + (uint32_t)(b * buf_cols);
@@ -279,7 +334,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           tc_commit(accf_bar(b));         // accumulator ready for the epilogue
         }
         tc_commit(qempty_bar);            // Q tile free once the run's MMAs are done
-        gt += r.count;
+        pos = advance(pos, r);
         ++run_idx;
       }
     }
@@ -293,8 +348,8 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const float inv_g = 1.0f / (float)a.G;
     int it = 0, run_idx = 0;
     bool ok = true;
-    for (int gt = begin; gt < end;) {
-      const Run r = locate(a, gt, end);
+    for (int pos = pos0; more(pos);) {
+      const Run r = locate<REV>(a, pos, begin, end);
       const int seg = r.s * a.n_kv_heads + r.g;
       const int first_cta = r.seg_tile0 / a.tiles_per_cta;
       float m_run[2] = {-INFINITY, -INFINITY}, z_run[2] = {0.f, 0.f};
@@ -313,66 +368,100 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
         epi_bar();
       }
-      for (int t = 0; t < r.count; ++t, ++it) {
+      for (int i = 0; i < r.count; ++i, ++it) {
         if ((it & 1) != wg) continue;
         const int b = it % n_bufs;
         if (ok) ok = mbar_wait(accf_bar(b), (it / n_bufs) & 1, abort_flag);
         ok = __all_sync(0xffffffffu, ok) != 0;         // the TMEM loads below need the whole warp
         if (!ok) continue;
         tc_fence_after();
-        const int key0 = (r.t0 + t) * kTileKeys;
+        if (row == 0 && it < 28) trace_mark(a.trace, 8 + 2 * it);
+        const int key0 = tile_of(r, i) * kTileKeys;
         const uint32_t tb = tmem_base + lane_sel + (uint32_t)(b * buf_cols);
+        uint32_t ra[32], rb[32];
         if (PASS == 1) {
           const int n_valid = min(r.n_hist - key0, kTileKeys);
           for (int mt = 0; mt < MT; ++mt) {
+            const uint32_t tcol = tb + mt * 128;
             float m = m_run[mt], z = z_run[mt];
+            bool exact = !(m > -INFINITY) || n_valid < kTileKeys;
+            if (!exact) {
+              // Optimistic: keep the reference maximum m of earlier tiles (any m gives the same log-sum-exp
+              // as long as nothing overflows); an overflow shows as a non-finite sum and is redone exactly.
+              float zt = z;
+              tc_ld32_issue(tcol, ra);
+              tc_ld_wait(ra);
+              tc_ld32_issue(tcol + 32, rb);
+              zt += sum_ex2_32(ra, sc, m);
+              tc_ld_wait(rb);
+              tc_ld32_issue(tcol + 64, ra);
+              zt += sum_ex2_32(rb, sc, m);
+              tc_ld_wait(ra);
+              tc_ld32_issue(tcol + 96, rb);
+              zt += sum_ex2_32(ra, sc, m);
+              tc_ld_wait(rb);
+              zt += sum_ex2_32(rb, sc, m);
+              if (zt < INFINITY) z = zt; else exact = true;
+            }
+            if (exact) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
-              float v[32];
-              tc_ld32(tb + mt * 128 + c0, v);
-              if (n_valid < kTileKeys) {
-#pragma unroll
-                for (int e = 0; e < 32; ++e) if (c0 + e >= n_valid) v[e] = -INFINITY;
-              }
-              float cm = v[0];
-#pragma unroll
-              for (int e = 1; e < 32; ++e) cm = fmaxf(cm, v[e]);
-              const float mn = fmaxf(m, cm * sc);
-              if (mn > -INFINITY) {
+              for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
+                if (c0 >= n_valid) break;
+                tc_ld32_issue(tcol + c0, ra);
+                tc_ld_wait(ra);
+                const float mn = fmaxf(m, max_32(ra, n_valid - c0) * sc);
                 z *= ex2(m - mn);
                 m = mn;
-                float s0 = 0.f, s1 = 0.f;
+                float zc = 0.f;
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                  s0 += ex2(fmaf(v[e], sc, -m));
-                  s1 += ex2(fmaf(v[e + 1], sc, -m));
-                }
-                z += s0 + s1;
+                for (int e = 0; e < 32; ++e)
+                  if (e < n_valid - c0) zc += ex2(fmaf(__uint_as_float(ra[e]), sc, -m));
+                z += zc;
               }
             }
             m_run[mt] = m; z_run[mt] = z;
           }
         } else {
-          float acc0 = 0.f, acc1 = 0.f;
+          float acc = 0.f;
+          tc_ld32_issue(tb, ra);
 #pragma unroll 1
-          for (int c0 = 0; c0 < R; c0 += 32) {
-            float v[32];
-            tc_ld32(tb + c0, v);
+          for (int c0 = 0; c0 < R; c0 += 64) {
+            tc_ld_wait(ra);
+            if (c0 + 32 < R) tc_ld32_issue(tb + c0 + 32, rb);
+            {
+              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-            for (int e = 0; e < 32; e += 4) {
-              const float4 l4 = *reinterpret_cast<const float4*>(lse + c0 + e);
-              acc0 += ex2(fmaf(v[e], sc, -l4.x));
-              acc1 += ex2(fmaf(v[e + 1], sc, -l4.y));
-              acc0 += ex2(fmaf(v[e + 2], sc, -l4.z));
-              acc1 += ex2(fmaf(v[e + 3], sc, -l4.w));
+              for (int e = 0; e < 32; e += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(lse + c0 + e);
+                s0 += ex2(fmaf(__uint_as_float(ra[e]), sc, -l4.x));
+                s1 += ex2(fmaf(__uint_as_float(ra[e + 1]), sc, -l4.y));
+                s2 += ex2(fmaf(__uint_as_float(ra[e + 2]), sc, -l4.z));
+                s3 += ex2(fmaf(__uint_as_float(ra[e + 3]), sc, -l4.w));
+              }
+              acc += (s0 + s1) + (s2 + s3);
+            }
+            if (c0 + 32 < R) {
+              tc_ld_wait(rb);
+              if (c0 + 64 < R) tc_ld32_issue(tb + c0 + 64, ra);
+              float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+              for (int e = 0; e < 32; e += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(lse + c0 + 32 + e);
+                s0 += ex2(fmaf(__uint_as_float(rb[e]), sc, -l4.x));
+                s1 += ex2(fmaf(__uint_as_float(rb[e + 1]), sc, -l4.y));
+                s2 += ex2(fmaf(__uint_as_float(rb[e + 2]), sc, -l4.z));
+                s3 += ex2(fmaf(__uint_as_float(rb[e + 3]), sc, -l4.w));
+              }
+              acc += (s0 + s1) + (s2 + s3);
             }
           }
           const int j = key0 + row;
-          if (j < r.n_hist) a.vote[a.hist_off[r.s] * a.n_kv_heads + (long long)r.g * r.n_hist + j] = (acc0 + acc1) * inv_g;
+          if (j < r.n_hist) a.vote[a.hist_off[r.s] * a.n_kv_heads + (long long)r.g * r.n_hist + j] = acc * inv_g;
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(acce_bar(b));
+        if (row == 0 && it < 28) trace_mark(a.trace, 9 + 2 * it);
       }
       if (PASS == 1) {
         // combine the two warpgroups' statistics and publish this CTA's partial for the segment
@@ -394,7 +483,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           epi_bar();
         }
       }
-      gt += r.count;
+      pos = advance(pos, r);
       ++run_idx;
     }
   }
@@ -402,6 +491,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   if (abort_sh && tid == 0 && a.status) atomicExch(a.status, (int)SLKV_ERR_DEVICE_TIMEOUT);
+  if (tid == 0) trace_mark(a.trace, 4);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -438,6 +528,15 @@ int sm_count() {
 
 struct Schedule { int total_tiles, tiles_per_cta, n_cta; };
 
+// Timeline tracing (diagnostics): a caller-owned device buffer, two halves (pass 1, pass 2).
+thread_local unsigned long long* g_trace = nullptr;
+thread_local size_t g_trace_bytes = 0;
+unsigned long long* trace_buffer(int pass, int n_cta) {
+  const size_t need = (size_t)n_cta * kTraceSlots * sizeof(unsigned long long);
+  if (!g_trace || g_trace_bytes < 2 * need) return nullptr;
+  return g_trace + (pass - 1) * (size_t)n_cta * kTraceSlots;
+}
+
 Schedule schedule_of(const Problem& pb, const int32_t* cu_host) {
   long long tiles = 0;
   for (int s = 0; s < pb.p.n_seqs; ++s) {
@@ -453,6 +552,11 @@ Schedule schedule_of(const Problem& pb, const int32_t* cu_host) {
 }
 
 }  // namespace
+
+void set_tensor_trace(void* dev_buf, size_t bytes) {
+  g_trace = static_cast<unsigned long long*>(dev_buf);
+  g_trace_bytes = bytes;
+}
 
 bool tensor_path_supported(const slkv_params& p) {
   if (p.dtype != SLKV_BF16 || p.head_dim != 128) return false;
@@ -511,6 +615,7 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
   TcArgs a;
   a.cu = pb.cu; a.hist_off = pb.hist_off; a.tile_off = pb.tile_off;
   a.part_m = pb.part_m; a.part_z = pb.part_z; a.vote = pb.vote; a.status = status;
+  a.trace = nullptr;
   a.n_seqs = p.n_seqs; a.n_kv_heads = p.n_kv_heads; a.G = pb.G; a.window = p.window; a.R = pb.R;
   a.MT = (pb.R + 127) / 128;
   a.q_head_inner = q_head_inner; a.k_head_inner = k_head_inner;
@@ -532,11 +637,13 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
   }
   {
     LaunchScope scope(KID_SCORE_LSE, st, launches);
+    a.trace = trace_buffer(1, sc.n_cta);
     k_score_tc<1><<<sc.n_cta, kThreads, smem, st>>>(tm_q, tm_k, a);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
   LaunchScope scope(KID_SCORE_VOTE, st, launches);
+  a.trace = trace_buffer(2, sc.n_cta);
   k_score_tc<2><<<sc.n_cta, kThreads, smem, st>>>(tm_q, tm_k, a);
   return cudaGetLastError();
 }
