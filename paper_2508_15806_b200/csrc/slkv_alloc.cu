@@ -43,6 +43,8 @@ k_alloc(const float* __restrict__ inf, int L, int H, int fixed, long long total,
   __shared__ int sh_bad, sh_uniform;
   const int tid = threadIdx.x;
   const long long D = total - (long long)N * fixed;
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (tid == 0) sh_bad = 0;
   __syncthreads();

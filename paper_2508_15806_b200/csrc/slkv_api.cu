@@ -88,6 +88,22 @@ int describe(const slkv_params* p, const int32_t* cu_host, Problem* pb) {
   pb->total_tokens = T;
   pb->total_hist = total_hist;
   pb->n_seg = p->n_seqs * p->n_kv_heads;
+  if (p->n_seqs <= kInlineSeqs) {
+    pb->tab.n_inline = p->n_seqs;
+    long long hacc = 0;
+    int tacc = 0;
+    for (int s = 0; s <= p->n_seqs; ++s) {
+      pb->tab.cu[s] = cu_host[s];
+      pb->tab.hist_off[s] = hacc;
+      pb->tab.tile_off[s] = tacc;
+      if (s < p->n_seqs) {
+        long long nh = (long long)cu_host[s + 1] - cu_host[s] - p->window;
+        if (nh < 0) nh = 0;
+        hacc += nh;
+        tacc += (int)((nh + 127) / 128);
+      }
+    }
+  }
   if (pb->n_seg > 65535 * 16) return SLKV_ERR_BAD_SHAPE;
   if (pb->R > 1024) return SLKV_ERR_BAD_SHAPE;
   return SLKV_OK;
@@ -129,6 +145,8 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path) {
   unsigned char* b = static_cast<unsigned char*>(ws);
   pb->hist_off = reinterpret_cast<int64_t*>(b + L.hist_off);
   pb->tile_off = reinterpret_cast<int32_t*>(b + L.tile_off);
+  pb->tab.tile_ptr = pb->tile_off;
+  pb->tab.hist_ptr = reinterpret_cast<const long long*>(pb->hist_off);
   pb->vote = reinterpret_cast<float*>(b + L.vote);
   pb->pooled_ws = reinterpret_cast<float*>(b + L.pooled);
   pb->part_m = reinterpret_cast<float*>(b + L.part_m);
@@ -171,10 +189,14 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
   rc = bind_workspace(&pb, ws, ws_bytes, path);
   if (rc != SLKV_OK) return rc;
   pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
+  pb.tab.cu_ptr = cu_dev;
   int launches = 0;
   const bool clustered = select_cluster_supported(pb);
-  cudaError_t e = launch_setup(pb, clustered ? nullptr : budgets, offsets, capacity, status, st, &launches);
-  if (e != cudaSuccess) return cuda_fail(e);
+  cudaError_t e = cudaSuccess;
+  if (!clustered || pb.tab.n_inline == 0) {       // tables in global memory and / or the packed offsets
+    e = launch_setup(pb, clustered ? nullptr : budgets, offsets, capacity, status, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   rc = enqueue_votes(pb, path, cu_host, status, st, &launches);
   if (rc != SLKV_OK) return rc;
   if (clustered) {
@@ -319,10 +341,14 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
   rc = bind_workspace(&pb, workspace, workspace_bytes, path);
   if (rc != SLKV_OK) return rc;
   pb.cu = cu_seqlens_dev; pb.q = q_win; pb.k = k; pb.v = nullptr;
+  pb.tab.cu_ptr = cu_seqlens_dev;
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
-  cudaError_t e = launch_setup(pb, nullptr, nullptr, 0, nullptr, st, &launches);
-  if (e != cudaSuccess) return cuda_fail(e);
+  cudaError_t e = cudaSuccess;
+  if (pb.tab.n_inline == 0) {
+    e = launch_setup(pb, nullptr, nullptr, 0, nullptr, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   rc = enqueue_votes(pb, path, cu_seqlens_host, status, st, &launches);
   if (rc != SLKV_OK) return rc;
   e = launch_pool(pb, pooled, st, &launches);

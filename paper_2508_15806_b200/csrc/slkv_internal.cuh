@@ -13,6 +13,59 @@ namespace slkv {
 constexpr double kLayerFloor = 0.01;   // minimum layer budget (Sec. 3.3)
 constexpr float kLog2e = 1.4426950408889634f;
 
+constexpr int kInlineSeqs = 64;
+
+// Per-sequence tables: token starts (cu), exclusive prefixes of the history lengths n_hist_s and of the
+// 128-key tile counts.  Batches of up to kInlineSeqs sequences carry them inside the kernel parameters
+// (filled on the host from cu_seqlens_host); larger batches read the arrays a set-up kernel wrote.
+struct SeqTables {
+  int32_t n_inline;                       // n_seqs when the inline arrays are valid, else 0
+  int32_t cu[kInlineSeqs + 1];
+  int32_t tile_off[kInlineSeqs + 1];
+  long long hist_off[kInlineSeqs + 1];
+  const int32_t* cu_ptr;
+  const int32_t* tile_ptr;
+  const long long* hist_ptr;
+#ifdef __CUDACC__
+  __device__ __forceinline__ int cu_at(int i) const { return n_inline ? cu[i] : cu_ptr[i]; }
+  __device__ __forceinline__ int tile_at(int i) const { return n_inline ? tile_off[i] : tile_ptr[i]; }
+  __device__ __forceinline__ long long hist_at(int i) const { return n_inline ? hist_off[i] : hist_ptr[i]; }
+#endif
+};
+
+// Programmatic dependent launch: a kernel may start while its predecessor in the stream drains; it must
+// not touch global memory the predecessor may write before pdl_wait() returns.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
+// Launches `kernel` with the programmatic-serialisation attribute (and optionally a cluster shape).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              int cluster_x, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster_x > 1) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Everything a score / select / gather launch needs, resolved by the host entry points.
 struct Problem {
   slkv_params p;
@@ -24,6 +77,7 @@ struct Problem {
   int64_t total_hist;     // sum_s n_hist_s
   int n_seg;              // n_seqs * n_kv_heads
   const int32_t* cu;      // dev
+  SeqTables tab;          // per-sequence tables (inline or pointing into the workspace)
   const void* q;          // dev
   const void* k;          // dev
   const void* v;          // dev

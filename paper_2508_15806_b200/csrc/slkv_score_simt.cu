@@ -51,8 +51,8 @@ __device__ __forceinline__ float dot_row(const T* __restrict__ qrow /*smem*/, co
 
 template <typename T, int D, int PASS>
 __global__ void __launch_bounds__(kThreads)
-k_score_simt(const T* __restrict__ q, const T* __restrict__ k, const int32_t* __restrict__ cu,
-             const int64_t* __restrict__ hist_off, float* __restrict__ part_m, float* __restrict__ part_z,
+k_score_simt(const T* __restrict__ q, const T* __restrict__ k, const __grid_constant__ SeqTables tab,
+             float* __restrict__ part_m, float* __restrict__ part_z,
              float* __restrict__ vote, int n_kv_heads, int G, int window, int n_chunks, long long k_stride_tok,
              long long k_stride_head, long long q_stride_seq, long long q_stride_row, long long q_stride_head,
              float scale_log2) {
@@ -67,8 +67,10 @@ k_score_simt(const T* __restrict__ q, const T* __restrict__ k, const int32_t* __
 
   const int chunk = blockIdx.x, g = blockIdx.y, s = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int t0 = cu[s];
-  const int n_hist = max(cu[s + 1] - t0 - window, 0);
+  pdl_launch_dependents();
+  pdl_wait();
+  const int t0 = tab.cu_at(s);
+  const int n_hist = max(tab.cu_at(s + 1) - t0 - window, 0);
   const int key0 = chunk * (kThreads * kTilesPerChunk);
   if (key0 >= n_hist) return;
   const int seg = s * n_kv_heads + g;
@@ -148,7 +150,7 @@ k_score_simt(const T* __restrict__ q, const T* __restrict__ k, const int32_t* __
     } else {
       float acc = 0.f;
       for (int r = 0; r < R; ++r) acc += exp2f(dot_row<T, D>(qs + r * D, kreg) * scale_log2 - run_m[r]);
-      if (valid) vote[hist_off[s] * n_kv_heads + (long long)g * n_hist + j] = acc / (float)G;
+      if (valid) vote[tab.hist_at(s) * n_kv_heads + (long long)g * n_hist + j] = acc / (float)G;
     }
   }
   if (PASS == 1) {
@@ -180,19 +182,17 @@ cudaError_t launch_both(const Problem& pb, cudaStream_t st, int* launches) {
   const slkv_params& p = pb.p;
   {
     LaunchScope scope(KID_SCORE_LSE, st, launches);
-    k_score_simt<T, D, 1><<<grid, kThreads, smem, st>>>(
-        (const T*)pb.q, (const T*)pb.k, pb.cu, pb.hist_off, pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G,
-        p.window, pb.n_chunks, p.k_stride_tok, p.k_stride_head, p.q_stride_seq, p.q_stride_row, p.q_stride_head,
-        scale_log2);
-    e = cudaGetLastError();
+    e = launch_pdl(k_score_simt<T, D, 1>, grid, dim3(kThreads), smem, st, 1, (const T*)pb.q, (const T*)pb.k, pb.tab,
+                   pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G, p.window, pb.n_chunks,
+                   (long long)p.k_stride_tok, (long long)p.k_stride_head, (long long)p.q_stride_seq,
+                   (long long)p.q_stride_row, (long long)p.q_stride_head, scale_log2);
     if (e != cudaSuccess) return e;
   }
   LaunchScope scope(KID_SCORE_VOTE, st, launches);
-  k_score_simt<T, D, 2><<<grid, kThreads, smem, st>>>(
-      (const T*)pb.q, (const T*)pb.k, pb.cu, pb.hist_off, pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G,
-      p.window, pb.n_chunks, p.k_stride_tok, p.k_stride_head, p.q_stride_seq, p.q_stride_row, p.q_stride_head,
-      scale_log2);
-  return cudaGetLastError();
+  return launch_pdl(k_score_simt<T, D, 2>, grid, dim3(kThreads), smem, st, 1, (const T*)pb.q, (const T*)pb.k, pb.tab,
+                    pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G, p.window, pb.n_chunks,
+                    (long long)p.k_stride_tok, (long long)p.k_stride_head, (long long)p.q_stride_seq,
+                    (long long)p.q_stride_row, (long long)p.q_stride_head, scale_log2);
 }
 
 }  // namespace

@@ -30,9 +30,7 @@ constexpr int kTraceSlots = 64;               // per CTA: 0 start, 1 set-up done
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per wait
 
 struct TcArgs {
-  const int32_t* cu;
-  const int64_t* hist_off;
-  const int32_t* tile_off;      // [n_seqs+1] exclusive prefix of ceil(n_hist_s / 128)
+  SeqTables tab;
   float* part_m;
   float* part_z;
   float* vote;
@@ -156,12 +154,12 @@ __device__ __forceinline__ Run locate(const TcArgs& a, int pos, int begin, int e
   int lo = 0, hi = a.n_seqs;                       // last s with Hkv*tile_off[s] <= pos
   while (hi - lo > 1) {
     int mid = (lo + hi) >> 1;
-    if (a.n_kv_heads * a.tile_off[mid] <= pos) lo = mid; else hi = mid;
+    if (a.n_kv_heads * a.tab.tile_at(mid) <= pos) lo = mid; else hi = mid;
   }
   Run r;
   r.s = lo;
-  r.tiles_seg = a.tile_off[lo + 1] - a.tile_off[lo];
-  const int rel = pos - a.n_kv_heads * a.tile_off[lo];
+  r.tiles_seg = a.tab.tile_at(lo + 1) - a.tab.tile_at(lo);
+  const int rel = pos - a.n_kv_heads * a.tab.tile_at(lo);
   r.g = rel / r.tiles_seg;
   const int t = rel - r.g * r.tiles_seg;
   r.seg_tile0 = pos - t;
@@ -172,7 +170,7 @@ __device__ __forceinline__ Run locate(const TcArgs& a, int pos, int begin, int e
     r.t0 = t;
     r.count = min(end - pos, r.tiles_seg - t);
   }
-  r.n_hist = max(a.cu[lo + 1] - a.cu[lo] - a.window, 0);
+  r.n_hist = max(a.tab.cu_at(lo + 1) - a.tab.cu_at(lo) - a.window, 0);
   return r;
 }
 
@@ -201,7 +199,8 @@ __device__ __forceinline__ float max_32(const uint32_t (&r)[32], int n_valid_her
 
 template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
-k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const TcArgs a) {
+k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+           const __grid_constant__ TcArgs a) {
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) unsigned long long bars[2 * kStages + 2 * 4 + 2];
   __shared__ uint32_t tmem_base_sh;
@@ -249,6 +248,9 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_sh;
+  // everything above touched only this CTA's own resources; global inputs are read from here on
+  pdl_launch_dependents();
+  pdl_wait();
   if (tid == 0) trace_mark(a.trace, 1);
 
   constexpr bool REV = PASS == 2;      // pass 2 walks the CTA's tiles backwards: the last ones read are likeliest in L2
@@ -270,7 +272,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const int qy = a.q_head_inner ? r.g * a.G : 0, qz = a.q_head_inner ? 0 : r.g * a.G;
         tma_load_4d(q_smem, &tm_q, 0, qy, qz, r.s, qfull_bar);
         tma_load_4d(q_smem + q_half_bytes, &tm_q, 64, qy, qz, r.s, qfull_bar);
-        const int tok0 = a.cu[r.s];
+        const int tok0 = a.tab.cu_at(r.s);
         for (int i = 0; i < r.count; ++i, ++it) {
           const int st = it % kStages;
           ok = mbar_wait(empty_bar(st), ((it / kStages) & 1) ^ 1, abort_flag);
@@ -456,7 +458,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             }
           }
           const int j = key0 + row;
-          if (j < r.n_hist) a.vote[a.hist_off[r.s] * a.n_kv_heads + (long long)r.g * r.n_hist + j] = acc * inv_g;
+          if (j < r.n_hist) a.vote[a.tab.hist_at(r.s) * a.n_kv_heads + (long long)r.g * r.n_hist + j] = acc * inv_g;
         }
         tc_fence_before();
         __syncwarp();
@@ -613,7 +615,7 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
   }
 
   TcArgs a;
-  a.cu = pb.cu; a.hist_off = pb.hist_off; a.tile_off = pb.tile_off;
+  a.tab = pb.tab;
   a.part_m = pb.part_m; a.part_z = pb.part_z; a.vote = pb.vote; a.status = status;
   a.trace = nullptr;
   a.n_seqs = p.n_seqs; a.n_kv_heads = p.n_kv_heads; a.G = pb.G; a.window = p.window; a.R = pb.R;
@@ -638,14 +640,12 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
   {
     LaunchScope scope(KID_SCORE_LSE, st, launches);
     a.trace = trace_buffer(1, sc.n_cta);
-    k_score_tc<1><<<sc.n_cta, kThreads, smem, st>>>(tm_q, tm_k, a);
-    e = cudaGetLastError();
+    e = launch_pdl(k_score_tc<1>, dim3(sc.n_cta), dim3(kThreads), smem, st, 1, tm_q, tm_k, a);
     if (e != cudaSuccess) return e;
   }
   LaunchScope scope(KID_SCORE_VOTE, st, launches);
   a.trace = trace_buffer(2, sc.n_cta);
-  k_score_tc<2><<<sc.n_cta, kThreads, smem, st>>>(tm_q, tm_k, a);
-  return cudaGetLastError();
+  return launch_pdl(k_score_tc<2>, dim3(sc.n_cta), dim3(kThreads), smem, st, 1, tm_q, tm_k, a);
 }
 
 }  // namespace slkv

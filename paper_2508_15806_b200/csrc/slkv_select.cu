@@ -42,6 +42,8 @@ k_setup(const int32_t* __restrict__ cu, int n_seqs, int n_kv_heads, int window, 
         long long capacity, int32_t* __restrict__ status) {
   __shared__ long long wt[32];
   const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   long long run = 0, run_tiles = 0;
   for (int s0 = 0; s0 < n_seqs; s0 += kScanThreads) {
     int s = s0 + tid;
@@ -77,13 +79,15 @@ k_setup(const int32_t* __restrict__ cu, int n_seqs, int n_kv_heads, int window, 
 
 // pooled[j] = max (or zero-padded mean) of vote[j-r .. j+r] inside the segment's history.
 __global__ void __launch_bounds__(256)
-k_pool(const float* __restrict__ vote, float* __restrict__ pooled, const int32_t* __restrict__ cu,
-       const int64_t* __restrict__ hist_off, int n_kv_heads, int window, int pool_kernel, int pool_mode) {
+k_pool(const float* __restrict__ vote, float* __restrict__ pooled, const __grid_constant__ SeqTables tab,
+       int n_kv_heads, int window, int pool_kernel, int pool_mode) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int s = blockIdx.z, h = blockIdx.y;
-  const int n_hist = max(cu[s + 1] - cu[s] - window, 0);
+  const int n_hist = max(tab.cu_at(s + 1) - tab.cu_at(s) - window, 0);
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n_hist) return;
-  const long long base = hist_off[s] * n_kv_heads + (long long)h * n_hist;
+  const long long base = tab.hist_at(s) * n_kv_heads + (long long)h * n_hist;
   const float* src = vote + base;
   const int r = pool_kernel >> 1;
   const int lo = max(j - r, 0), hi = min(j + r, n_hist - 1);
@@ -103,7 +107,7 @@ k_pool(const float* __restrict__ vote, float* __restrict__ pooled, const int32_t
 // float bit patterns (scores are >= 0, so unsigned order = float order), then writes the positions of
 // the k best in ascending order (equal scores: lower position first) followed by the window positions.
 __global__ void __launch_bounds__(kScanThreads, 1)
-k_select(const float* __restrict__ pooled, const int32_t* __restrict__ cu, const int64_t* __restrict__ hist_off,
+k_select(const float* __restrict__ pooled, const __grid_constant__ SeqTables tab,
          const int32_t* __restrict__ budgets, const int32_t* __restrict__ offsets, int32_t* __restrict__ kept_idx,
          int n_kv_heads, int window, long long capacity) {
   __shared__ int hist[256];
@@ -111,14 +115,16 @@ k_select(const float* __restrict__ pooled, const int32_t* __restrict__ cu, const
   __shared__ unsigned sh_prefix;
   __shared__ int sh_need;
   const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();
   const int seg = blockIdx.x;
   const int s = seg / n_kv_heads, h = seg - s * n_kv_heads;
-  const int len = cu[s + 1] - cu[s];
+  const int len = tab.cu_at(s + 1) - tab.cu_at(s);
   const int n_hist = max(len - window, 0);
   const int n_win = min(len, window);
   const int k = kept_rows(len, budgets[h], window) - n_win;      // history rows to keep (C_H = C - window)
   const long long out0 = offsets[seg];
-  const unsigned* src = reinterpret_cast<const unsigned*>(pooled + hist_off[s] * n_kv_heads + (long long)h * n_hist);
+  const unsigned* src = reinterpret_cast<const unsigned*>(pooled + tab.hist_at(s) * n_kv_heads + (long long)h * n_hist);
 
   // window rows (Algorithm 3 l.4, l.10): always kept, appended after the history rows
   for (int t = tid; t < n_win; t += kScanThreads) {
@@ -180,9 +186,12 @@ k_select(const float* __restrict__ pooled, const int32_t* __restrict__ cu, const
 // Copies the kept rows of K and V into the packed cache: 16 bytes per lane, a row per lane group.
 __global__ void __launch_bounds__(256)
 k_gather(const unsigned char* __restrict__ k, const unsigned char* __restrict__ v, unsigned char* __restrict__ k_out,
-         unsigned char* __restrict__ v_out, const int32_t* __restrict__ cu, const int32_t* __restrict__ offsets,
-         const int32_t* __restrict__ kept_idx, int n_seg, int n_kv_heads, int row_bytes, long long k_tok_bytes,
-         long long k_head_bytes, long long v_tok_bytes, long long v_head_bytes, long long capacity) {
+         unsigned char* __restrict__ v_out, const __grid_constant__ SeqTables tab,
+         const int32_t* __restrict__ offsets, const int32_t* __restrict__ kept_idx, int n_seg, int n_kv_heads,
+         int row_bytes, long long k_tok_bytes, long long k_head_bytes, long long v_tok_bytes,
+         long long v_head_bytes, long long capacity) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lanes = row_bytes >> 4;                       // 16-byte lanes per row (power of two <= 32)
   const int rows_per_cta = blockDim.x / lanes;
   const int lane = threadIdx.x % lanes, sub = threadIdx.x / lanes;
@@ -195,7 +204,7 @@ k_gather(const unsigned char* __restrict__ k, const unsigned char* __restrict__ 
       if ((long long)offsets[mid] <= r) lo = mid; else hi = mid;
     }
     const int s = lo / n_kv_heads, h = lo - s * n_kv_heads;
-    const long long tok = (long long)cu[s] + kept_idx[r];
+    const long long tok = (long long)tab.cu_at(s) + kept_idx[r];
     const uint4 kv = *reinterpret_cast<const uint4*>(k + tok * k_tok_bytes + h * k_head_bytes + lane * 16);
     const uint4 vv = *reinterpret_cast<const uint4*>(v + tok * v_tok_bytes + h * v_head_bytes + lane * 16);
     *reinterpret_cast<uint4*>(k_out + r * row_bytes + lane * 16) = kv;
@@ -208,26 +217,23 @@ k_gather(const unsigned char* __restrict__ k, const unsigned char* __restrict__ 
 cudaError_t launch_setup(const Problem& pb, const int32_t* budgets, int32_t* offsets, int64_t capacity,
                          int32_t* status, cudaStream_t st, int* launches) {
   LaunchScope scope(KID_SETUP, st, launches);
-  k_setup<<<1, kScanThreads, 0, st>>>(pb.cu, pb.p.n_seqs, pb.p.n_kv_heads, pb.p.window, budgets, pb.hist_off,
-                                      pb.tile_off, offsets, (long long)capacity, status);
-  return cudaGetLastError();
+  return launch_pdl(k_setup, dim3(1), dim3(kScanThreads), 0, st, 1, pb.cu, pb.p.n_seqs, pb.p.n_kv_heads,
+                    pb.p.window, budgets, pb.hist_off, pb.tile_off, offsets, (long long)capacity, status);
 }
 
 cudaError_t launch_pool(const Problem& pb, float* pooled, cudaStream_t st, int* launches) {
   if (pb.max_hist <= 0) return cudaSuccess;
   dim3 grid((pb.max_hist + 255) / 256, pb.p.n_kv_heads, pb.p.n_seqs);
   LaunchScope scope(KID_POOL, st, launches);
-  k_pool<<<grid, 256, 0, st>>>(pb.vote, pooled, pb.cu, pb.hist_off, pb.p.n_kv_heads, pb.p.window,
-                               pb.p.pool_kernel, pb.p.pool_mode);
-  return cudaGetLastError();
+  return launch_pdl(k_pool, grid, dim3(256), 0, st, 1, (const float*)pb.vote, pooled, pb.tab, pb.p.n_kv_heads,
+                    pb.p.window, pb.p.pool_kernel, pb.p.pool_mode);
 }
 
 cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t capacity, cudaStream_t st, int* launches) {
   LaunchScope scope(KID_SELECT, st, launches);
-  k_select<<<pb.n_seg, kScanThreads, 0, st>>>(pooled, pb.cu, pb.hist_off, budgets, offsets, kept_idx,
-                                              pb.p.n_kv_heads, pb.p.window, (long long)capacity);
-  return cudaGetLastError();
+  return launch_pdl(k_select, dim3(pb.n_seg), dim3(kScanThreads), 0, st, 1, pooled, pb.tab, budgets, offsets,
+                    kept_idx, pb.p.n_kv_heads, pb.p.window, (long long)capacity);
 }
 
 cudaError_t launch_gather(const Problem& pb, const int32_t* offsets, const int32_t* kept_idx, void* k_out,
@@ -240,11 +246,11 @@ cudaError_t launch_gather(const Problem& pb, const int32_t* offsets, const int32
   long long want = (max_rows + rows_per_cta - 1) / rows_per_cta;
   int grid = (int)(want < 148 * 16 ? want : 148 * 16);
   LaunchScope scope(KID_GATHER, st, launches);
-  k_gather<<<grid, 256, 0, st>>>((const unsigned char*)pb.k, (const unsigned char*)pb.v, (unsigned char*)k_out,
-                                 (unsigned char*)v_out, pb.cu, offsets, kept_idx, pb.n_seg, pb.p.n_kv_heads,
-                                 row_bytes, pb.p.k_stride_tok * pb.elem, pb.p.k_stride_head * pb.elem,
-                                 pb.p.v_stride_tok * pb.elem, pb.p.v_stride_head * pb.elem, (long long)capacity);
-  return cudaGetLastError();
+  return launch_pdl(k_gather, dim3(grid), dim3(256), 0, st, 1, (const unsigned char*)pb.k,
+                    (const unsigned char*)pb.v, (unsigned char*)k_out, (unsigned char*)v_out, pb.tab, offsets, kept_idx,
+                    pb.n_seg, pb.p.n_kv_heads, row_bytes, (long long)(pb.p.k_stride_tok * pb.elem),
+                    (long long)(pb.p.k_stride_head * pb.elem), (long long)(pb.p.v_stride_tok * pb.elem),
+                    (long long)(pb.p.v_stride_head * pb.elem), (long long)capacity);
 }
 
 }  // namespace slkv

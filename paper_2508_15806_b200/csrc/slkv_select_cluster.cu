@@ -22,8 +22,7 @@ constexpr int kMaxCluster = 8;
 struct SelArgs {
   const float* vote;
   float* pooled_out;          // optional
-  const int32_t* cu;
-  const int64_t* hist_off;
+  SeqTables tab;
   const int32_t* budgets;
   int32_t* offsets;
   int32_t* kept_idx;
@@ -59,7 +58,7 @@ __device__ __forceinline__ T block_excl_scan(T v, T* warp_tot /*[32]*/, T* total
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_select_cluster(const SelArgs a) {
+k_select_cluster(const __grid_constant__ SelArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ int hist[2][256];
   __shared__ long long wt[32];
@@ -72,9 +71,11 @@ k_select_cluster(const SelArgs a) {
   const int CS = (int)cluster.num_blocks();
   const int rank = (int)cluster.block_rank();
   const int tid = threadIdx.x, lane = tid & 31;
+  pdl_launch_dependents();
+  pdl_wait();
   const int seg = blockIdx.x / CS;
   const int s = seg / a.n_kv_heads, h = seg - s * a.n_kv_heads;
-  const int len = a.cu[s + 1] - a.cu[s];
+  const int len = a.tab.cu_at(s + 1) - a.tab.cu_at(s);
   const int n_hist = max(len - a.window, 0);
   const int n_win = min(len, a.window);
   const int k_keep = kept_rows(len, a.budgets[h], a.window) - n_win;    // C_H = C - window, clamped
@@ -85,7 +86,7 @@ k_select_cluster(const SelArgs a) {
     long long part = 0;
     for (int g = tid; g < seg; g += kThreads) {
       const int s2 = g / a.n_kv_heads, h2 = g - s2 * a.n_kv_heads;
-      part += kept_rows(a.cu[s2 + 1] - a.cu[s2], a.budgets[h2], a.window);
+      part += kept_rows(a.tab.cu_at(s2 + 1) - a.tab.cu_at(s2), a.budgets[h2], a.window);
     }
     long long tot;
     block_excl_scan<long long>(part, wt, &tot);
@@ -108,7 +109,7 @@ k_select_cluster(const SelArgs a) {
   const int per = ((n_hist + CS - 1) / CS + 3) & ~3;
   const int lo = min(rank * per, n_hist), hi = min(lo + per, n_hist);
   const int n_own = hi - lo;
-  const long long seg_base = a.hist_off[s] * a.n_kv_heads + (long long)h * n_hist;
+  const long long seg_base = a.tab.hist_at(s) * a.n_kv_heads + (long long)h * n_hist;
   const float* vote = a.vote + seg_base;
   const int r = a.pool_kernel >> 1;
   float* sv = reinterpret_cast<float*>(smem_raw);                    // votes of [lo - r, hi + r), then pooled keys
@@ -274,26 +275,14 @@ cudaError_t launch_select_cluster(const Problem& pb, float* pooled_out, const in
     configured_dev = dev;
   }
   SelArgs a;
-  a.vote = pb.vote; a.pooled_out = pooled_out; a.cu = pb.cu; a.hist_off = pb.hist_off; a.budgets = budgets;
+  a.vote = pb.vote; a.pooled_out = pooled_out; a.tab = pb.tab; a.budgets = budgets;
   a.offsets = offsets; a.kept_idx = kept_idx; a.status = status;
   a.n_seqs = pb.p.n_seqs; a.n_kv_heads = pb.p.n_kv_heads; a.window = pb.p.window;
   a.pool_kernel = pb.p.pool_kernel; a.pool_mode = pb.p.pool_mode; a.capacity = capacity;
   a.keys_off = keys_off;
 
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(pb.n_seg * cs));
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)cs;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
   LaunchScope scope(KID_SELECT, st, launches);
-  return cudaLaunchKernelEx(&cfg, k_select_cluster, a);
+  return launch_pdl(k_select_cluster, dim3((unsigned)(pb.n_seg * cs)), dim3(kThreads), smem, st, cs, a);
 }
 
 }  // namespace slkv
