@@ -108,6 +108,27 @@ def rows_of_layer(lens, budgets_row, window):
     return sum(min(n, max(int(c), window)) for n in lens for c in budgets_row)
 
 
+def rank_workload(wl, rank: int, world: int):
+    """Weak scaling: every rank compresses its own sequence batch (same shapes, its own seed)."""
+    if world > 1:
+        wl.seed = wl.seed + 1000 * rank
+    return wl
+
+
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The step time of the job is the slowest rank's (dist = torch.distributed or None)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, tokens_per_rank: int, n_layers: int, ms_per_step: float) -> float:
+    """Tokens per second per layer summed over all ranks (= world * T / t_layer)."""
+    return world * tokens_per_rank * n_layers / (ms_per_step * 1e-3)
+
+
 def run_cuda(args):
     from paper_2508_15806_b200 import binding as B
 
@@ -128,8 +149,7 @@ def run_cuda(args):
     if args.layers:
         wl = synth.small_variant(wl, wl.seq_lens, n_layers=args.layers,
                                  totals=[t // 32 * args.layers for t in wl.totals])
-    if world > 1:
-        wl.seed = wl.seed + 1000 * rank          # weak scaling: every rank compresses its own sequence
+    wl = rank_workload(wl, rank, world)
     total = wl.totals[TOTAL_INDEX]
     cu = wl.cu_seqlens
     T, nl, hkv, d, w = wl.total_tokens, wl.n_layers, wl.n_kv_heads, wl.head_dim, wl.window
@@ -184,12 +204,7 @@ def run_cuda(args):
             fn()
         b.record(stream)
         barrier()
-        ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(a.elapsed_time(b), dist, dev)
 
     warmup = max(args.warmup, 3)
     for _ in range(warmup):
@@ -218,7 +233,7 @@ def run_cuda(args):
 
     ms_per_step = ms_total / steps
     t_layer_us = ms_per_step * 1e3 / nl
-    value = world * T * nl / (ms_per_step * 1e-3)      # = world * T / t_layer: tokens per second per layer
+    value = whole_job_value(world, T, nl, ms_per_step)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies in the timed region)
     e2e = None
@@ -251,7 +266,7 @@ def run_cuda(args):
         h2d = sum((Hh["q"].numel() + Hh["k"].numel() + Hh["v"].numel()) * e + (len(cu) + hkv) * 4
                   for Hh in (host[l % n_host] for l in range(nl)))
         d2h = sum(host[l % n_host]["rows"] * (2 * d * e + 4) + (len(wl.seq_lens) * hkv + 1) * 4 for l in range(nl))
-        e2e = {"value": world * T * nl / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": whole_job_value(world, T, nl, e2e_ms / e2e_steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
                "host_layers_cycled": n_host, "wall_ms": wall_ms,
                "api": "slkv_compress_host (pinned host buffers in, packed rows + offsets + indices out)"}
