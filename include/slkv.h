@@ -171,6 +171,36 @@ int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, c
                        int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx, int64_t* rows_out,
                        void* arena, size_t arena_bytes, void* stream);
 
+/*
+ * slkv_score without a workspace argument, for callers that cannot allocate device memory.  (The paper has
+ * no counterpart: this is a property of the library, not of the method.)
+ *
+ * Who needs it: code that runs inside a host application which has already handed every free byte of the
+ * GPU to its own pool (a serving engine that sizes its KV-cache blocks from "all memory that is left"), or a
+ * plug-in that is given tensors but no handle to the host's allocator.  There cudaMalloc fails, or succeeds
+ * only by synchronising the whole device and shrinking somebody else's pool, and torch's allocator is not
+ * the caller's to use.  Such a caller still owns its inputs and outputs; what it lacks is scratch.
+ *
+ * The scratch is a fixed array of SLKV_NOALLOC_SCRATCH_BYTES inside the library's device image: every GPU
+ * that loads the library holds that much memory until the process exits, used or not.  The call computes
+ * exactly what slkv_score computes, with the same kernels and the same results.
+ *   - Shapes whose slkv_workspace_bytes exceed the array are rejected with SLKV_ERR_WORKSPACE before anything
+ *     is enqueued (32k tokens x 8 KV heads x 128 score rows needs about 4.2 MB).
+ *   - The first call on each device looks up the array's device address (a CUDA runtime query, made with that
+ *     device current) and keeps it; make that first call outside any stream capture.
+ *   - No cudaMalloc, cudaFree or other allocating routine is called, on the first call or later.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left; nothing in it has
+ *     to be zero, each call overwrites what it reads.  Two calls whose kernels may overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them.
+ * Arguments and return value as slkv_score, minus workspace / workspace_bytes.  If the address query fails
+ * the call returns SLKV_ERR_CUDA and slkv_noalloc_last_cuda_error() gives the runtime's code.
+ */
+#define SLKV_NOALLOC_SCRATCH_BYTES (8u << 20)
+int slkv_score_noalloc(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+                       const int32_t* cu_seqlens_host, float* pooled, int32_t* status, void* stream);
+size_t slkv_noalloc_scratch_bytes(void);      /* = SLKV_NOALLOC_SCRATCH_BYTES */
+int slkv_noalloc_last_cuda_error(void);
+
 /* Number of kernels the most recent slkv_score / slkv_compress / slkv_compress_host call on this
  * thread enqueued (launch accounting for benchmarks). */
 int slkv_last_launch_count(void);

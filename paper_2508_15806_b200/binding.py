@@ -74,6 +74,10 @@ def lib() -> C.CDLL:
         L.slkv_compress_host.restype = C.c_int
         L.slkv_compress_host.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, i64, vp, vp, C.POINTER(C.c_int64),
                                          vp, sz, vp]
+        L.slkv_score_noalloc.restype = C.c_int
+        L.slkv_score_noalloc.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp]
+        L.slkv_noalloc_scratch_bytes.restype = sz
+        L.slkv_noalloc_last_cuda_error.restype = C.c_int
         L.slkv_profile_enable.restype = C.c_int
         L.slkv_profile_enable.argtypes = [C.c_int]
         L.slkv_profile_collect.restype = C.c_int
@@ -165,6 +169,22 @@ def slkv_score(params: SlkvParams, q_win: torch.Tensor, k: torch.Tensor, cu_dev:
     if rc != SLKV_OK:
         raise SlkvError(rc, "slkv_score")
     return pooled
+
+
+def slkv_score_noalloc(params: SlkvParams, q_win: torch.Tensor, k: torch.Tensor, cu_dev: torch.Tensor,
+                       cu_seqlens: Sequence[int], pooled: torch.Tensor, status: Optional[torch.Tensor] = None,
+                       stream=None) -> torch.Tensor:
+    """slkv_score for callers that cannot allocate: the scratch is a fixed array inside the library
+    (slkv_noalloc_scratch_bytes() bytes); larger shapes raise SLKV_ERR_WORKSPACE."""
+    rc = lib().slkv_score_noalloc(C.byref(params), q_win.data_ptr(), k.data_ptr(), cu_dev.data_ptr(),
+                                  _cu_host(cu_seqlens), pooled.data_ptr(), _ptr(status), _stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_score_noalloc")
+    return pooled
+
+
+def slkv_noalloc_scratch_bytes() -> int:
+    return int(lib().slkv_noalloc_scratch_bytes())
 
 
 def slkv_compress(params: SlkvParams, q_win, k, v, cu_dev, cu_seqlens: Sequence[int], budgets, k_out, v_out,
