@@ -185,7 +185,7 @@ int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, c
  * that loads the library holds that much memory until the process exits, used or not.  The call computes
  * exactly what slkv_score computes, with the same kernels and the same results.
  *   - Shapes whose slkv_workspace_bytes exceed the array are rejected with SLKV_ERR_WORKSPACE before anything
- *     is enqueued (32k tokens x 8 KV heads x 128 score rows needs about 4.2 MB).
+ *     is enqueued (32k tokens x 8 KV heads x 128 score rows needs about 5.3 MB).
  *   - The first call on each device looks up the array's device address (a CUDA runtime query, made with that
  *     device current) and keeps it; make that first call outside any stream capture.
  *   - No cudaMalloc, cudaFree or other allocating routine is called, on the first call or later.

@@ -41,7 +41,7 @@ int cuda_fail(cudaError_t e) {
 }
 
 struct Layout {
-  size_t hist_off, tile_off, vote, pooled, part_m, part_z, flags, total;
+  size_t hist_off, tile_off, vote, pooled, part_m, part_z, flags, gather_src, total;
 };
 
 // Validates p and cu_seqlens_host and fills the host-known fields of `pb`.
@@ -122,6 +122,7 @@ Layout layout_of(const Problem& pb) {
   L.part_m = o; o = align_up(o + parts);
   L.part_z = o; o = align_up(o + parts);
   L.flags = o; o = align_up(o + 8 * sizeof(int32_t));
+  L.gather_src = o; o = align_up(o + (size_t)pb.p.n_kv_heads * (size_t)pb.total_tokens * sizeof(int32_t));
   L.total = o;
   return L;
 }
@@ -152,6 +153,7 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path) {
   pb->part_m = reinterpret_cast<float*>(b + L.part_m);
   pb->part_z = reinterpret_cast<float*>(b + L.part_z);
   pb->dev_flags = reinterpret_cast<int32_t*>(b + L.flags);
+  pb->gather_src = reinterpret_cast<int32_t*>(b + L.gather_src);
   pb->chunk_keys = path == SLKV_PATH_TENSOR ? 128 : simt_chunk_keys();
   pb->n_chunks = path == SLKV_PATH_TENSOR ? tensor_slot_stride(*pb)
                                           : (pb->max_hist + pb->chunk_keys - 1) / pb->chunk_keys;

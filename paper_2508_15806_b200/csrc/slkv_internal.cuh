@@ -90,6 +90,7 @@ struct Problem {
   int n_chunks;           // chunks per segment (stride of part_*), per score path
   int chunk_keys;         // keys per chunk
   float* pooled_ws;       // [n_kv_heads * total_hist] used when the caller wants no pooled output
+  int32_t* gather_src;    // [n_kv_heads * total_tokens] per packed row: token * n_kv_heads + head of its source
   int32_t* dev_flags;     // [8] scratch words (timeouts etc.)
 };
 

@@ -20,9 +20,11 @@ namespace slkv {
 namespace {
 
 constexpr int kTileKeys = 128;                 // keys per tile (MMA N in pass 1, M in pass 2)
-constexpr int kStages = 4;                     // K tiles in flight in shared memory
+constexpr int kMaxStages = 6;                  // K tiles in flight in shared memory (as many as fit beside Q)
 constexpr int kHalfBytes = kTileKeys * 128;    // one 64-element (128-byte) half of a 128-row tile
 constexpr int kStageBytes = 2 * kHalfBytes;    // 32 KB
+constexpr int kTailBytes = 512 + 2048;         // mbarriers + flags, then 512 floats of row statistics
+constexpr int kSmemLimit = 227 * 1024;         // dynamic shared memory a CTA can have
 constexpr int kThreads = 384;                  // warps 0-3: TMA, MMA, 2 idle; warps 4-11: epilogue
 constexpr int kEpiThreads = 256;
 constexpr int kTraceSlots = 64;               // per CTA: 0 start, 1 set-up done, 2 Q landed, 3 first K landed,
@@ -36,7 +38,7 @@ struct TcArgs {
   float* vote;
   int32_t* status;
   unsigned long long* trace;    // optional timeline buffer: kTraceSlots timestamps (ns) per CTA, or null
-  int n_seqs, n_kv_heads, G, window, R, MT, slot_stride, tiles_per_cta, total_tiles;
+  int n_seqs, n_kv_heads, G, window, R, MT, n_stages, slot_stride, tiles_per_cta, total_tiles;
   int q_head_inner, k_head_inner;   // tensor-map dimension order: 1 = the head axis comes before the row axis
   float scale_log2;
 };
@@ -201,20 +203,27 @@ template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
 k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ TcArgs a) {
-  extern __shared__ unsigned char smem_dyn[];
-  __shared__ __align__(8) unsigned long long bars[2 * kStages + 2 * 4 + 2];
-  __shared__ uint32_t tmem_base_sh;
-  __shared__ int abort_sh;
-  __shared__ __align__(16) float lse_sh[2][256];
-  __shared__ float stat_m[256], stat_z[256];
+  // Shared memory, all dynamic and 1024-byte aligned (the swizzled tiles need it):
+  //   [Q tile: MT x 32 KB][K ring: n_stages x 32 KB][mbarriers, flags: 512 B][row statistics: 2 KB]
+  extern __shared__ __align__(1024) unsigned char smem[];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int MT = a.MT, R = a.R;
+  const int MT = a.MT, R = a.R, kStages = a.n_stages;
   const int buf_cols = MT * 128;
   const int n_bufs = 512 / buf_cols;                        // 4 or 2 TMEM accumulator buffers
   const int q_half_bytes = MT * 128 * 128;                  // one 64-element half of the (padded) Q tile
 
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  unsigned char* tail = smem + 2 * q_half_bytes + kStages * kStageBytes;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);
+  uint32_t& tmem_base_sh = *reinterpret_cast<uint32_t*>(tail + 256);
+  int& abort_sh = *reinterpret_cast<int*>(tail + 260);
+  float* stats = reinterpret_cast<float*>(tail + 512);      // pass 1: stat_m[256], stat_z[256]; pass 2: lse[2][256]
+  float* stat_m = stats;
+  float* stat_z = stats + 256;
+  if ((smem_u32(smem) & 1023u) != 0) {                      // never run on a skewed layout (uniform over the CTA)
+    if (tid == 0 && a.status) atomicExch(a.status, (int)SLKV_ERR_BAD_ALIGN);
+    return;
+  }
   const uint32_t q_smem = smem_u32(smem);
   const uint32_t k_smem = q_smem + 2 * q_half_bytes;
   const uint32_t bar0 = smem_u32(bars);
@@ -238,8 +247,10 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // rows of the Q tile beyond R are never written by TMA: keep them zero
-  for (int i = tid; i < 2 * q_half_bytes / 16; i += kThreads) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (R != MT * 128) {
+    for (int i = tid; i < 2 * q_half_bytes / 16; i += kThreads) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -248,9 +259,11 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_sh;
-  // everything above touched only this CTA's own resources; global inputs are read from here on
+  // Everything above touched only this CTA's own resources.  Pass 1 reads its inputs after the kernels
+  // before it have finished.  In pass 2 the loads and the tensor-core work need only Q and K, which pass 1
+  // has already read, so they start at once; the epilogue alone waits for pass 1's row statistics.
   pdl_launch_dependents();
-  pdl_wait();
+  if (PASS == 1 || warp >= 4) pdl_wait();
   if (tid == 0) trace_mark(a.trace, 1);
 
   constexpr bool REV = PASS == 2;      // pass 2 walks the CTA's tiles backwards: the last ones read are likeliest in L2
@@ -259,10 +272,15 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   auto advance = [&](int pos, const Run& r) { return REV ? pos - r.count : pos + r.count; };
   auto tile_of = [&](const Run& r, int i) { return r.t0 + (REV ? r.count - 1 - i : i); };
 
+  // The two single-thread loops below are the pipeline's metronome: whatever they spend per tile between two
+  // issues is dead time for the tensor pipe (a tcgen05.mma issue blocks its thread while the pipe is busy),
+  // so ring positions and phase bits advance by increments (no divisions) and the operand descriptors are
+  // built once.
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      int it = 0, run_idx = 0;
+      int it = 0, run_idx = 0, st = 0;
+      uint32_t st_phase = 0;                                             // parity of the ring pass in progress
       bool ok = true;
       for (int pos = pos0; more(pos) && ok;) {
         const Run r = locate<REV>(a, pos, begin, end);
@@ -272,16 +290,17 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const int qy = a.q_head_inner ? r.g * a.G : 0, qz = a.q_head_inner ? 0 : r.g * a.G;
         tma_load_4d(q_smem, &tm_q, 0, qy, qz, r.s, qfull_bar);
         tma_load_4d(q_smem + q_half_bytes, &tm_q, 64, qy, qz, r.s, qfull_bar);
-        const int tok0 = a.tab.cu_at(r.s);
-        for (int i = 0; i < r.count; ++i, ++it) {
-          const int st = it % kStages;
-          ok = mbar_wait(empty_bar(st), ((it / kStages) & 1) ^ 1, abort_flag);
+        int tok = a.tab.cu_at(r.s) + tile_of(r, 0) * kTileKeys;
+        const int tok_step = REV ? -kTileKeys : kTileKeys;
+        for (int i = 0; i < r.count; ++i, ++it, tok += tok_step) {
+          ok = mbar_wait(empty_bar(st), st_phase ^ 1u, abort_flag);
           if (!ok) break;
-          mbar_expect_tx(full_bar(st), kStageBytes);
-          const int tok = tok0 + tile_of(r, i) * kTileKeys;
+          const uint32_t fb = full_bar(st), dst = k_smem + (uint32_t)st * kStageBytes;
+          mbar_expect_tx(fb, kStageBytes);
           const int ky = a.k_head_inner ? r.g : tok, kz = a.k_head_inner ? tok : r.g;
-          tma_load_3d(k_smem + st * kStageBytes, &tm_k, 0, ky, kz, full_bar(st));
-          tma_load_3d(k_smem + st * kStageBytes + kHalfBytes, &tm_k, 64, ky, kz, full_bar(st));
+          tma_load_3d(dst, &tm_k, 0, ky, kz, fb);
+          tma_load_3d(dst + kHalfBytes, &tm_k, 64, ky, kz, fb);
+          if (++st == kStages) { st = 0; st_phase ^= 1u; }
         }
         pos = advance(pos, r);
         ++run_idx;
@@ -289,10 +308,10 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       if (!ok) {
         // give loads already in flight a bounded chance to land before the CTA's shared memory goes away
         const unsigned long long t0 = now_ns();
-        for (int st = 0; st < kStages; ++st) {
-          const int last = it - 1 - ((it - 1 - st) % kStages + kStages) % kStages;   // last issue into stage st
+        for (int s2 = 0; s2 < kStages; ++s2) {
+          const int last = it - 1 - ((it - 1 - s2) % kStages + kStages) % kStages;   // last issue into stage s2
           if (it == 0 || last < 0) continue;
-          while (!mbar_try(full_bar(st), (last / kStages) & 1) && now_ns() - t0 < kWaitLimitNs) {}
+          while (!mbar_try(full_bar(s2), (last / kStages) & 1) && now_ns() - t0 < kWaitLimitNs) {}
         }
       }
     }
@@ -300,7 +319,14 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       const uint32_t idesc = PASS == 1 ? instr_desc(128, kTileKeys) : instr_desc(kTileKeys, R);
-      int it = 0, run_idx = 0;
+      // descriptor of the k-step ks of a tile = descriptor of the tile + (byte offset >> 4); the address field
+      // cannot carry out of its 14 bits because shared memory ends below 256 KB
+      const uint64_t q_desc0 = smem_desc(q_smem), k_desc0 = smem_desc(k_smem);
+      const uint64_t q_hi = (uint64_t)(q_half_bytes >> 4), k_hi = (uint64_t)(kHalfBytes >> 4);
+      int it = 0, run_idx = 0, st = 0, b = 0;
+      uint32_t st_phase = 0, b_phase = 0;
+      uint64_t k_desc = k_desc0;
+      uint32_t d0 = tmem_base;
       bool ok = true;
       for (int pos = pos0; more(pos) && ok;) {
         const Run r = locate<REV>(a, pos, begin, end);
@@ -308,32 +334,32 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         if (!ok) break;
         if (run_idx == 0) trace_mark(a.trace, 2);
         for (int i = 0; i < r.count; ++i, ++it) {
-          const int st = it % kStages, b = it % n_bufs;
-          ok = mbar_wait(full_bar(st), (it / kStages) & 1, abort_flag) &&
-               mbar_wait(acce_bar(b), ((it / n_bufs) & 1) ^ 1, abort_flag);
+          ok = mbar_wait(full_bar(st), st_phase, abort_flag) && mbar_wait(acce_bar(b), b_phase ^ 1u, abort_flag);
           if (!ok) break;
           if (it == 0) trace_mark(a.trace, 3);
           tc_fence_after();
-          const uint32_t kst = k_smem + st * kStageBytes;
-          const uint32_t d0 = tmem_base + (uint32_t)(b * buf_cols);
           if (PASS == 1) {
-            for (int mt = 0; mt < MT; ++mt)
+            for (int mt = 0; mt < MT; ++mt) {
+              const uint64_t qd = q_desc0 + (uint64_t)(mt * ((128 * 128) >> 4));
 #pragma unroll
               for (int ks = 0; ks < 8; ++ks) {
-                const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                const uint32_t qoff = (uint32_t)(ks >> 2) * q_half_bytes + (uint32_t)(ks & 3) * 32u + mt * (128 * 128);
-                tc_mma(d0 + mt * 128, smem_desc(q_smem + qoff), smem_desc(kst + koff), idesc, ks > 0);
+                const uint64_t off = (uint64_t)((ks & 3) * 2);
+                tc_mma(d0 + mt * 128, qd + (ks >> 2) * q_hi + off, k_desc + (ks >> 2) * k_hi + off, idesc, ks > 0);
               }
+            }
           } else {
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-              const uint32_t koff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-              const uint32_t qoff = (uint32_t)(ks >> 2) * q_half_bytes + (uint32_t)(ks & 3) * 32u;
-              tc_mma(d0, smem_desc(kst + koff), smem_desc(q_smem + qoff), idesc, ks > 0);
+              const uint64_t off = (uint64_t)((ks & 3) * 2);
+              tc_mma(d0, k_desc + (ks >> 2) * k_hi + off, q_desc0 + (ks >> 2) * q_hi + off, idesc, ks > 0);
             }
           }
           tc_commit(empty_bar(st));       // K stage free once these MMAs have read it
           tc_commit(accf_bar(b));         // accumulator ready for the epilogue
+          k_desc += (uint64_t)(kStageBytes >> 4);
+          if (++st == kStages) { st = 0; st_phase ^= 1u; k_desc = k_desc0; }
+          d0 += (uint32_t)buf_cols;
+          if (++b == n_bufs) { b = 0; b_phase ^= 1u; d0 = tmem_base; }
         }
         tc_commit(qempty_bar);            // Q tile free once the run's MMAs are done
         pos = advance(pos, r);
@@ -355,25 +381,38 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const int seg = r.s * a.n_kv_heads + r.g;
       const int first_cta = r.seg_tile0 / a.tiles_per_cta;
       float m_run[2] = {-INFINITY, -INFINITY}, z_run[2] = {0.f, 0.f};
-      float* lse = lse_sh[run_idx & 1];
+      float* lse = stats + 256 * (run_idx & 1);
       if (PASS == 2) {
         // merge the per-CTA partials of this segment into the rows' log-sum-exp (log2 units)
         const int n_slots = (r.seg_tile0 + r.tiles_seg - 1) / a.tiles_per_cta - first_cta + 1;
         if (et < R) {
-          const float* pm = a.part_m + ((long long)seg * R + et) * a.slot_stride;
-          const float* pz = a.part_z + ((long long)seg * R + et) * a.slot_stride;
-          float M = -INFINITY;
-          for (int c = 0; c < n_slots; ++c) M = fmaxf(M, pm[c]);
-          float Z = 0.f;
-          for (int c = 0; c < n_slots; ++c) Z += pz[c] * exp2f(pm[c] - M);
+          const float* pm = a.part_m + (long long)seg * a.slot_stride * R + et;      // [segment][slot][row]
+          const float* pz = a.part_z + (long long)seg * a.slot_stride * R + et;
+          float M = -INFINITY, Z = 0.f;
+          for (int c0 = 0; c0 < n_slots; c0 += 8) {                                   // sixteen loads in flight
+            float m8[8], z8[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const bool in = c0 + u < n_slots;
+              m8[u] = in ? __ldcg(pm + (long long)(c0 + u) * R) : -INFINITY;
+              z8[u] = in ? __ldcg(pz + (long long)(c0 + u) * R) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              if (m8[u] > -INFINITY) {
+                const float Mn = fmaxf(M, m8[u]);
+                Z = Z * ex2(M - Mn) + z8[u] * ex2(m8[u] - Mn);      // ex2(-inf) = 0 covers the first term
+                M = Mn;
+              }
+          }
           lse[et] = M + log2f(Z);
         }
         epi_bar();
       }
       for (int i = 0; i < r.count; ++i, ++it) {
         if ((it & 1) != wg) continue;
-        const int b = it % n_bufs;
-        if (ok) ok = mbar_wait(accf_bar(b), (it / n_bufs) & 1, abort_flag);
+        const int b = it & (n_bufs - 1);                // n_bufs is 4 or 2
+        if (ok) ok = mbar_wait(accf_bar(b), (it >> (n_bufs == 4 ? 2 : 1)) & 1, abort_flag);
         ok = __all_sync(0xffffffffu, ok) != 0;         // the TMEM loads below need the whole warp
         if (!ok) continue;
         tc_fence_after();
@@ -457,12 +496,19 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               acc += (s0 + s1) + (s2 + s3);
             }
           }
+          // The accumulator is in registers now: hand its TMEM buffer back before the vote leaves for global
+          // memory (the arrive has release semantics and would otherwise wait for that store).
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acce_bar(b));
           const int j = key0 + row;
           if (j < r.n_hist) a.vote[a.tab.hist_at(r.s) * a.n_kv_heads + (long long)r.g * r.n_hist + j] = acc * inv_g;
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(acce_bar(b));
+        if (PASS == 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acce_bar(b));
+        }
         if (row == 0 && it < 28) trace_mark(a.trace, 9 + 2 * it);
       }
       if (PASS == 1) {
@@ -478,8 +524,8 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               const float M = fmaxf(m_run[mt], m1);
               float Z = 0.f;
               if (M > -INFINITY) Z = z_run[mt] * ex2(m_run[mt] - M) + z1 * ex2(m1 - M);
-              a.part_m[((long long)seg * R + rr) * a.slot_stride + slot] = M;
-              a.part_z[((long long)seg * R + rr) * a.slot_stride + slot] = Z;
+              a.part_m[((long long)seg * a.slot_stride + slot) * R + rr] = M;
+              a.part_z[((long long)seg * a.slot_stride + slot) * R + rr] = Z;
             }
           }
           epi_bar();
@@ -625,15 +671,18 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
   a.tiles_per_cta = sc.tiles_per_cta; a.total_tiles = sc.total_tiles;
   a.scale_log2 = kLog2e / sqrtf((float)p.head_dim);
 
-  const size_t smem = 1024 + (size_t)a.MT * 2 * 128 * 128 + (size_t)kStages * kStageBytes;
+  const size_t q_bytes = (size_t)a.MT * 2 * 128 * 128;
+  a.n_stages = (int)((kSmemLimit - kTailBytes - q_bytes) / kStageBytes);
+  if (a.n_stages > kMaxStages) a.n_stages = kMaxStages;
+  const size_t smem = q_bytes + (size_t)a.n_stages * kStageBytes + kTailBytes;
   static thread_local int configured_dev = -1;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (configured_dev != dev) {
-    e = cudaFuncSetAttribute(k_score_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    e = cudaFuncSetAttribute(k_score_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_score_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    e = cudaFuncSetAttribute(k_score_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return e;
     configured_dev = dev;
   }

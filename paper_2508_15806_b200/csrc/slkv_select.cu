@@ -109,7 +109,7 @@ k_pool(const float* __restrict__ vote, float* __restrict__ pooled, const __grid_
 __global__ void __launch_bounds__(kScanThreads, 1)
 k_select(const float* __restrict__ pooled, const __grid_constant__ SeqTables tab,
          const int32_t* __restrict__ budgets, const int32_t* __restrict__ offsets, int32_t* __restrict__ kept_idx,
-         int n_kv_heads, int window, long long capacity) {
+         int32_t* __restrict__ gather_src, int n_kv_heads, int window, long long capacity) {
   __shared__ int hist[256];
   __shared__ int wt[32];
   __shared__ unsigned sh_prefix;
@@ -124,17 +124,24 @@ k_select(const float* __restrict__ pooled, const __grid_constant__ SeqTables tab
   const int n_win = min(len, window);
   const int k = kept_rows(len, budgets[h], window) - n_win;      // history rows to keep (C_H = C - window)
   const long long out0 = offsets[seg];
+  const int src_base = tab.cu_at(s) * n_kv_heads + h;           // source row of position j: src_base + j * n_kv_heads
   const unsigned* src = reinterpret_cast<const unsigned*>(pooled + tab.hist_at(s) * n_kv_heads + (long long)h * n_hist);
 
   // window rows (Algorithm 3 l.4, l.10): always kept, appended after the history rows
   for (int t = tid; t < n_win; t += kScanThreads) {
     long long o = out0 + k + t;
-    if (o < capacity) kept_idx[o] = len - n_win + t;
+    if (o < capacity) {
+      kept_idx[o] = len - n_win + t;
+      gather_src[o] = src_base + (len - n_win + t) * n_kv_heads;
+    }
   }
   if (k <= 0) return;
   if (k >= n_hist) {                                             // nothing to drop
     for (int j = tid; j < n_hist; j += kScanThreads)
-      if (out0 + j < capacity) kept_idx[out0 + j] = j;
+      if (out0 + j < capacity) {
+        kept_idx[out0 + j] = j;
+        gather_src[out0 + j] = src_base + j * n_kv_heads;
+      }
     return;
   }
 
@@ -176,35 +183,35 @@ k_select(const float* __restrict__ pooled, const __grid_constant__ SeqTables tab
     const int gt_before = gt_seen + (ex & 0xffff), eq_before = eq_seen + (ex >> 16);
     if (gt || (eq && eq_before < need)) {
       long long o = out0 + gt_before + min(eq_before, need);
-      if (o < capacity) kept_idx[o] = j;
+      if (o < capacity) {
+        kept_idx[o] = j;
+        gather_src[o] = src_base + j * n_kv_heads;
+      }
     }
     gt_seen += tot & 0xffff;
     eq_seen += tot >> 16;
   }
 }
 
-// Copies the kept rows of K and V into the packed cache: 16 bytes per lane, a row per lane group.
+// Copies the kept rows of K and V into the packed cache: 16 bytes per lane, a row per lane group.  The
+// selection kernel left the source row (token * n_kv_heads + head) of every packed row in gather_src, so a
+// row costs two dependent memory round trips (source index, then the row itself).
 __global__ void __launch_bounds__(256)
 k_gather(const unsigned char* __restrict__ k, const unsigned char* __restrict__ v, unsigned char* __restrict__ k_out,
-         unsigned char* __restrict__ v_out, const __grid_constant__ SeqTables tab,
-         const int32_t* __restrict__ offsets, const int32_t* __restrict__ kept_idx, int n_seg, int n_kv_heads,
-         int row_bytes, long long k_tok_bytes, long long k_head_bytes, long long v_tok_bytes,
-         long long v_head_bytes, long long capacity) {
+         unsigned char* __restrict__ v_out, const int32_t* __restrict__ offsets,
+         const int32_t* __restrict__ gather_src, int n_seg, int n_kv_heads, int row_bytes, long long k_tok_bytes,
+         long long k_head_bytes, long long v_tok_bytes, long long v_head_bytes, long long max_rows) {
   pdl_launch_dependents();
-  pdl_wait();
   const int lanes = row_bytes >> 4;                       // 16-byte lanes per row (power of two <= 32)
   const int rows_per_cta = blockDim.x / lanes;
   const int lane = threadIdx.x % lanes, sub = threadIdx.x / lanes;
-  const long long n_rows = min((long long)offsets[n_seg], capacity);
-  for (long long r = (long long)blockIdx.x * rows_per_cta + sub; r < n_rows;
+  pdl_wait();
+  const long long n_rows = min((long long)offsets[n_seg], max_rows);
+  for (long long r = (long long)blockIdx.x * rows_per_cta + sub; r < max_rows;
        r += (long long)gridDim.x * rows_per_cta) {
-    int lo = 0, hi = n_seg;                               // last seg with offsets[seg] <= r
-    while (hi - lo > 1) {
-      int mid = (lo + hi) >> 1;
-      if ((long long)offsets[mid] <= r) lo = mid; else hi = mid;
-    }
-    const int s = lo / n_kv_heads, h = lo - s * n_kv_heads;
-    const long long tok = (long long)tab.cu_at(s) + kept_idx[r];
+    const int src = gather_src[r];                        // in bounds for r < max_rows; valid for r < n_rows
+    if (r >= n_rows) break;
+    const int tok = src / n_kv_heads, h = src - tok * n_kv_heads;
     const uint4 kv = *reinterpret_cast<const uint4*>(k + tok * k_tok_bytes + h * k_head_bytes + lane * 16);
     const uint4 vv = *reinterpret_cast<const uint4*>(v + tok * v_tok_bytes + h * v_head_bytes + lane * 16);
     *reinterpret_cast<uint4*>(k_out + r * row_bytes + lane * 16) = kv;
@@ -233,24 +240,25 @@ cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t*
                           int32_t* kept_idx, int64_t capacity, cudaStream_t st, int* launches) {
   LaunchScope scope(KID_SELECT, st, launches);
   return launch_pdl(k_select, dim3(pb.n_seg), dim3(kScanThreads), 0, st, 1, pooled, pb.tab, budgets, offsets,
-                    kept_idx, pb.p.n_kv_heads, pb.p.window, (long long)capacity);
+                    kept_idx, pb.gather_src, pb.p.n_kv_heads, pb.p.window, (long long)capacity);
 }
 
 cudaError_t launch_gather(const Problem& pb, const int32_t* offsets, const int32_t* kept_idx, void* k_out,
                           void* v_out, int64_t capacity, cudaStream_t st, int* launches) {
+  (void)kept_idx;
   const int row_bytes = pb.p.head_dim * pb.elem;
   const int rows_per_cta = 256 / (row_bytes >> 4);
   long long max_rows = (long long)pb.p.n_kv_heads * pb.total_tokens;
   if (capacity < max_rows) max_rows = capacity;
   if (max_rows <= 0) return cudaSuccess;
   long long want = (max_rows + rows_per_cta - 1) / rows_per_cta;
-  int grid = (int)(want < 148 * 16 ? want : 148 * 16);
+  int grid = (int)(want < 148 * 8 ? want : 148 * 8);
   LaunchScope scope(KID_GATHER, st, launches);
   return launch_pdl(k_gather, dim3(grid), dim3(256), 0, st, 1, (const unsigned char*)pb.k,
-                    (const unsigned char*)pb.v, (unsigned char*)k_out, (unsigned char*)v_out, pb.tab, offsets, kept_idx,
-                    pb.n_seg, pb.p.n_kv_heads, row_bytes, (long long)(pb.p.k_stride_tok * pb.elem),
-                    (long long)(pb.p.k_stride_head * pb.elem), (long long)(pb.p.v_stride_tok * pb.elem),
-                    (long long)(pb.p.v_stride_head * pb.elem), (long long)capacity);
+                    (const unsigned char*)pb.v, (unsigned char*)k_out, (unsigned char*)v_out, offsets,
+                    (const int32_t*)pb.gather_src, pb.n_seg, pb.p.n_kv_heads, row_bytes,
+                    (long long)(pb.p.k_stride_tok * pb.elem), (long long)(pb.p.k_stride_head * pb.elem),
+                    (long long)(pb.p.v_stride_tok * pb.elem), (long long)(pb.p.v_stride_head * pb.elem), max_rows);
 }
 
 }  // namespace slkv
