@@ -7,8 +7,8 @@
 //           registers; per CTA and segment one (max, sum) pair per row goes to global memory.
 //   pass 2 (votes)           S^T = K Q^T per tile with the keys as the M dimension, so that a thread owns
 //           a key: vote[j] = (1/G) sum_rows 2^(s_rj - lse_r) is a thread-local sum and a coalesced store.
-// Warp roles: warp 0 issues TMA loads (128-byte-swizzled K-major tiles, no multicast), warp 1 issues
-// tcgen05.mma into TMEM accumulators and commits to mbarriers, warps 4..11 (two warpgroups, alternating
+// Warp roles: warp 0 issues TMA loads (128-byte-swizzled K-major tiles, no multicast), warps 1 and 2 issue
+// tcgen05.mma (alternate tiles) into TMEM accumulators and commit to mbarriers, warps 4..11 (two warpgroups, alternating
 // tiles) read TMEM with tcgen05.ld and do the softmax arithmetic in fp32.
 // Every mbarrier wait is bounded by a wall-clock limit; when one runs out the CTA raises
 // SLKV_ERR_DEVICE_TIMEOUT in the status word, stops waiting everywhere, releases TMEM and returns.
@@ -114,6 +114,23 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// 2^x on the FMA and integer pipes instead of the special-function unit, which is the busiest pipe of both
+// passes (one exponential per query row and key): x = n + f with n = round(x), 2^f by a degree-4 minimax
+// polynomial on [-0.5, 0.5] (relative error 2.7e-6 in fp32 Horner form), n added into the exponent field.
+// x is clamped to [-125, 128.5]: below, the result is 2^-125 at most (negligible in any sum that holds a term
+// near 1); above, the exponent field overflows to Inf/NaN, which the caller's overflow check catches.
+// One exponential in four goes this way; the split balances the pipes' issue slots.
+__device__ __forceinline__ float ex2_fma(float x, bool clamp_hi) {
+  x = fmaxf(x, -125.f);
+  if (clamp_hi) x = fminf(x, 128.5f);
+  const float t = x + 12582912.f;                    // 1.5 * 2^23: round(x) lands in the low mantissa bits
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(0.009570101276040077f, f, 0.05591785907745361f);
+  p = fmaf(p, f, 0.240247443318367f);
+  p = fmaf(p, f, 0.6931217908859253f);
+  p = fmaf(p, f, 0.9999992847442627f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
 // Issues a TMEM load of 32 consecutive columns of this thread's lane; the registers are valid only after
 // tc_ld_wait on the same array.
 __device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
@@ -184,7 +201,7 @@ __device__ __forceinline__ float sum_ex2_32(const uint32_t (&r)[32], float sc, f
     s0 += ex2(fmaf(__uint_as_float(r[e]), sc, -m));
     s1 += ex2(fmaf(__uint_as_float(r[e + 1]), sc, -m));
     s2 += ex2(fmaf(__uint_as_float(r[e + 2]), sc, -m));
-    s3 += ex2(fmaf(__uint_as_float(r[e + 3]), sc, -m));
+    s3 += ex2_fma(fmaf(__uint_as_float(r[e + 3]), sc, -m), true);
   }
   return (s0 + s1) + (s2 + s3);
 }
@@ -243,7 +260,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     for (int st = 0; st < kStages; ++st) { mbar_init(full_bar(st), 1); mbar_init(empty_bar(st), 1); }
     for (int b = 0; b < 4; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
     mbar_init(qfull_bar, 1);
-    mbar_init(qempty_bar, 1);
+    mbar_init(qempty_bar, 2);                                 // one arrival per MMA issuer
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // rows of the Q tile beyond R are never written by TMA: keep them zero
@@ -315,9 +332,13 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
+  } else if (warp == 1 || warp == 2) {
+    // ---------------- MMA issuers ----------------
+    // Two threads take alternate tiles.  Issuing a tile's MMAs blocks the thread for about as long as the
+    // tensor pipe needs them; with one issuer the waits and bookkeeping between two tiles would leave the pipe
+    // idle, with two the other thread is already past its waits and its MMAs queue up right behind.
     if (lane == 0) {
+      const int me = warp - 1;
       const uint32_t idesc = PASS == 1 ? instr_desc(128, kTileKeys) : instr_desc(kTileKeys, R);
       // descriptor of the k-step ks of a tile = descriptor of the tile + (byte offset >> 4); the address field
       // cannot carry out of its 14 bits because shared memory ends below 256 KB
@@ -332,8 +353,9 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const Run r = locate<REV>(a, pos, begin, end);
         ok = mbar_wait(qfull_bar, run_idx & 1, abort_flag);
         if (!ok) break;
-        if (run_idx == 0) trace_mark(a.trace, 2);
+        if (run_idx == 0 && me == 0) trace_mark(a.trace, 2);
         for (int i = 0; i < r.count; ++i, ++it) {
+         if ((it & 1) == me) {
           ok = mbar_wait(full_bar(st), st_phase, abort_flag) && mbar_wait(acce_bar(b), b_phase ^ 1u, abort_flag);
           if (!ok) break;
           if (it == 0) trace_mark(a.trace, 3);
@@ -356,12 +378,13 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
           tc_commit(empty_bar(st));       // K stage free once these MMAs have read it
           tc_commit(accf_bar(b));         // accumulator ready for the epilogue
+         }
           k_desc += (uint64_t)(kStageBytes >> 4);
           if (++st == kStages) { st = 0; st_phase ^= 1u; k_desc = k_desc0; }
           d0 += (uint32_t)buf_cols;
           if (++b == n_bufs) { b = 0; b_phase ^= 1u; d0 = tmem_base; }
         }
-        tc_commit(qempty_bar);            // Q tile free once the run's MMAs are done
+        tc_commit(qempty_bar);            // Q tile free once the run's MMAs (of both issuers) are done
         pos = advance(pos, r);
         ++run_idx;
       }
@@ -425,13 +448,15 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           for (int mt = 0; mt < MT; ++mt) {
             const uint32_t tcol = tb + mt * 128;
             float m = m_run[mt], z = z_run[mt];
-            bool exact = !(m > -INFINITY) || n_valid < kTileKeys;
+            bool exact = n_valid < kTileKeys;
             if (!exact) {
-              // Optimistic: keep the reference maximum m of earlier tiles (any m gives the same log-sum-exp
-              // as long as nothing overflows); an overflow shows as a non-finite sum and is redone exactly.
+              // Optimistic: keep the reference maximum m of earlier tiles -- on a run's first tile, the maximum
+              // of its first 32 keys (any m gives the same log-sum-exp as long as nothing overflows or all
+              // underflows); a non-finite or zero sum shows that and the tile is redone exactly.
               float zt = z;
               tc_ld32_issue(tcol, ra);
               tc_ld_wait(ra);
+              if (!(m > -INFINITY)) m = max_32(ra, 32) * sc;
               tc_ld32_issue(tcol + 32, rb);
               zt += sum_ex2_32(ra, sc, m);
               tc_ld_wait(rb);
@@ -442,7 +467,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               zt += sum_ex2_32(ra, sc, m);
               tc_ld_wait(rb);
               zt += sum_ex2_32(rb, sc, m);
-              if (zt < INFINITY) z = zt; else exact = true;
+              if (zt < INFINITY && zt > 0.f) z = zt; else { exact = true; m = m_run[mt]; }
             }
             if (exact) {
 #pragma unroll 1
@@ -477,7 +502,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 s0 += ex2(fmaf(__uint_as_float(ra[e]), sc, -l4.x));
                 s1 += ex2(fmaf(__uint_as_float(ra[e + 1]), sc, -l4.y));
                 s2 += ex2(fmaf(__uint_as_float(ra[e + 2]), sc, -l4.z));
-                s3 += ex2(fmaf(__uint_as_float(ra[e + 3]), sc, -l4.w));
+                s3 += ex2_fma(fmaf(__uint_as_float(ra[e + 3]), sc, -l4.w), false);
               }
               acc += (s0 + s1) + (s2 + s3);
             }
@@ -491,7 +516,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 s0 += ex2(fmaf(__uint_as_float(rb[e]), sc, -l4.x));
                 s1 += ex2(fmaf(__uint_as_float(rb[e + 1]), sc, -l4.y));
                 s2 += ex2(fmaf(__uint_as_float(rb[e + 2]), sc, -l4.z));
-                s3 += ex2(fmaf(__uint_as_float(rb[e + 3]), sc, -l4.w));
+                s3 += ex2_fma(fmaf(__uint_as_float(rb[e + 3]), sc, -l4.w), false);
               }
               acc += (s0 + s1) + (s2 + s3);
             }
