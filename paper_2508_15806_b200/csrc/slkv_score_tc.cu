@@ -216,6 +216,31 @@ __device__ __forceinline__ float max_32(const uint32_t (&r)[32], int n_valid_her
   return t[0];
 }
 
+// Pass 1, exact path for one 128-row accumulator: running maximum and rescaled sum over the tile's first n_valid
+// keys.  Used for a segment's ragged last tile and when the fast path over- or underflows.  A function of its
+// own (not inlined) so that a CTA which will need it can run it once before the K stream starts: fetching
+// these instructions for the first time while the stream saturates the memory system stalled the tile for
+// microseconds.
+__device__ __noinline__ void tile_row_stats_exact(uint32_t tcol, float sc, int n_valid, float& m_io, float& z_io) {
+  uint32_t ra[32];
+  float m = m_io, z = z_io;
+#pragma unroll 1
+  for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
+    if (c0 >= n_valid) break;
+    tc_ld32_issue(tcol + c0, ra);
+    tc_ld_wait(ra);
+    const float mn = fmaxf(m, max_32(ra, n_valid - c0) * sc);
+    z *= ex2(m - mn);
+    m = mn;
+    float zc = 0.f;
+#pragma unroll
+    for (int e = 0; e < 32; ++e)
+      if (e < n_valid - c0) zc += ex2(fmaf(__uint_as_float(ra[e]), sc, -m));
+    z += zc;
+  }
+  m_io = m; z_io = z;
+}
+
 template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
 k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -280,6 +305,19 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   // before it have finished.  In pass 2 the loads and the tensor-core work need only Q and K, which pass 1
   // has already read, so they start at once; the epilogue alone waits for pass 1's row statistics.
   pdl_launch_dependents();
+  if (PASS == 1 && warp >= 4) {
+    bool ragged = false;                                            // a segment's ragged last tile in this CTA's range?
+    for (int pos = begin; pos < end;) {
+      const Run r = locate<false>(a, pos, begin, end);
+      ragged |= r.t0 + r.count == r.tiles_seg && (r.n_hist & (kTileKeys - 1)) != 0;
+      pos += r.count;
+    }
+    if (ragged) {                                                   // instruction-cache warm-up, results unused
+      float mw = 0.f, zw = 0.f;
+      tile_row_stats_exact(tmem_base + ((uint32_t)((warp & 3) * 32) << 16), 0.f, kTileKeys - 1, mw, zw);
+      if (zw == 12345.f) abort_sh = 0;                              // keeps the call alive; writes what is there
+    }
+  }
   if (PASS == 1 || warp >= 4) pdl_wait();
   if (tid == 0) trace_mark(a.trace, 1);
 
@@ -403,7 +441,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const Run r = locate<REV>(a, pos, begin, end);
       const int seg = r.s * a.n_kv_heads + r.g;
       const int first_cta = r.seg_tile0 / a.tiles_per_cta;
-      float m_run[2] = {-INFINITY, -INFINITY}, z_run[2] = {0.f, 0.f};
+      float m_run[2] = {0.f, 0.f}, z_run[2] = {0.f, 0.f};      // reference 0: see the fast path below
       float* lse = stats + 256 * (run_idx & 1);
       if (PASS == 2) {
         // merge the per-CTA partials of this segment into the rows' log-sum-exp (log2 units)
@@ -450,13 +488,12 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             float m = m_run[mt], z = z_run[mt];
             bool exact = n_valid < kTileKeys;
             if (!exact) {
-              // Optimistic: keep the reference maximum m of earlier tiles -- on a run's first tile, the maximum
-              // of its first 32 keys (any m gives the same log-sum-exp as long as nothing overflows or all
-              // underflows); a non-finite or zero sum shows that and the tile is redone exactly.
+              // Fast path: a fixed reference m (0 until a fallback moves it) instead of a running maximum -- any
+              // reference gives the same log-sum-exp as long as nothing overflows and not everything underflows;
+              // a non-finite or zero sum shows that, and the tile is then redone exactly.
               float zt = z;
               tc_ld32_issue(tcol, ra);
               tc_ld_wait(ra);
-              if (!(m > -INFINITY)) m = max_32(ra, 32) * sc;
               tc_ld32_issue(tcol + 32, rb);
               zt += sum_ex2_32(ra, sc, m);
               tc_ld_wait(rb);
@@ -467,24 +504,9 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               zt += sum_ex2_32(ra, sc, m);
               tc_ld_wait(rb);
               zt += sum_ex2_32(rb, sc, m);
-              if (zt < INFINITY && zt > 0.f) z = zt; else { exact = true; m = m_run[mt]; }
+              if (zt < INFINITY && zt > 0.f) z = zt; else exact = true;
             }
-            if (exact) {
-#pragma unroll 1
-              for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
-                if (c0 >= n_valid) break;
-                tc_ld32_issue(tcol + c0, ra);
-                tc_ld_wait(ra);
-                const float mn = fmaxf(m, max_32(ra, n_valid - c0) * sc);
-                z *= ex2(m - mn);
-                m = mn;
-                float zc = 0.f;
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                  if (e < n_valid - c0) zc += ex2(fmaf(__uint_as_float(ra[e]), sc, -m));
-                z += zc;
-              }
-            }
+            if (exact) tile_row_stats_exact(tcol, sc, n_valid, m, z);
             m_run[mt] = m; z_run[mt] = z;
           }
         } else {
