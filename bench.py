@@ -175,7 +175,8 @@ def run_cuda(args):
                        "v_out": torch.empty(rows, d, dtype=wl.torch_dtype, device=dev),
                        "offsets": torch.empty(len(wl.seq_lens) * hkv + 1, dtype=torch.int32, device=dev),
                        "kept": torch.empty(rows, dtype=torch.int32, device=dev)})
-    ws = B.new_workspace(params, cu, dev)
+    overlap = not args.no_overlap
+    ws = torch.empty(B.slkv_workspace_bytes_overlapped(params, cu), dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
 
@@ -184,10 +185,14 @@ def run_cuda(args):
     def step():
         nonlocal launches_per_step
         n = 0
+        # the layers of a step are independent: their calls may overlap on the GPU (selection and gather of one
+        # layer beside the score kernels of the next); the join orders the stream after all of them
+        call = B.slkv_compress_overlapped if overlap else B.slkv_compress
         for L in layers:
-            B.slkv_compress(params, L["q"], L["k"], L["v"], cu_dev, cu, L["bud"], L["k_out"], L["v_out"],
-                            L["offsets"], L["kept"], ws, None, status, stream)
+            call(params, L["q"], L["k"], L["v"], cu_dev, cu, L["bud"], L["k_out"], L["v_out"],
+                 L["offsets"], L["kept"], ws, None, status, stream)
             n += B.slkv_last_launch_count()
+        B.slkv_join(stream)
         launches_per_step = n
 
     def barrier():
@@ -328,6 +333,7 @@ def run_cuda(args):
                           "head_dim": d, "seq_lens": wl.seq_lens, "window": w, "pool_kernel": wl.pool_kernel,
                           "avg_budget_per_kv_head": total // (nl * hkv), "fixed": wl.fixed, "parallelism":
                           f"dp{world} (one sequence batch per GPU, no collective)",
+                          "api": "slkv_compress_overlapped + slkv_join per step" if overlap else "slkv_compress",
                           "l2": "inputs larger than L2: every layer has its own Q/K/V (%.1f GB per step)" %
                                 (nl * (2 * T * hkv * d * e) / 1e9)},
                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * steps,
@@ -419,6 +425,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="use fewer layers (profiling captures only)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="one layer at a time (slkv_compress) instead of overlapped calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--e2e-layers", type=int, default=8, help="distinct layers kept in pinned host memory")

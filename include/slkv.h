@@ -6,6 +6,7 @@
  *   slkv_score           relevance of every history key to the query window     (Sec. 3.4, Eq. 7, Alg. 3 l.4-6)
  *   slkv_compress        score -> top-(C - window) history rows + window, gather (Sec. 3.4, Eq. 8, Algorithm 3)
  *   slkv_compress_host   the same, from/to host buffers (copies included)
+ *   slkv_compress_overlapped / slkv_join   the same, successive layers overlapped on the GPU
  *
  * Conventions
  *   - "dev" pointers are device memory of the current CUDA device, "host" pointers are host memory.
@@ -150,6 +151,34 @@ int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const 
                   const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
                   void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx,
                   float* pooled_opt, int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * slkv_compress with the calls of successive layers overlapped on the GPU (Algorithm 3, same results).
+ *
+ * The selection and the gather of a layer are latency-bound and need few SMs; the score kernels of the next
+ * layer are bandwidth-bound and do not depend on them.  This entry point enqueues the score kernels on
+ * `stream` and the selection + gather on a stream of the library's own, ordered after them by an event, so
+ * that the next call's score kernels (which leave a few SMs free) run beside them.  Consequences:
+ *   - The outputs of a call (k_out, v_out, offsets, kept_idx, pooled_opt, status) are NOT ordered on `stream`
+ *     when the call returns.  slkv_join(stream) makes `stream` wait for every overlapped call enqueued so far
+ *     on the current device (no host wait); consume outputs, or free / overwrite any input, output or
+ *     workspace buffer, only behind it.  Any other slkv_* call that uses a workspace joins by itself first.
+ *   - workspace must hold slkv_workspace_bytes_overlapped (two vote arrays: successive calls alternate).
+ *     Successive calls may share one workspace; q_win, k, v, budgets and the outputs of calls that may be in
+ *     flight together must not alias each other's outputs.
+ *   - The first call on a device creates the side stream and four events (no device memory).
+ *   - Shapes the overlapped path does not take (more than 64 sequences, a segment with more than 32768
+ *     history positions, pool_kernel > 9) run as slkv_compress does, on `stream`, after a join.
+ * Arguments, results and error codes otherwise as slkv_compress.
+ */
+int slkv_compress_overlapped(const slkv_params* p, const void* q_win, const void* k, const void* v,
+                             const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
+                             void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets,
+                             int32_t* kept_idx, float* pooled_opt, int32_t* status, void* workspace,
+                             size_t workspace_bytes, void* stream);
+size_t slkv_workspace_bytes_overlapped(const slkv_params* p, const int32_t* cu_seqlens_host);
+/* Orders `stream` after every overlapped call enqueued so far on the current device (see above). */
+int slkv_join(void* stream);
 
 /* Bytes of device arena slkv_compress_host needs (inputs, outputs and workspace; 0 on invalid arguments). */
 size_t slkv_compress_host_arena_bytes(const slkv_params* p, const int32_t* cu_seqlens_host,

@@ -69,6 +69,12 @@ def lib() -> C.CDLL:
         L.slkv_score.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, sz, vp]
         L.slkv_compress.restype = C.c_int
         L.slkv_compress.argtypes = [pp, vp, vp, vp, vp, i32p, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+        L.slkv_compress_overlapped.restype = C.c_int
+        L.slkv_compress_overlapped.argtypes = L.slkv_compress.argtypes
+        L.slkv_workspace_bytes_overlapped.restype = sz
+        L.slkv_workspace_bytes_overlapped.argtypes = [pp, i32p]
+        L.slkv_join.restype = C.c_int
+        L.slkv_join.argtypes = [vp]
         L.slkv_compress_host_arena_bytes.restype = sz
         L.slkv_compress_host_arena_bytes.argtypes = [pp, i32p, i64]
         L.slkv_compress_host.restype = C.c_int
@@ -196,6 +202,29 @@ def slkv_compress(params: SlkvParams, q_win, k, v, cu_dev, cu_seqlens: Sequence[
                              workspace.data_ptr(), workspace.numel(), _stream(stream))
     if rc != SLKV_OK:
         raise SlkvError(rc, "slkv_compress")
+
+
+def slkv_compress_overlapped(params: SlkvParams, q_win, k, v, cu_dev, cu_seqlens: Sequence[int], budgets, k_out,
+                             v_out, offsets, kept_idx, workspace, pooled: Optional[torch.Tensor] = None,
+                             status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """slkv_compress with successive calls overlapped on the GPU; outputs are valid behind slkv_join()."""
+    rc = lib().slkv_compress_overlapped(C.byref(params), q_win.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                        cu_dev.data_ptr(), _cu_host(cu_seqlens), budgets.data_ptr(),
+                                        k_out.data_ptr(), v_out.data_ptr(), k_out.shape[0], offsets.data_ptr(),
+                                        kept_idx.data_ptr(), _ptr(pooled), _ptr(status), workspace.data_ptr(),
+                                        workspace.numel(), _stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_compress_overlapped")
+
+
+def slkv_workspace_bytes_overlapped(params: SlkvParams, cu_seqlens: Sequence[int]) -> int:
+    return int(lib().slkv_workspace_bytes_overlapped(C.byref(params), _cu_host(cu_seqlens)))
+
+
+def slkv_join(stream=None) -> None:
+    rc = lib().slkv_join(_stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_join")
 
 
 def slkv_compress_host_arena_bytes(params: SlkvParams, cu_seqlens: Sequence[int], capacity_rows: int) -> int:

@@ -1,6 +1,7 @@
 // extern "C" entry points of libslkv: argument validation, workspace carve-up, launch sequencing.
 // No step of the method runs here; every step is a kernel in the other translation units.
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "slkv_internal.cuh"
@@ -41,7 +42,7 @@ int cuda_fail(cudaError_t e) {
 }
 
 struct Layout {
-  size_t hist_off, tile_off, vote, pooled, part_m, part_z, flags, gather_src, total;
+  size_t hist_off, tile_off, vote, vote2, pooled, part_m, part_z, flags, gather_src, total;
 };
 
 // Validates p and cu_seqlens_host and fills the host-known fields of `pb`.
@@ -109,13 +110,15 @@ int describe(const slkv_params* p, const int32_t* cu_host, Problem* pb) {
   return SLKV_OK;
 }
 
-Layout layout_of(const Problem& pb) {
+Layout layout_of(const Problem& pb, bool overlapped = false) {
   Layout L;
   size_t o = 0;
   L.hist_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int64_t));
   L.tile_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int32_t));
   const size_t votes = (size_t)pb.p.n_kv_heads * (size_t)pb.total_hist * sizeof(float);
   L.vote = o; o = align_up(o + votes);
+  L.vote2 = L.vote;                                  // overlapped calls alternate between two vote arrays
+  if (overlapped) { L.vote2 = o; o = align_up(o + votes); }
   L.pooled = o; o = align_up(o + votes);
   const size_t nchunks = (size_t)(pb.max_hist + kMinChunkKeys - 1) / kMinChunkKeys + 2;
   const size_t parts = (size_t)pb.n_seg * pb.R * nchunks * sizeof(float);
@@ -138,17 +141,17 @@ int resolve_path(const Problem& pb, int* path) {
   return SLKV_OK;
 }
 
-int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path) {
+int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overlapped = false, int half = 0) {
   if (!ws) return SLKV_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) % kAlign != 0) return SLKV_ERR_BAD_ALIGN;
-  Layout L = layout_of(*pb);
+  Layout L = layout_of(*pb, overlapped);
   if (ws_bytes < L.total) return SLKV_ERR_WORKSPACE;
   unsigned char* b = static_cast<unsigned char*>(ws);
   pb->hist_off = reinterpret_cast<int64_t*>(b + L.hist_off);
   pb->tile_off = reinterpret_cast<int32_t*>(b + L.tile_off);
   pb->tab.tile_ptr = pb->tile_off;
   pb->tab.hist_ptr = reinterpret_cast<const long long*>(pb->hist_off);
-  pb->vote = reinterpret_cast<float*>(b + L.vote);
+  pb->vote = reinterpret_cast<float*>(b + (half ? L.vote2 : L.vote));
   pb->pooled_ws = reinterpret_cast<float*>(b + L.pooled);
   pb->part_m = reinterpret_cast<float*>(b + L.part_m);
   pb->part_z = reinterpret_cast<float*>(b + L.part_z);
@@ -172,10 +175,61 @@ int enqueue_votes(const Problem& pb, int path, const int32_t* cu_host, int32_t* 
   return SLKV_OK;
 }
 
+// ---- overlapped calls: selection and gather of one call run on a side stream while the next call's score
+// kernels run on the caller's stream --------------------------------------------------------------------
+struct OverlapState {
+  cudaStream_t side = nullptr;
+  cudaEvent_t scored[2] = {nullptr, nullptr};     // recorded on the caller's stream after the vote pass
+  cudaEvent_t done[2] = {nullptr, nullptr};       // recorded on the side stream after the gather
+  bool in_flight[2] = {false, false};
+  unsigned seq = 0;
+};
+constexpr int kMaxDevices = 64;
+OverlapState g_overlap[kMaxDevices];
+std::mutex g_overlap_mu;
+constexpr int kSelectSmReserve = 16;              // SMs left to the selection kernel of the previous call
+
+cudaError_t overlap_state(OverlapState** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  OverlapState& s = g_overlap[dev];
+  if (!s.side) {
+    e = cudaStreamCreateWithFlags(&s.side, cudaStreamNonBlocking);
+    if (e != cudaSuccess) return e;
+    for (int h = 0; h < 2; ++h) {
+      e = cudaEventCreateWithFlags(&s.scored[h], cudaEventDisableTiming);
+      if (e != cudaSuccess) return e;
+      e = cudaEventCreateWithFlags(&s.done[h], cudaEventDisableTiming);
+      if (e != cudaSuccess) return e;
+    }
+  }
+  *out = &s;
+  return cudaSuccess;
+}
+
+// Makes `st` wait for every overlapped call still in flight on this device (no host wait).
+cudaError_t join_overlapped(cudaStream_t st) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaSuccess;
+  std::lock_guard<std::mutex> lock(g_overlap_mu);
+  OverlapState& s = g_overlap[dev];
+  for (int h = 0; h < 2; ++h)
+    if (s.in_flight[h]) {
+      e = cudaStreamWaitEvent(st, s.done[h], 0);
+      if (e != cudaSuccess) return e;
+      s.in_flight[h] = false;
+    }
+  return cudaSuccess;
+}
+
 int compress_impl(const slkv_params* p, const void* q_win, const void* k, const void* v, const int32_t* cu_dev,
                   const int32_t* cu_host, const int32_t* budgets, void* k_out, void* v_out, int64_t capacity,
                   int32_t* offsets, int32_t* kept_idx, float* pooled_opt, int32_t* status, void* ws,
-                  size_t ws_bytes, cudaStream_t st) {
+                  size_t ws_bytes, cudaStream_t st, bool overlapped = false) {
   g_last_launches = 0;
   if (!q_win || !k || !v || !cu_dev || !budgets || !k_out || !v_out || !offsets || !kept_idx)
     return SLKV_ERR_NULL_PTR;
@@ -188,13 +242,60 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
   int path = 0;
   rc = resolve_path(pb, &path);
   if (rc != SLKV_OK) return rc;
+  // pooling, offsets and selection run in one kernel when the segments fit it: one CTA per segment up to
+  // 32768 history positions (overlapped calls), a thread-block cluster per segment otherwise
+  const bool one_cta = overlapped && select_cta_supported(pb) && pb.tab.n_inline > 0;
+  if (!one_cta) {
+    // ordinary call (or shapes the overlapped path does not take): everything on the caller's stream, after
+    // whatever overlapped calls are still in flight
+    cudaError_t je = join_overlapped(st);
+    if (je != cudaSuccess) return cuda_fail(je);
+    overlapped = false;
+  }
+  cudaError_t e = cudaSuccess;
+  int launches = 0;
+  if (overlapped) {
+    std::lock_guard<std::mutex> lock(g_overlap_mu);
+    OverlapState* os = nullptr;
+    e = overlap_state(&os);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const int half = (int)(os->seq & 1u);
+    rc = bind_workspace(&pb, ws, ws_bytes, path, true, half);
+    if (rc != SLKV_OK) return rc;
+    ++os->seq;
+    pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
+    pb.tab.cu_ptr = cu_dev;
+    // the score kernels leave a few SMs to the selection kernel of the call before this one
+    int sms = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int reserve = pb.n_seg < kSelectSmReserve ? pb.n_seg : kSelectSmReserve;
+    pb.max_score_ctas = sms - reserve > 0 ? sms - reserve : 0;
+    if (os->in_flight[half]) {                     // the vote array of this half is read by a selection two calls back
+      e = cudaStreamWaitEvent(st, os->done[half], 0);
+      if (e != cudaSuccess) return cuda_fail(e);
+      os->in_flight[half] = false;
+    }
+    rc = enqueue_votes(pb, path, cu_host, status, st, &launches);
+    if (rc != SLKV_OK) return rc;
+    e = cudaEventRecord(os->scored[half], st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side, os->scored[half], 0);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_select_cta(pb, pooled_opt, budgets, offsets, kept_idx, capacity, status, os->side, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_gather(pb, offsets, kept_idx, k_out, v_out, capacity, os->side, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaEventRecord(os->done[half], os->side);
+    if (e != cudaSuccess) return cuda_fail(e);
+    os->in_flight[half] = true;
+    g_last_launches = launches;
+    return SLKV_OK;
+  }
   rc = bind_workspace(&pb, ws, ws_bytes, path);
   if (rc != SLKV_OK) return rc;
   pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
   pb.tab.cu_ptr = cu_dev;
-  int launches = 0;
   const bool clustered = select_cluster_supported(pb);
-  cudaError_t e = cudaSuccess;
   if (!clustered || pb.tab.n_inline == 0) {       // tables in global memory and / or the packed offsets
     e = launch_setup(pb, clustered ? nullptr : budgets, offsets, capacity, status, st, &launches);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -316,6 +417,33 @@ size_t slkv_workspace_bytes(const slkv_params* p, const int32_t* cu_seqlens_host
   return layout_of(pb).total;
 }
 
+size_t slkv_workspace_bytes_overlapped(const slkv_params* p, const int32_t* cu_seqlens_host) {
+  Problem pb;
+  if (describe(p, cu_seqlens_host, &pb) != SLKV_OK) return 0;
+  return layout_of(pb, true).total;
+}
+
+int slkv_compress_overlapped(const slkv_params* p, const void* q_win, const void* k, const void* v,
+                             const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
+                             void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets,
+                             int32_t* kept_idx, float* pooled_opt, int32_t* status, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  {
+    Problem pb;                                   // the overlapped layout is the larger one: check it up front
+    if (p && cu_seqlens_host && describe(p, cu_seqlens_host, &pb) == SLKV_OK && workspace &&
+        workspace_bytes < layout_of(pb, true).total)
+      return SLKV_ERR_WORKSPACE;
+  }
+  return compress_impl(p, q_win, k, v, cu_seqlens_dev, cu_seqlens_host, budgets, k_out, v_out, out_capacity_rows,
+                       offsets, kept_idx, pooled_opt, status, workspace, workspace_bytes, (cudaStream_t)stream, true);
+}
+
+int slkv_join(void* stream) {
+  cudaError_t e = join_overlapped((cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return SLKV_OK;
+}
+
 int64_t slkv_pooled_elems(const slkv_params* p, const int32_t* cu_seqlens_host) {
   Problem pb;
   if (describe(p, cu_seqlens_host, &pb) != SLKV_OK) return -1;
@@ -346,7 +474,8 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
   pb.tab.cu_ptr = cu_seqlens_dev;
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
-  cudaError_t e = cudaSuccess;
+  cudaError_t e = join_overlapped(st);             // the workspace may still serve an overlapped call
+  if (e != cudaSuccess) return cuda_fail(e);
   if (pb.tab.n_inline == 0) {
     e = launch_setup(pb, nullptr, nullptr, 0, nullptr, st, &launches);
     if (e != cudaSuccess) return cuda_fail(e);

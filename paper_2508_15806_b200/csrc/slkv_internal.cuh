@@ -92,6 +92,7 @@ struct Problem {
   float* pooled_ws;       // [n_kv_heads * total_hist] used when the caller wants no pooled output
   int32_t* gather_src;    // [n_kv_heads * total_tokens] per packed row: token * n_kv_heads + head of its source
   int32_t* dev_flags;     // [8] scratch words (timeouts etc.)
+  int max_score_ctas;     // > 0: the score kernels use at most this many CTAs (SMs); 0 = all
 };
 
 // kernel ids for launch accounting / per-kernel timing
@@ -121,6 +122,9 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
 cudaError_t launch_pool(const Problem& pb, float* pooled, cudaStream_t st, int* launches);
 cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t capacity, cudaStream_t st, int* launches);
+bool select_cta_supported(const Problem& pb);
+cudaError_t launch_select_cta(const Problem& pb, float* pooled_out, const int32_t* budgets, int32_t* offsets,
+                              int32_t* kept_idx, int64_t capacity, int32_t* status, cudaStream_t st, int* launches);
 bool select_cluster_supported(const Problem& pb);
 cudaError_t launch_select_cluster(const Problem& pb, float* pooled_out, const int32_t* budgets, int32_t* offsets,
                                   int32_t* kept_idx, int64_t capacity, int32_t* status, cudaStream_t st,

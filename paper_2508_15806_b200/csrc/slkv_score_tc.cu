@@ -640,7 +640,8 @@ Schedule schedule_of(const Problem& pb, const int32_t* cu_host) {
   }
   Schedule sc;
   sc.total_tiles = (int)(tiles * pb.p.n_kv_heads);
-  const int sms = sm_count();
+  int sms = sm_count();
+  if (pb.max_score_ctas > 0 && pb.max_score_ctas < sms) sms = pb.max_score_ctas;
   sc.tiles_per_cta = sc.total_tiles > 0 ? (sc.total_tiles + sms - 1) / sms : 1;
   sc.n_cta = sc.total_tiles > 0 ? (sc.total_tiles + sc.tiles_per_cta - 1) / sc.tiles_per_cta : 0;
   return sc;

@@ -183,3 +183,54 @@ def test_host_buffer_entry_point():
         B.slkv_compress_host(params, x.q_win, x.k, x.v, cu, torch.tensor(bud, dtype=torch.int32),
                              k_out[:10], v_out[:10], offsets, kept[:10], arena)
     assert e.value.code == B.ERR["CAPACITY"]
+
+
+def test_overlapped_calls_match_ordinary_calls():
+    # four layers back to back through one workspace, then a join: bit-identical to one call at a time
+    wl = synth.small_variant(synth.workloads()[2], [9000], n_layers=4, totals=[4 * 8 * 300])
+    dev = torch.device("cuda:0")
+    budgets = O.alloc_budgets(synth.inf_sc(wl).numpy(), wl.fixed, wl.totals[0])
+    xs = [synth.layer_inputs(wl, l, device=dev) for l in range(4)]
+    cu = wl.cu_seqlens
+    cu_dev = torch.tensor(cu, dtype=torch.int32, device=dev)
+    params = B.make_params(xs[0].q_win, xs[0].k, xs[0].v, wl.window, wl.pool_kernel)
+    ws = torch.empty(B.slkv_workspace_bytes_overlapped(params, cu), dtype=torch.uint8, device=dev)
+    assert ws.numel() > B.slkv_workspace_bytes(params, cu)
+    cap = B.slkv_packed_rows_upper_bound(params, cu)
+    # inputs of a call in flight must stay put: the budget rows live as long as the test
+    buds = [torch.tensor(budgets[l].tolist(), dtype=torch.int32, device=dev) for l in range(4)]
+
+    def outputs():
+        return [dict(k_out=torch.zeros(cap, 128, dtype=torch.bfloat16, device=dev),
+                     v_out=torch.zeros(cap, 128, dtype=torch.bfloat16, device=dev),
+                     offsets=torch.zeros(9, dtype=torch.int32, device=dev),
+                     kept=torch.full((cap,), -1, dtype=torch.int32, device=dev),
+                     status=torch.zeros(1, dtype=torch.int32, device=dev)) for _ in range(4)]
+
+    def run(fn, outs):
+        for rep in range(3):                   # several rounds: both vote arrays get reused while in flight
+            for l in range(4):
+                o = outs[l]
+                fn(params, xs[l].q_win, xs[l].k, xs[l].v, cu_dev, cu, buds[l], o["k_out"], o["v_out"],
+                   o["offsets"], o["kept"], ws, None, o["status"])
+        B.slkv_join()
+        torch.cuda.synchronize()
+
+    a, b = outputs(), outputs()
+    run(B.slkv_compress, a)
+    run(B.slkv_compress_overlapped, b)
+    for l in range(4):
+        assert int(b[l]["status"].item()) == 0
+        n = int(a[l]["offsets"][-1].item())
+        assert torch.equal(a[l]["offsets"], b[l]["offsets"]) and n == int(budgets[l].sum())
+        assert torch.equal(a[l]["kept"][:n], b[l]["kept"][:n])
+        assert torch.equal(a[l]["k_out"][:n], b[l]["k_out"][:n]) and torch.equal(a[l]["v_out"][:n], b[l]["v_out"][:n])
+    # an ordinary call right after overlapped ones joins by itself
+    o = outputs()[0]
+    B.slkv_compress_overlapped(params, xs[0].q_win, xs[0].k, xs[0].v, cu_dev, cu, buds[0], b[0]["k_out"],
+                               b[0]["v_out"], b[0]["offsets"], b[0]["kept"], ws, None, b[0]["status"])
+    B.slkv_compress(params, xs[1].q_win, xs[1].k, xs[1].v, cu_dev, cu, buds[1], o["k_out"], o["v_out"],
+                    o["offsets"], o["kept"], ws, None, o["status"])
+    torch.cuda.synchronize()
+    n = int(a[1]["offsets"][-1].item())
+    assert torch.equal(o["kept"][:n], a[1]["kept"][:n]) and torch.equal(b[0]["kept"][:int(a[0]["offsets"][-1])], a[0]["kept"][:int(a[0]["offsets"][-1])])
