@@ -283,7 +283,7 @@ def run_cuda(args):
     q_bytes = len(wl.seq_lens) * w * wl.n_q_heads * d * e
     k_scan = hkv * n_hist * d * e
     rows_avg = sum(L["rows"] for L in layers) / nl
-    alg = {"k_score_lse": k_scan + q_bytes, "k_score_vote": k_scan + q_bytes + 4 * hkv * n_hist,
+    alg = {"k_score_fused": k_scan + q_bytes + 4 * hkv * n_hist, "k_score_lse": k_scan + q_bytes, "k_score_vote": k_scan + q_bytes + 4 * hkv * n_hist,
            "k_pool": 8 * hkv * n_hist, "k_select": 4 * hkv * n_hist + 4 * rows_avg,
            "k_gather": 4 * rows_avg * d * e + 4 * rows_avg, "k_setup": 0}
     kern = {}

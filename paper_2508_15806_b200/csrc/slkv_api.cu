@@ -384,7 +384,7 @@ int slkv_profile_collect(float* total_ms, int32_t* launches, int32_t n_kernels) 
 
 const char* slkv_kernel_name(int kernel_id) {
   static const char* names[KID_COUNT] = {"k_setup", "k_score_lse", "k_score_vote", "k_pool", "k_select",
-                                         "k_gather", "k_alloc"};
+                                         "k_gather", "k_alloc", "k_score_fused"};
   return (kernel_id >= 0 && kernel_id < KID_COUNT) ? names[kernel_id] : "";
 }
 

@@ -96,7 +96,7 @@ struct Problem {
 };
 
 // kernel ids for launch accounting / per-kernel timing
-enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_COUNT };
+enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_COUNT };
 
 // Brackets one kernel launch: counts it and, when per-kernel timing is on for this thread, records a
 // CUDA event pair around it on the launch stream.

@@ -14,6 +14,8 @@
 // SLKV_ERR_DEVICE_TIMEOUT in the status word, stops waiting everywhere, releases TMEM and returns.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "slkv_internal.cuh"
 
 namespace slkv {
@@ -28,7 +30,8 @@ constexpr int kSmemLimit = 227 * 1024;         // dynamic shared memory a CTA ca
 constexpr int kThreads = 384;                  // warps 0-3: TMA, MMA, 2 idle; warps 4-11: epilogue
 constexpr int kEpiThreads = 256;
 constexpr int kTraceSlots = 64;               // per CTA: 0 start, 1 set-up done, 2 Q landed, 3 first K landed,
-                                               // 4 end; 8+2i / 9+2i = epilogue of the CTA's i-th tile begins / ends
+                                               // 4 end; 5 / 6 grid barrier reached / passed, 7 first log-sum-exp merged; 8+2i / 9+2i = epilogue of the
+                                               // CTA's i-th tile begins / ends
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per wait
 
 struct TcArgs {
@@ -38,7 +41,7 @@ struct TcArgs {
   float* vote;
   int32_t* status;
   unsigned long long* trace;    // optional timeline buffer: kTraceSlots timestamps (ns) per CTA, or null
-  int n_seqs, n_kv_heads, G, window, R, MT, n_stages, slot_stride, tiles_per_cta, total_tiles;
+  int n_seqs, n_kv_heads, G, window, R, MT, n_stages, slot_stride, tiles_per_cta, total_tiles, barrier_slot;
   int q_head_inner, k_head_inner;   // tensor-map dimension order: 1 = the head axis comes before the row axis
   float scale_log2;
 };
@@ -59,9 +62,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(2000u) : "memory");   // may sleep up to 2 us: a waiting thread must
+                                                                   // not eat the issue slots of the epilogue warps
   return ok != 0;
 }
 __device__ __forceinline__ unsigned long long now_ns() {
@@ -168,8 +172,7 @@ struct Run { int s, g, t0, count, n_hist, seg_tile0, tiles_seg; };
 
 // A run = consecutive tiles of one segment inside the CTA's range [begin, end).  Forward walks (pass 1)
 // name a run by its first tile, backward walks (pass 2) by its last one.
-template <bool REV>
-__device__ __forceinline__ Run locate(const TcArgs& a, int pos, int begin, int end) {
+__device__ __forceinline__ Run locate(const TcArgs& a, int pos, int begin, int end, bool REV) {
   int lo = 0, hi = a.n_seqs;                       // last s with Hkv*tile_off[s] <= pos
   while (hi - lo > 1) {
     int mid = (lo + hi) >> 1;
@@ -241,7 +244,35 @@ __device__ __noinline__ void tile_row_stats_exact(uint32_t tcol, float sc, int n
   m_io = m; z_io = z;
 }
 
-template <int PASS>
+// Grid-wide barrier of the fused kernel (both passes in one launch): one arrival counter per launch, taken in
+// turn from a small table in the module's globals (zero at load).  atom.inc wraps the counter back to zero with
+// the last arrival, so a waiter -- which has arrived itself, hence has seen the counter above zero -- is done
+// when it reads zero, and the slot is clean for its next user 64 launches later.  The kernel is launched
+// cooperatively (all CTAs resident); the wait is bounded all the same.
+constexpr int kBarrierSlots = 64;
+__device__ unsigned g_grid_arrivals[kBarrierSlots];
+
+__device__ __forceinline__ bool grid_barrier(unsigned* counter, unsigned n_cta, volatile int* abort_flag) {
+  // Called by one thread after a CTA-wide barrier: the release on the arrival makes the CTA's earlier writes
+  // visible to whoever acquires the counter afterwards.
+  unsigned prev;
+  asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(prev) : "l"(counter), "r"(n_cta - 1) : "memory");
+  if (prev == n_cta - 1) return true;
+  const unsigned long long t0 = now_ns();
+  for (unsigned it = 1;; ++it) {
+    unsigned c;
+    asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(c) : "l"(counter) : "memory");
+    if (c == 0) return true;
+    if ((it & 15u) == 0) {
+      if (*abort_flag) return false;
+      if (now_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+    __nanosleep(32);
+  }
+}
+
+// MODE 1: row statistics pass only; MODE 2: vote pass only; MODE 3: both, separated by a grid-wide barrier.
+template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ TcArgs a) {
@@ -304,11 +335,12 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   // Everything above touched only this CTA's own resources.  Pass 1 reads its inputs after the kernels
   // before it have finished.  In pass 2 the loads and the tensor-core work need only Q and K, which pass 1
   // has already read, so they start at once; the epilogue alone waits for pass 1's row statistics.
+  constexpr int kFirstPass = MODE == 2 ? 2 : 1, kLastPass = MODE == 1 ? 1 : 2;
   pdl_launch_dependents();
-  if (PASS == 1 && warp >= 4) {
+  if (MODE != 2 && warp >= 4) {
     bool ragged = false;                                            // a segment's ragged last tile in this CTA's range?
     for (int pos = begin; pos < end;) {
-      const Run r = locate<false>(a, pos, begin, end);
+      const Run r = locate(a, pos, begin, end, false);
       ragged |= r.t0 + r.count == r.tiles_seg && (r.n_hist & (kTileKeys - 1)) != 0;
       pos += r.count;
     }
@@ -318,14 +350,14 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       if (zw == 12345.f) abort_sh = 0;                              // keeps the call alive; writes what is there
     }
   }
-  if (PASS == 1 || warp >= 4) pdl_wait();
+  if (MODE != 2 || warp >= 4) pdl_wait();
   if (tid == 0) trace_mark(a.trace, 1);
 
-  constexpr bool REV = PASS == 2;      // pass 2 walks the CTA's tiles backwards: the last ones read are likeliest in L2
-  const int pos0 = REV ? end - 1 : begin;
-  auto more = [&](int pos) { return REV ? pos >= begin : pos < end; };
-  auto advance = [&](int pos, const Run& r) { return REV ? pos - r.count : pos + r.count; };
-  auto tile_of = [&](const Run& r, int i) { return r.t0 + (REV ? r.count - 1 - i : i); };
+  // pass 2 walks the CTA's tiles backwards: the last ones read are likeliest in L2
+  auto first_pos = [&](bool REV) { return REV ? end - 1 : begin; };
+  auto more = [&](int pos, bool REV) { return REV ? pos >= begin : pos < end; };
+  auto advance = [&](int pos, const Run& r, bool REV) { return REV ? pos - r.count : pos + r.count; };
+  auto tile_of = [&](const Run& r, int i, bool REV) { return r.t0 + (REV ? r.count - 1 - i : i); };
 
   // The two single-thread loops below are the pipeline's metronome: whatever they spend per tile between two
   // issues is dead time for the tensor pipe (a tcgen05.mma issue blocks its thread while the pipe is busy),
@@ -337,15 +369,17 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       int it = 0, run_idx = 0, st = 0;
       uint32_t st_phase = 0;                                             // parity of the ring pass in progress
       bool ok = true;
-      for (int pos = pos0; more(pos) && ok;) {
-        const Run r = locate<REV>(a, pos, begin, end);
+     for (int pass = kFirstPass; pass <= kLastPass && ok; ++pass) {
+      const bool REV = pass == 2;
+      for (int pos = first_pos(REV); more(pos, REV) && ok;) {
+        const Run r = locate(a, pos, begin, end, REV);
         ok = mbar_wait(qempty_bar, (run_idx & 1) ^ 1, abort_flag);      // previous run's MMAs are done with Q
         if (!ok) break;
         mbar_expect_tx(qfull_bar, 2u * (uint32_t)R * 128u);
         const int qy = a.q_head_inner ? r.g * a.G : 0, qz = a.q_head_inner ? 0 : r.g * a.G;
         tma_load_4d(q_smem, &tm_q, 0, qy, qz, r.s, qfull_bar);
         tma_load_4d(q_smem + q_half_bytes, &tm_q, 64, qy, qz, r.s, qfull_bar);
-        int tok = a.tab.cu_at(r.s) + tile_of(r, 0) * kTileKeys;
+        int tok = a.tab.cu_at(r.s) + tile_of(r, 0, REV) * kTileKeys;
         const int tok_step = REV ? -kTileKeys : kTileKeys;
         for (int i = 0; i < r.count; ++i, ++it, tok += tok_step) {
           ok = mbar_wait(empty_bar(st), st_phase ^ 1u, abort_flag);
@@ -357,9 +391,10 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           tma_load_3d(dst + kHalfBytes, &tm_k, 64, ky, kz, fb);
           if (++st == kStages) { st = 0; st_phase ^= 1u; }
         }
-        pos = advance(pos, r);
+        pos = advance(pos, r, REV);
         ++run_idx;
       }
+     }
       if (!ok) {
         // give loads already in flight a bounded chance to land before the CTA's shared memory goes away
         const unsigned long long t0 = now_ns();
@@ -377,7 +412,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // idle, with two the other thread is already past its waits and its MMAs queue up right behind.
     if (lane == 0) {
       const int me = warp - 1;
-      const uint32_t idesc = PASS == 1 ? instr_desc(128, kTileKeys) : instr_desc(kTileKeys, R);
+      const uint32_t idesc1 = instr_desc(128, kTileKeys), idesc2 = instr_desc(kTileKeys, R);
       // descriptor of the k-step ks of a tile = descriptor of the tile + (byte offset >> 4); the address field
       // cannot carry out of its 14 bits because shared memory ends below 256 KB
       const uint64_t q_desc0 = smem_desc(q_smem), k_desc0 = smem_desc(k_smem);
@@ -387,8 +422,11 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       uint64_t k_desc = k_desc0;
       uint32_t d0 = tmem_base;
       bool ok = true;
-      for (int pos = pos0; more(pos) && ok;) {
-        const Run r = locate<REV>(a, pos, begin, end);
+     for (int pass = kFirstPass; pass <= kLastPass && ok; ++pass) {
+      const bool REV = pass == 2;
+      const uint32_t idesc = pass == 1 ? idesc1 : idesc2;
+      for (int pos = first_pos(REV); more(pos, REV) && ok;) {
+        const Run r = locate(a, pos, begin, end, REV);
         ok = mbar_wait(qfull_bar, run_idx & 1, abort_flag);
         if (!ok) break;
         if (run_idx == 0 && me == 0) trace_mark(a.trace, 2);
@@ -398,7 +436,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           if (!ok) break;
           if (it == 0) trace_mark(a.trace, 3);
           tc_fence_after();
-          if (PASS == 1) {
+          if (pass == 1) {
             for (int mt = 0; mt < MT; ++mt) {
               const uint64_t qd = q_desc0 + (uint64_t)(mt * ((128 * 128) >> 4));
 #pragma unroll
@@ -423,9 +461,10 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           if (++b == n_bufs) { b = 0; b_phase ^= 1u; d0 = tmem_base; }
         }
         tc_commit(qempty_bar);            // Q tile free once the run's MMAs (of both issuers) are done
-        pos = advance(pos, r);
+        pos = advance(pos, r, REV);
         ++run_idx;
       }
+     }
     }
   } else if (warp >= 4) {
     // ---------------- epilogue: two warpgroups, alternating tiles ----------------
@@ -437,38 +476,66 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const float inv_g = 1.0f / (float)a.G;
     int it = 0, run_idx = 0;
     bool ok = true;
-    for (int pos = pos0; more(pos);) {
-      const Run r = locate<REV>(a, pos, begin, end);
+   for (int pass = kFirstPass; pass <= kLastPass; ++pass) {
+    const bool REV = pass == 2;
+    if (MODE == 3 && pass == 2) {
+      // every CTA's row statistics must be in memory before any row's log-sum-exp is formed
+      epi_bar();
+      if (et == 0) trace_mark(a.trace, 5);
+      if (et == 0 && ok) grid_barrier(&g_grid_arrivals[a.barrier_slot], gridDim.x, abort_flag);
+      if (et == 0) trace_mark(a.trace, 6);
+      epi_bar();
+      ok = ok && *abort_flag == 0;
+    }
+    for (int pos = first_pos(REV); more(pos, REV);) {
+      const Run r = locate(a, pos, begin, end, REV);
       const int seg = r.s * a.n_kv_heads + r.g;
       const int first_cta = r.seg_tile0 / a.tiles_per_cta;
       float m_run[2] = {0.f, 0.f}, z_run[2] = {0.f, 0.f};      // reference 0: see the fast path below
       float* lse = stats + 256 * (run_idx & 1);
-      if (PASS == 2) {
+      if (pass == 2) {
         // merge the per-CTA partials of this segment into the rows' log-sum-exp (log2 units)
         const int n_slots = (r.seg_tile0 + r.tiles_seg - 1) / a.tiles_per_cta - first_cta + 1;
-        if (et < R) {
-          const float* pm = a.part_m + (long long)seg * a.slot_stride * R + et;      // [segment][slot][row]
-          const float* pz = a.part_z + (long long)seg * a.slot_stride * R + et;
+        // Every thread has all its loads in flight before it uses one.  With R <= 128 two neighbouring lanes
+        // share a row (even / odd slots) and combine through a shuffle.
+        {
+          const int halves = 2 * R <= kEpiThreads ? 2 : 1;
+          const int rr = halves == 2 ? ((et >> 1) < R ? (et >> 1) : -1) : (et < R ? et : -1);
+          const int half = halves == 2 ? (et & 1) : 0;
           float M = -INFINITY, Z = 0.f;
-          for (int c0 = 0; c0 < n_slots; c0 += 8) {                                   // sixteen loads in flight
-            float m8[8], z8[8];
+          if (rr >= 0) {
+            const float* pm = a.part_m + (long long)seg * a.slot_stride * R + rr;      // [segment][slot][row]
+            const float* pz = a.part_z + (long long)seg * a.slot_stride * R + rr;
+            for (int c0 = half; c0 < n_slots; c0 += 12 * halves) {
+              float m12[12], z12[12];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              const bool in = c0 + u < n_slots;
-              m8[u] = in ? __ldcg(pm + (long long)(c0 + u) * R) : -INFINITY;
-              z8[u] = in ? __ldcg(pz + (long long)(c0 + u) * R) : 0.f;
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              if (m8[u] > -INFINITY) {
-                const float Mn = fmaxf(M, m8[u]);
-                Z = Z * ex2(M - Mn) + z8[u] * ex2(m8[u] - Mn);      // ex2(-inf) = 0 covers the first term
-                M = Mn;
+              for (int u = 0; u < 12; ++u) {
+                const int c = c0 + u * halves;
+                const bool in = c < n_slots;
+                m12[u] = in ? __ldcg(pm + (long long)c * R) : -INFINITY;
+                z12[u] = in ? __ldcg(pz + (long long)c * R) : 0.f;
               }
+#pragma unroll
+              for (int u = 0; u < 12; ++u)
+                if (m12[u] > -INFINITY) {
+                  const float Mn = fmaxf(M, m12[u]);
+                  Z = Z * ex2(M - Mn) + z12[u] * ex2(m12[u] - Mn);      // ex2(-inf) = 0 covers the first term
+                  M = Mn;
+                }
+            }
           }
-          lse[et] = M + log2f(Z);
+          if (halves == 2) {                                              // uniform over the warp
+            const float M1 = __shfl_xor_sync(0xffffffffu, M, 1), Z1 = __shfl_xor_sync(0xffffffffu, Z, 1);
+            const float Mn = fmaxf(M, M1);
+            float Zt = 0.f;
+            if (M > -INFINITY) Zt += Z * ex2(M - Mn);
+            if (M1 > -INFINITY) Zt += Z1 * ex2(M1 - Mn);
+            M = Mn; Z = Zt;
+          }
+          if (half == 0 && rr >= 0) lse[rr] = M + log2f(Z);
         }
         epi_bar();
+        if (et == 0 && pass == 2 && pos == first_pos(true)) trace_mark(a.trace, 7);
       }
       for (int i = 0; i < r.count; ++i, ++it) {
         if ((it & 1) != wg) continue;
@@ -478,10 +545,10 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         if (!ok) continue;
         tc_fence_after();
         if (row == 0 && it < 28) trace_mark(a.trace, 8 + 2 * it);
-        const int key0 = tile_of(r, i) * kTileKeys;
+        const int key0 = tile_of(r, i, REV) * kTileKeys;
         const uint32_t tb = tmem_base + lane_sel + (uint32_t)(b * buf_cols);
         uint32_t ra[32], rb[32];
-        if (PASS == 1) {
+        if (pass == 1) {
           const int n_valid = min(r.n_hist - key0, kTileKeys);
           for (int mt = 0; mt < MT; ++mt) {
             const uint32_t tcol = tb + mt * 128;
@@ -551,14 +618,14 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const int j = key0 + row;
           if (j < r.n_hist) a.vote[a.tab.hist_at(r.s) * a.n_kv_heads + (long long)r.g * r.n_hist + j] = acc * inv_g;
         }
-        if (PASS == 1) {
+        if (pass == 1) {
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(acce_bar(b));
         }
         if (row == 0 && it < 28) trace_mark(a.trace, 9 + 2 * it);
       }
-      if (PASS == 1) {
+      if (pass == 1) {
         // combine the two warpgroups' statistics and publish this CTA's partial for the segment
         const int slot = blockIdx.x - first_cta;
         for (int mt = 0; mt < MT; ++mt) {
@@ -578,9 +645,10 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           epi_bar();
         }
       }
-      pos = advance(pos, r);
+      pos = advance(pos, r, REV);
       ++run_idx;
     }
+   }
   }
 
   tc_fence_before();
@@ -712,6 +780,7 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
   a.tab = pb.tab;
   a.part_m = pb.part_m; a.part_z = pb.part_z; a.vote = pb.vote; a.status = status;
   a.trace = nullptr;
+  a.barrier_slot = 0;
   a.n_seqs = p.n_seqs; a.n_kv_heads = p.n_kv_heads; a.G = pb.G; a.window = p.window; a.R = pb.R;
   a.MT = (pb.R + 127) / 128;
   a.q_head_inner = q_head_inner; a.k_head_inner = k_head_inner;
@@ -733,6 +802,51 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
     e = cudaFuncSetAttribute(k_score_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
     if (e != cudaSuccess) return e;
     configured_dev = dev;
+  }
+  // Both passes in one cooperative launch when the device takes it (all CTAs resident: the kernel has a
+  // grid-wide barrier); otherwise two launches.
+  static thread_local int fused_state[64] = {};       // per device: 0 untried, 1 cooperative + dependent launch,
+                                                      // 2 cooperative only, -1 not available
+  int& fs = fused_state[dev < 64 ? dev : 0];
+  if (fs == 0) {
+    int coop = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) fs = -1;
+    else if (cudaFuncSetAttribute(k_score_tc<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
+      fs = -1;
+    else fs = 1;
+  }
+  if (fs > 0 && sc.n_cta <= sm_count()) {
+    for (int attempt = 0; attempt < 2 && fs > 0; ++attempt) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(sc.n_cta);
+      cfg.blockDim = dim3(kThreads);
+      cfg.dynamicSmemBytes = smem;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[2];
+      int n = 0;
+      attr[n].id = cudaLaunchAttributeCooperative;
+      attr[n].val.cooperative = 1;
+      ++n;
+      if (fs == 1) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+      }
+      cfg.attrs = attr;
+      cfg.numAttrs = n;
+      a.trace = trace_buffer(1, sc.n_cta);
+      static std::atomic<unsigned> launch_seq{0};
+      a.barrier_slot = (int)(launch_seq.fetch_add(1) % kBarrierSlots);
+      cudaError_t le;
+      {
+        LaunchScope scope(KID_SCORE_FUSED, st, launches);
+        le = cudaLaunchKernelEx(&cfg, k_score_tc<3>, tm_q, tm_k, a);
+      }
+      if (le == cudaSuccess) return cudaSuccess;
+      (void)cudaGetLastError();                       // not a sticky error: the launch was refused
+      --*launches;
+      fs = fs == 1 ? 2 : -1;                          // try without dependent launch, then give up on fusing
+    }
   }
   {
     LaunchScope scope(KID_SCORE_LSE, st, launches);

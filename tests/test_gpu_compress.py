@@ -129,7 +129,7 @@ def test_deterministic_and_pooled_optional():
     a = P.gpu_compress(x.q_win, x.k, x.v, wl.cu_seqlens, bud, wl.window, wl.pool_kernel)
     b = P.gpu_compress(x.q_win, x.k, x.v, wl.cu_seqlens, bud, wl.window, wl.pool_kernel, want_pooled=False)
     assert np.array_equal(a["kept_idx"], b["kept_idx"]) and torch.equal(a["k_out"], b["k_out"])
-    assert a["launches"] >= 4
+    assert a["launches"] >= 3          # score (both passes in one launch where the device allows), select, gather
 
 
 def test_strided_kv_layout():
