@@ -163,10 +163,10 @@ int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const 
  *     when the call returns.  slkv_join(stream) makes `stream` wait for every overlapped call enqueued so far
  *     on the current device (no host wait); consume outputs, or free / overwrite any input, output or
  *     workspace buffer, only behind it.  Any other slkv_* call that uses a workspace joins by itself first.
- *   - workspace must hold slkv_workspace_bytes_overlapped (two vote arrays: successive calls alternate).
+ *   - workspace must hold slkv_workspace_bytes_overlapped (two vote arrays and two source-row lists: successive calls alternate).
  *     Successive calls may share one workspace; q_win, k, v, budgets and the outputs of calls that may be in
  *     flight together must not alias each other's outputs.
- *   - The first call on a device creates the side stream and four events (no device memory).
+ *   - The first call on a device creates two side streams and six events (no device memory).
  *   - Shapes the overlapped path does not take (more than 64 sequences, a segment with more than 32768
  *     history positions, pool_kernel > 9) run as slkv_compress does, on `stream`, after a join.
  * Arguments, results and error codes otherwise as slkv_compress.

@@ -42,7 +42,7 @@ int cuda_fail(cudaError_t e) {
 }
 
 struct Layout {
-  size_t hist_off, tile_off, vote, vote2, pooled, part_m, part_z, flags, gather_src, total;
+  size_t hist_off, tile_off, vote, vote2, pooled, part_m, part_z, flags, gather_src, gather_src2, total;
 };
 
 // Validates p and cu_seqlens_host and fills the host-known fields of `pb`.
@@ -126,6 +126,10 @@ Layout layout_of(const Problem& pb, bool overlapped = false) {
   L.part_z = o; o = align_up(o + parts);
   L.flags = o; o = align_up(o + 8 * sizeof(int32_t));
   L.gather_src = o; o = align_up(o + (size_t)pb.p.n_kv_heads * (size_t)pb.total_tokens * sizeof(int32_t));
+  L.gather_src2 = L.gather_src;                      // overlapped calls: a gather may still read one list while
+  if (overlapped) {                                  // the next selection writes the other
+    L.gather_src2 = o; o = align_up(o + (size_t)pb.p.n_kv_heads * (size_t)pb.total_tokens * sizeof(int32_t));
+  }
   L.total = o;
   return L;
 }
@@ -156,7 +160,7 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overla
   pb->part_m = reinterpret_cast<float*>(b + L.part_m);
   pb->part_z = reinterpret_cast<float*>(b + L.part_z);
   pb->dev_flags = reinterpret_cast<int32_t*>(b + L.flags);
-  pb->gather_src = reinterpret_cast<int32_t*>(b + L.gather_src);
+  pb->gather_src = reinterpret_cast<int32_t*>(b + (half ? L.gather_src2 : L.gather_src));
   pb->chunk_keys = path == SLKV_PATH_TENSOR ? 128 : simt_chunk_keys();
   pb->n_chunks = path == SLKV_PATH_TENSOR ? tensor_slot_stride(*pb)
                                           : (pb->max_hist + pb->chunk_keys - 1) / pb->chunk_keys;
@@ -178,9 +182,10 @@ int enqueue_votes(const Problem& pb, int path, const int32_t* cu_host, int32_t* 
 // ---- overlapped calls: selection and gather of one call run on a side stream while the next call's score
 // kernels run on the caller's stream --------------------------------------------------------------------
 struct OverlapState {
-  cudaStream_t side = nullptr;
+  cudaStream_t side_select = nullptr, side_gather = nullptr;
   cudaEvent_t scored[2] = {nullptr, nullptr};     // recorded on the caller's stream after the vote pass
-  cudaEvent_t done[2] = {nullptr, nullptr};       // recorded on the side stream after the gather
+  cudaEvent_t selected[2] = {nullptr, nullptr};   // recorded on the selection stream after the selection
+  cudaEvent_t done[2] = {nullptr, nullptr};       // recorded on the gather stream after the gather
   bool in_flight[2] = {false, false};
   unsigned seq = 0;
 };
@@ -195,11 +200,15 @@ cudaError_t overlap_state(OverlapState** out) {
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   OverlapState& s = g_overlap[dev];
-  if (!s.side) {
-    e = cudaStreamCreateWithFlags(&s.side, cudaStreamNonBlocking);
+  if (!s.side_select) {
+    e = cudaStreamCreateWithFlags(&s.side_select, cudaStreamNonBlocking);
+    if (e != cudaSuccess) return e;
+    e = cudaStreamCreateWithFlags(&s.side_gather, cudaStreamNonBlocking);
     if (e != cudaSuccess) return e;
     for (int h = 0; h < 2; ++h) {
       e = cudaEventCreateWithFlags(&s.scored[h], cudaEventDisableTiming);
+      if (e != cudaSuccess) return e;
+      e = cudaEventCreateWithFlags(&s.selected[h], cudaEventDisableTiming);
       if (e != cudaSuccess) return e;
       e = cudaEventCreateWithFlags(&s.done[h], cudaEventDisableTiming);
       if (e != cudaSuccess) return e;
@@ -271,21 +280,25 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int reserve = pb.n_seg < kSelectSmReserve ? pb.n_seg : kSelectSmReserve;
     pb.max_score_ctas = sms - reserve > 0 ? sms - reserve : 0;
-    if (os->in_flight[half]) {                     // the vote array of this half is read by a selection two calls back
-      e = cudaStreamWaitEvent(st, os->done[half], 0);
+    if (os->in_flight[half]) {                     // the vote array of this half is read by the selection two calls
+      e = cudaStreamWaitEvent(st, os->selected[half], 0);          // back, its source-row list by that call's gather
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_select, os->done[half], 0);
       if (e != cudaSuccess) return cuda_fail(e);
-      os->in_flight[half] = false;
     }
     rc = enqueue_votes(pb, path, cu_host, status, st, &launches);
     if (rc != SLKV_OK) return rc;
+    // selection on one side stream, gather on another: the gather of a call runs beside the selection of the next
     e = cudaEventRecord(os->scored[half], st);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side, os->scored[half], 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_select, os->scored[half], 0);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_select_cta(pb, pooled_opt, budgets, offsets, kept_idx, capacity, status, os->side, &launches);
+    e = launch_select_cta(pb, pooled_opt, budgets, offsets, kept_idx, capacity, status, os->side_select, &launches);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_gather(pb, offsets, kept_idx, k_out, v_out, capacity, os->side, &launches);
+    e = cudaEventRecord(os->selected[half], os->side_select);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_gather, os->selected[half], 0);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = cudaEventRecord(os->done[half], os->side);
+    e = launch_gather(pb, offsets, kept_idx, k_out, v_out, capacity, os->side_gather, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaEventRecord(os->done[half], os->side_gather);
     if (e != cudaSuccess) return cuda_fail(e);
     os->in_flight[half] = true;
     g_last_launches = launches;
