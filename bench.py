@@ -30,7 +30,7 @@ from paper_2508_15806_b200 import synth  # noqa: E402
 
 METRIC = "context tokens compressed per second per layer"
 UNIT = "tokens/s/layer"
-WORKLOAD_INDEX = 2          # configs[2]: the 32k-context, 32-layer configuration the target is quoted on
+WORKLOAD_INDEX = 2          # the 32k-context, 32-layer configuration (third of the five workloads)
 TOTAL_INDEX = 1             # average budget 512 per KV head
 # DRAM bytes per key row (256 B of K) of one launch, from an ncu capture of the kernel as it stands; a kernel
 # that has changed since its capture has no entry (traffic is then reported as null)
