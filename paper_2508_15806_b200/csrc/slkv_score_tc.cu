@@ -64,7 +64,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity), "r"(2000u) : "memory");   // may sleep up to 2 us: a waiting thread must
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(100u) : "memory");    // may sleep up to 0.1 us: a waiting thread must
                                                                    // not eat the issue slots of the epilogue warps
   return ok != 0;
 }
@@ -312,6 +312,9 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 
   if (tid == 0) trace_mark(a.trace, 0);
   if (tid == 0) {
+    // the tensor maps travel as kernel parameters: have them fetched while the CTA sets itself up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_k)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_q)) : "memory");
     abort_sh = 0;
     for (int st = 0; st < kStages; ++st) { mbar_init(full_bar(st), 1); mbar_init(empty_bar(st), 1); }
     for (int b = 0; b < 4; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
@@ -560,17 +563,15 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               // a non-finite or zero sum shows that, and the tile is then redone exactly.
               float zt = z;
               tc_ld32_issue(tcol, ra);
-              tc_ld_wait(ra);
-              tc_ld32_issue(tcol + 32, rb);
-              zt += sum_ex2_32(ra, sc, m);
-              tc_ld_wait(rb);
-              tc_ld32_issue(tcol + 64, ra);
-              zt += sum_ex2_32(rb, sc, m);
-              tc_ld_wait(ra);
-              tc_ld32_issue(tcol + 96, rb);
-              zt += sum_ex2_32(ra, sc, m);
-              tc_ld_wait(rb);
-              zt += sum_ex2_32(rb, sc, m);
+#pragma unroll 1
+              for (int c0 = 0; c0 < kTileKeys; c0 += 64) {      // rolled: half the code to keep in the instruction cache
+                tc_ld_wait(ra);
+                tc_ld32_issue(tcol + c0 + 32, rb);
+                zt += sum_ex2_32(ra, sc, m);
+                tc_ld_wait(rb);
+                if (c0 + 64 < kTileKeys) tc_ld32_issue(tcol + c0 + 64, ra);
+                zt += sum_ex2_32(rb, sc, m);
+              }
               if (zt < INFINITY && zt > 0.f) z = zt; else exact = true;
             }
             if (exact) tile_row_stats_exact(tcol, sc, n_valid, m, z);
