@@ -151,12 +151,12 @@ def run_cuda(args):
         dist.init_process_group("nccl", device_id=dev)
     B.lib()
 
-    wl = synth.workloads()[WORKLOAD_INDEX]
+    wl = synth.workloads()[(args.workload - 1) if args.workload else WORKLOAD_INDEX]
     if args.layers:
         wl = synth.small_variant(wl, wl.seq_lens, n_layers=args.layers,
-                                 totals=[t // 32 * args.layers for t in wl.totals])
+                                 totals=[t // wl.n_layers * args.layers for t in wl.totals])
     wl = rank_workload(wl, rank, world)
-    total = wl.totals[TOTAL_INDEX]
+    total = wl.totals[TOTAL_INDEX if len(wl.totals) > TOTAL_INDEX else 0]
     cu = wl.cu_seqlens
     T, nl, hkv, d, w = wl.total_tokens, wl.n_layers, wl.n_kv_heads, wl.head_dim, wl.window
     e = wl.elem_size
@@ -425,6 +425,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="use fewer layers (profiling captures only)")
+    ap.add_argument("--workload", type=int, default=0, choices=[0, 1, 2, 3, 4, 5],
+                    help="time another of the five workloads (default: the 32k-context one); the others are parity cases")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="one layer at a time (slkv_compress) instead of overlapped calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
