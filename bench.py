@@ -289,7 +289,7 @@ def run_cuda(args):
     q_bytes = len(wl.seq_lens) * w * wl.n_q_heads * d * e
     k_scan = hkv * n_hist * d * e
     rows_avg = sum(L["rows"] for L in layers) / nl
-    alg = {"k_score_fused": k_scan + q_bytes + 4 * hkv * n_hist, "k_score_lse": k_scan + q_bytes, "k_score_vote": k_scan + q_bytes + 4 * hkv * n_hist,
+    alg = {"k_score_fused": k_scan + q_bytes + 4 * hkv * n_hist, "k_score_pipe": k_scan + q_bytes + 4 * hkv * n_hist, "k_score_lse": k_scan + q_bytes, "k_score_vote": k_scan + q_bytes + 4 * hkv * n_hist,
            "k_pool": 8 * hkv * n_hist, "k_select": 4 * hkv * n_hist + 4 * rows_avg,
            "k_gather": 4 * rows_avg * d * e + 4 * rows_avg, "k_setup": 0}
     kern = {}
@@ -315,6 +315,14 @@ def run_cuda(args):
                           "frac": layer_bytes / (t_layer_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
                           "frac_of_8TBs_nominal": layer_bytes / (t_layer_us * 1e-6) / 8e12},
                 "ceilings": ceilings}
+    # The score kernel's own ceiling is the special-function unit, not HBM: two exponentials per (query row, key)
+    # at 16 ex2.approx per clock per SM need longer than streaming K once.  Reported beside the HBM figures.
+    if top.startswith("k_score"):
+        n_exp = exps_layer if top in ("k_score_fused", "k_score_pipe") else exps_layer / 2
+        peak_gexp = 148 * 16 * 1965e6 / 1e9
+        roofline["alu"] = {"bound": "alu", "unit": "Gexp/s", "achieved": n_exp / (top_us * 1e-6) / 1e9, "peak": peak_gexp,
+                           "frac": n_exp / (top_us * 1e-6) / 1e9 / peak_gexp, "exps_per_launch": n_exp,
+                           "peak_source": "148 SMs x 16 ex2.approx per clock x 1965 MHz (nominal unit count and maximum clock)"}
     tr = DRAM_TRAFFIC_PER_KEY_ROW.get(top)
     if tr:
         roofline["traffic"] = tr["bytes"] * hkv * n_hist

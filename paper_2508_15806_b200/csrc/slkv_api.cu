@@ -42,7 +42,7 @@ int cuda_fail(cudaError_t e) {
 }
 
 struct Layout {
-  size_t hist_off, tile_off, vote, vote2, pooled, part_m, part_z, flags, gather_src, gather_src2, total;
+  size_t hist_off, tile_off, vote[3], pooled, part_m[2], part_z[2], flags, gather_src[3], total;
 };
 
 // Validates p and cu_seqlens_host and fills the host-known fields of `pb`.
@@ -115,20 +115,29 @@ Layout layout_of(const Problem& pb, bool overlapped = false) {
   size_t o = 0;
   L.hist_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int64_t));
   L.tile_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int32_t));
+  // Overlapped calls keep up to three layers in flight: the votes and the source-row list of a layer are read by
+  // its selection and its gather while the score kernels of the next two layers run; the per-CTA row statistics
+  // live from one launch to the next (two sets).  Ordinary calls use the first of each.
   const size_t votes = (size_t)pb.p.n_kv_heads * (size_t)pb.total_hist * sizeof(float);
-  L.vote = o; o = align_up(o + votes);
-  L.vote2 = L.vote;                                  // overlapped calls alternate between two vote arrays
-  if (overlapped) { L.vote2 = o; o = align_up(o + votes); }
+  const int n_slots = overlapped ? 3 : 1, n_parts = overlapped ? 2 : 1;
+  for (int i = 0; i < 3; ++i) {
+    L.vote[i] = i < n_slots ? o : L.vote[0];
+    if (i < n_slots) o = align_up(o + votes);
+  }
   L.pooled = o; o = align_up(o + votes);
   const size_t nchunks = (size_t)(pb.max_hist + kMinChunkKeys - 1) / kMinChunkKeys + 2;
   const size_t parts = (size_t)pb.n_seg * pb.R * nchunks * sizeof(float);
-  L.part_m = o; o = align_up(o + parts);
-  L.part_z = o; o = align_up(o + parts);
+  for (int i = 0; i < 2; ++i) {
+    L.part_m[i] = i < n_parts ? o : L.part_m[0];
+    if (i < n_parts) o = align_up(o + parts);
+    L.part_z[i] = i < n_parts ? o : L.part_z[0];
+    if (i < n_parts) o = align_up(o + parts);
+  }
   L.flags = o; o = align_up(o + 8 * sizeof(int32_t));
-  L.gather_src = o; o = align_up(o + (size_t)pb.p.n_kv_heads * (size_t)pb.total_tokens * sizeof(int32_t));
-  L.gather_src2 = L.gather_src;                      // overlapped calls: a gather may still read one list while
-  if (overlapped) {                                  // the next selection writes the other
-    L.gather_src2 = o; o = align_up(o + (size_t)pb.p.n_kv_heads * (size_t)pb.total_tokens * sizeof(int32_t));
+  const size_t srcs = (size_t)pb.p.n_kv_heads * (size_t)pb.total_tokens * sizeof(int32_t);
+  for (int i = 0; i < 3; ++i) {
+    L.gather_src[i] = i < n_slots ? o : L.gather_src[0];
+    if (i < n_slots) o = align_up(o + srcs);
   }
   L.total = o;
   return L;
@@ -145,7 +154,9 @@ int resolve_path(const Problem& pb, int* path) {
   return SLKV_OK;
 }
 
-int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overlapped = false, int half = 0) {
+// slot: which of the three vote arrays / source-row lists (overlapped calls), part: which set of row statistics
+int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overlapped = false, int slot = 0,
+                   int part = 0) {
   if (!ws) return SLKV_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) % kAlign != 0) return SLKV_ERR_BAD_ALIGN;
   Layout L = layout_of(*pb, overlapped);
@@ -155,12 +166,12 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overla
   pb->tile_off = reinterpret_cast<int32_t*>(b + L.tile_off);
   pb->tab.tile_ptr = pb->tile_off;
   pb->tab.hist_ptr = reinterpret_cast<const long long*>(pb->hist_off);
-  pb->vote = reinterpret_cast<float*>(b + (half ? L.vote2 : L.vote));
+  pb->vote = reinterpret_cast<float*>(b + L.vote[slot]);
   pb->pooled_ws = reinterpret_cast<float*>(b + L.pooled);
-  pb->part_m = reinterpret_cast<float*>(b + L.part_m);
-  pb->part_z = reinterpret_cast<float*>(b + L.part_z);
+  pb->part_m = reinterpret_cast<float*>(b + L.part_m[part]);
+  pb->part_z = reinterpret_cast<float*>(b + L.part_z[part]);
   pb->dev_flags = reinterpret_cast<int32_t*>(b + L.flags);
-  pb->gather_src = reinterpret_cast<int32_t*>(b + (half ? L.gather_src2 : L.gather_src));
+  pb->gather_src = reinterpret_cast<int32_t*>(b + L.gather_src[slot]);
   pb->chunk_keys = path == SLKV_PATH_TENSOR ? 128 : simt_chunk_keys();
   pb->n_chunks = path == SLKV_PATH_TENSOR ? tensor_slot_stride(*pb)
                                           : (pb->max_hist + pb->chunk_keys - 1) / pb->chunk_keys;
@@ -179,20 +190,50 @@ int enqueue_votes(const Problem& pb, int path, const int32_t* cu_host, int32_t* 
   return SLKV_OK;
 }
 
-// ---- overlapped calls: selection and gather of one call run on a side stream while the next call's score
-// kernels run on the caller's stream --------------------------------------------------------------------
+// ---- overlapped calls ---------------------------------------------------------------------------------------
+// The selection and the gather of a layer run on side streams while the score kernels of the following layers
+// run on the caller's stream.  Where the two-layer score kernel takes the shape, a call enqueues pass 1 of its
+// own layer together with pass 2 of the layer before (which stays "pending" until the next call or a join).
+constexpr int kSlots = 3;
+struct PendingCall {
+  bool valid = false;
+  Problem pb;
+  TcPlan plan;
+  int slot = 0;
+  const int32_t* budgets = nullptr;
+  void* k_out = nullptr;
+  void* v_out = nullptr;
+  int64_t capacity = 0;
+  int32_t* offsets = nullptr;
+  int32_t* kept_idx = nullptr;
+  float* pooled_opt = nullptr;
+  int32_t* status = nullptr;
+  cudaStream_t st = nullptr;
+};
+struct ShapeSig {                                  // calls in flight together must carve the workspace alike
+  const void* ws = nullptr;
+  size_t ws_bytes = 0;
+  int n_seqs = 0, n_kv_heads = 0, R = 0, max_hist = 0, path = 0;
+  int64_t total_hist = 0, total_tokens = 0;
+  bool operator==(const ShapeSig& o) const {
+    return ws == o.ws && ws_bytes == o.ws_bytes && n_seqs == o.n_seqs && n_kv_heads == o.n_kv_heads && R == o.R &&
+           max_hist == o.max_hist && path == o.path && total_hist == o.total_hist && total_tokens == o.total_tokens;
+  }
+};
 struct OverlapState {
-  cudaStream_t side_select = nullptr, side_gather = nullptr;
-  cudaEvent_t scored[2] = {nullptr, nullptr};     // recorded on the caller's stream after the vote pass
-  cudaEvent_t selected[2] = {nullptr, nullptr};   // recorded on the selection stream after the selection
-  cudaEvent_t done[2] = {nullptr, nullptr};       // recorded on the gather stream after the gather
-  bool in_flight[2] = {false, false};
+  cudaStream_t side_select[2] = {nullptr, nullptr}, side_gather = nullptr;
+  cudaEvent_t scored[kSlots] = {};       // recorded on the caller's stream after the vote pass of the slot's layer
+  cudaEvent_t selected[kSlots] = {};     // recorded on a selection stream after the selection
+  cudaEvent_t done[kSlots] = {};         // recorded on the gather stream after the gather
+  bool in_flight[kSlots] = {};
   unsigned seq = 0;
+  PendingCall pending;
+  ShapeSig sig;
 };
 constexpr int kMaxDevices = 64;
 OverlapState g_overlap[kMaxDevices];
 std::mutex g_overlap_mu;
-constexpr int kSelectSmReserve = 16;              // SMs left to the selection kernel of the previous call
+constexpr int kSelectSmReserve = 16;              // SMs left to the selection kernels of the layers before
 
 cudaError_t overlap_state(OverlapState** out) {
   int dev = 0;
@@ -200,12 +241,14 @@ cudaError_t overlap_state(OverlapState** out) {
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   OverlapState& s = g_overlap[dev];
-  if (!s.side_select) {
-    e = cudaStreamCreateWithFlags(&s.side_select, cudaStreamNonBlocking);
-    if (e != cudaSuccess) return e;
+  if (!s.side_gather) {
+    for (int i = 0; i < 2; ++i) {
+      e = cudaStreamCreateWithFlags(&s.side_select[i], cudaStreamNonBlocking);
+      if (e != cudaSuccess) return e;
+    }
     e = cudaStreamCreateWithFlags(&s.side_gather, cudaStreamNonBlocking);
     if (e != cudaSuccess) return e;
-    for (int h = 0; h < 2; ++h) {
+    for (int h = 0; h < kSlots; ++h) {
       e = cudaEventCreateWithFlags(&s.scored[h], cudaEventDisableTiming);
       if (e != cudaSuccess) return e;
       e = cudaEventCreateWithFlags(&s.selected[h], cudaEventDisableTiming);
@@ -218,6 +261,46 @@ cudaError_t overlap_state(OverlapState** out) {
   return cudaSuccess;
 }
 
+// Before a layer takes a slot: its vote array may still be read by the selection of the layer that had the slot,
+// its source-row list by that layer's gather.
+cudaError_t claim_slot(OverlapState* os, int slot, cudaStream_t st) {
+  if (!os->in_flight[slot]) return cudaSuccess;
+  cudaError_t e = cudaStreamWaitEvent(st, os->selected[slot], 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_select[slot & 1], os->done[slot], 0);
+  return e;
+}
+
+// The votes of layer `c` are enqueued on c.st: selection on a side stream, gather on another.
+cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pipe, int* launches) {
+  const int slot = c.slot;
+  cudaStream_t sel = os->side_select[slot & 1];
+  cudaError_t e = cudaEventRecord(os->scored[slot], c.st);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(sel, os->scored[slot], 0);
+  if (e != cudaSuccess) return e;
+  e = launch_select_cta(c.pb, c.pooled_opt, c.budgets, c.offsets, c.kept_idx, c.capacity, c.status, sel, launches);
+  if (e != cudaSuccess) return e;
+  e = cudaEventRecord(os->selected[slot], sel);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_gather, os->selected[slot], 0);
+  if (e != cudaSuccess) return e;
+  // beside the two-layer score kernel an SM has registers left for one 128-thread gather CTA
+  e = launch_gather(c.pb, c.offsets, c.kept_idx, c.k_out, c.v_out, c.capacity, os->side_gather, launches,
+                    beside_pipe ? 128 : 256);
+  if (e != cudaSuccess) return e;
+  e = cudaEventRecord(os->done[slot], os->side_gather);
+  if (e != cudaSuccess) return e;
+  os->in_flight[slot] = true;
+  return cudaSuccess;
+}
+
+// Pass 2, selection and gather of the pending layer (no layer after it yet).
+cudaError_t flush_pending(OverlapState* os, int* launches) {
+  if (!os->pending.valid) return cudaSuccess;
+  cudaError_t e = launch_score_pipe(nullptr, &os->pending.plan, os->pending.st, launches);
+  if (e == cudaSuccess) e = enqueue_tail(os, os->pending, true, launches);
+  os->pending.valid = false;
+  return e;
+}
+
 // Makes `st` wait for every overlapped call still in flight on this device (no host wait).
 cudaError_t join_overlapped(cudaStream_t st) {
   int dev = 0;
@@ -226,7 +309,11 @@ cudaError_t join_overlapped(cudaStream_t st) {
   if (dev < 0 || dev >= kMaxDevices) return cudaSuccess;
   std::lock_guard<std::mutex> lock(g_overlap_mu);
   OverlapState& s = g_overlap[dev];
-  for (int h = 0; h < 2; ++h)
+  int launches = 0;
+  e = flush_pending(&s, &launches);
+  g_last_launches += launches;
+  if (e != cudaSuccess) return e;
+  for (int h = 0; h < kSlots; ++h)
     if (s.in_flight[h]) {
       e = cudaStreamWaitEvent(st, s.done[h], 0);
       if (e != cudaSuccess) return e;
@@ -268,39 +355,60 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
     OverlapState* os = nullptr;
     e = overlap_state(&os);
     if (e != cudaSuccess) return cuda_fail(e);
-    const int half = (int)(os->seq & 1u);
-    rc = bind_workspace(&pb, ws, ws_bytes, path, true, half);
+    ShapeSig sig;
+    sig.ws = ws; sig.ws_bytes = ws_bytes; sig.n_seqs = pb.p.n_seqs; sig.n_kv_heads = pb.p.n_kv_heads; sig.R = pb.R;
+    sig.max_hist = pb.max_hist; sig.path = path; sig.total_hist = pb.total_hist; sig.total_tokens = pb.total_tokens;
+    if (!(sig == os->sig)) {
+      // another shape or workspace: the carve-up changes, so nothing of the old one may still be in flight
+      e = flush_pending(os, &launches);
+      for (int h = 0; h < kSlots && e == cudaSuccess; ++h)
+        if (os->in_flight[h]) {
+          e = cudaStreamWaitEvent(st, os->done[h], 0);
+          os->in_flight[h] = false;
+        }
+      if (e != cudaSuccess) return cuda_fail(e);
+      os->sig = sig;
+    }
+    const int slot = (int)(os->seq % kSlots), part = (int)(os->seq & 1u);
+    rc = bind_workspace(&pb, ws, ws_bytes, path, true, slot, part);
     if (rc != SLKV_OK) return rc;
     ++os->seq;
     pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
     pb.tab.cu_ptr = cu_dev;
-    // the score kernels leave a few SMs to the selection kernel of the call before this one
+    // the score kernels leave a few SMs to the selection kernels of the layers before this one
     int sms = 148;
     int dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int reserve = pb.n_seg < kSelectSmReserve ? pb.n_seg : kSelectSmReserve;
     pb.max_score_ctas = sms - reserve > 0 ? sms - reserve : 0;
-    if (os->in_flight[half]) {                     // the vote array of this half is read by the selection two calls
-      e = cudaStreamWaitEvent(st, os->selected[half], 0);          // back, its source-row list by that call's gather
-      if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_select, os->done[half], 0);
+    PendingCall cur;
+    cur.valid = true; cur.pb = pb; cur.slot = slot; cur.budgets = budgets; cur.k_out = k_out; cur.v_out = v_out;
+    cur.capacity = capacity; cur.offsets = offsets; cur.kept_idx = kept_idx; cur.pooled_opt = pooled_opt;
+    cur.status = status; cur.st = st;
+    const bool pipe = path == SLKV_PATH_TENSOR && score_pipe_supported(pb);
+    if (os->pending.valid && (!pipe || os->pending.st != st)) {
+      e = flush_pending(os, &launches);
       if (e != cudaSuccess) return cuda_fail(e);
     }
-    rc = enqueue_votes(pb, path, cu_host, status, st, &launches);
-    if (rc != SLKV_OK) return rc;
-    // selection on one side stream, gather on another: the gather of a call runs beside the selection of the next
-    e = cudaEventRecord(os->scored[half], st);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_select, os->scored[half], 0);
+    e = claim_slot(os, slot, st);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_select_cta(pb, pooled_opt, budgets, offsets, kept_idx, capacity, status, os->side_select, &launches);
-    if (e != cudaSuccess) return cuda_fail(e);
-    e = cudaEventRecord(os->selected[half], os->side_select);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_gather, os->selected[half], 0);
-    if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_gather(pb, offsets, kept_idx, k_out, v_out, capacity, os->side_gather, &launches);
-    if (e != cudaSuccess) return cuda_fail(e);
-    e = cudaEventRecord(os->done[half], os->side_gather);
-    if (e != cudaSuccess) return cuda_fail(e);
-    os->in_flight[half] = true;
+    if (pipe) {
+      // pass 1 of this layer beside pass 2 of the layer before; this layer's votes come with the next call
+      e = plan_score_tensor(pb, cu_host, status, &cur.plan);
+      if (e != cudaSuccess) return cuda_fail(e);
+      e = launch_score_pipe(&cur.plan, os->pending.valid ? &os->pending.plan : nullptr, st, &launches);
+      if (e != cudaSuccess) return cuda_fail(e);
+      if (os->pending.valid) {
+        e = enqueue_tail(os, os->pending, true, &launches);
+        if (e != cudaSuccess) return cuda_fail(e);
+      }
+      os->pending = cur;
+    } else {
+      rc = enqueue_votes(pb, path, cu_host, status, st, &launches);
+      if (rc != SLKV_OK) return rc;
+      e = enqueue_tail(os, cur, false, &launches);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
     g_last_launches = launches;
     return SLKV_OK;
   }
@@ -397,7 +505,7 @@ int slkv_profile_collect(float* total_ms, int32_t* launches, int32_t n_kernels) 
 
 const char* slkv_kernel_name(int kernel_id) {
   static const char* names[KID_COUNT] = {"k_setup", "k_score_lse", "k_score_vote", "k_pool", "k_select",
-                                         "k_gather", "k_alloc", "k_score_fused"};
+                                         "k_gather", "k_alloc", "k_score_fused", "k_score_pipe"};
   return (kernel_id >= 0 && kernel_id < KID_COUNT) ? names[kernel_id] : "";
 }
 

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -96,7 +97,7 @@ struct Problem {
 };
 
 // kernel ids for launch accounting / per-kernel timing
-enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_COUNT };
+enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_SCORE_PIPE, KID_COUNT };
 
 // Brackets one kernel launch: counts it and, when per-kernel timing is on for this thread, records a
 // CUDA event pair around it on the launch stream.
@@ -129,7 +130,37 @@ bool select_cluster_supported(const Problem& pb);
 cudaError_t launch_select_cluster(const Problem& pb, float* pooled_out, const int32_t* budgets, int32_t* offsets,
                                   int32_t* kept_idx, int64_t capacity, int32_t* status, cudaStream_t st,
                                   int* launches);
+// block_threads: 256, or 128 where the gather shares its SMs with a kernel that leaves few registers
 cudaError_t launch_gather(const Problem& pb, const int32_t* offsets, const int32_t* kept_idx, void* k_out,
-                          void* v_out, int64_t capacity, cudaStream_t st, int* launches);
+                          void* v_out, int64_t capacity, cudaStream_t st, int* launches, int block_threads = 256);
+
+// ---- tensor-core score kernels: arguments and launch plans ---------------------------------------------------
+struct TcArgs {
+  SeqTables tab;
+  float* part_m;
+  float* part_z;
+  float* vote;
+  int32_t* status;
+  unsigned long long* trace;    // optional timeline buffer: kTraceSlots timestamps (ns) per CTA, or null
+  int n_seqs, n_kv_heads, G, window, R, MT, n_stages, slot_stride, tiles_per_cta, total_tiles, barrier_slot;
+  int q_head_inner, k_head_inner;   // tensor-map dimension order: 1 = the head axis comes before the row axis
+  float scale_log2;
+};
+
+// One layer's score problem, ready to launch: tensor maps of Q_win and K, kernel arguments, grid size.
+struct TcPlan {
+  CUtensorMap tm_q, tm_k;
+  TcArgs a;
+  int n_cta;
+};
+// Fills a plan (tensor maps, schedule, arguments) for a problem whose workspace is bound; n_cta = 0 when there is
+// no history to score.  cudaErrorNotSupported when the driver has no tensor-map encoder.
+cudaError_t plan_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, TcPlan* plan);
+// Timeline buffer of this thread (diagnostics), or null: half 0 / 1, kTraceSlots words per CTA.
+unsigned long long* tensor_trace_buffer(int half, int n_cta);
+
+// Two layers per launch: pass 1 of plan `a` beside pass 2 of plan `b` (either may be null).  The shapes it takes:
+bool score_pipe_supported(const Problem& pb);
+cudaError_t launch_score_pipe(const TcPlan* a, const TcPlan* b, cudaStream_t st, int* launches);
 
 }  // namespace slkv

@@ -17,232 +17,10 @@
 #include <atomic>
 
 #include "slkv_internal.cuh"
+#include "slkv_tc_device.cuh"
 
 namespace slkv {
 namespace {
-
-constexpr int kTileKeys = 128;                 // keys per tile (MMA N in pass 1, M in pass 2)
-constexpr int kMaxStages = 6;                  // K tiles in flight in shared memory (as many as fit beside Q)
-constexpr int kHalfBytes = kTileKeys * 128;    // one 64-element (128-byte) half of a 128-row tile
-constexpr int kStageBytes = 2 * kHalfBytes;    // 32 KB
-constexpr int kTailBytes = 512 + 2048;         // mbarriers + flags, then 512 floats of row statistics
-constexpr int kSmemLimit = 227 * 1024;         // dynamic shared memory a CTA can have
-constexpr int kThreads = 384;                  // warps 0-3: TMA, MMA, 2 idle; warps 4-11: epilogue
-constexpr int kEpiThreads = 256;
-constexpr int kTraceSlots = 64;               // per CTA: 0 start, 1 set-up done, 2 Q landed, 3 first K landed,
-                                               // 4 end; 5 / 6 grid barrier reached / passed, 7 first log-sum-exp merged; 8+2i / 9+2i = epilogue of the
-                                               // CTA's i-th tile begins / ends
-constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per wait
-
-struct TcArgs {
-  SeqTables tab;
-  float* part_m;
-  float* part_z;
-  float* vote;
-  int32_t* status;
-  unsigned long long* trace;    // optional timeline buffer: kTraceSlots timestamps (ns) per CTA, or null
-  int n_seqs, n_kv_heads, G, window, R, MT, n_stages, slot_stride, tiles_per_cta, total_tiles, barrier_slot;
-  int q_head_inner, k_head_inner;   // tensor-map dimension order: 1 = the head axis comes before the row axis
-  float scale_log2;
-};
-
-// ---- PTX wrappers -------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity), "r"(100u) : "memory");    // may sleep up to 0.1 us: a waiting thread must
-                                                                   // not eat the issue slots of the epilogue warps
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long now_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void trace_mark(const unsigned long long* base, int slot) {
-  if (base) const_cast<unsigned long long*>(base)[(size_t)blockIdx.x * kTraceSlots + slot] = now_ns();
-}
-// Waits for the phase with the given parity.  false = gave up (limit reached or another thread did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  const unsigned long long t0 = now_ns();
-  for (unsigned it = 1;; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    if ((it & 63u) == 0) {
-      if (*abort_flag) return false;
-      if (now_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, int w,
-                                            uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// 2^x on the FMA and integer pipes instead of the special-function unit, which is the busiest pipe of both
-// passes (one exponential per query row and key): x = n + f with n = round(x), 2^f by a degree-4 minimax
-// polynomial on [-0.5, 0.5] (relative error 2.7e-6 in fp32 Horner form), n added into the exponent field.
-// x is clamped to [-125, 128.5]: below, the result is 2^-125 at most (negligible in any sum that holds a term
-// near 1); above, the exponent field overflows to Inf/NaN, which the caller's overflow check catches.
-// One exponential in four goes this way; the split balances the pipes' issue slots.
-__device__ __forceinline__ float ex2_fma(float x, bool clamp_hi) {
-  x = fmaxf(x, -125.f);
-  if (clamp_hi) x = fminf(x, 128.5f);
-  const float t = x + 12582912.f;                    // 1.5 * 2^23: round(x) lands in the low mantissa bits
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(0.009570101276040077f, f, 0.05591785907745361f);
-  p = fmaf(p, f, 0.240247443318367f);
-  p = fmaf(p, f, 0.6931217908859253f);
-  p = fmaf(p, f, 0.9999992847442627f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
-// Issues a TMEM load of 32 consecutive columns of this thread's lane; the registers are valid only after
-// tc_ld_wait on the same array.
-__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-// Waits for this thread's outstanding TMEM loads; naming the registers keeps their uses behind the wait.
-__device__ __forceinline__ void tc_ld_wait(uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.wait::ld.sync.aligned;"
-      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
-        "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
-        "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
-        "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-      :: "memory");
-}
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
-
-// K-major, 128-byte-swizzled operand: rows 128 bytes apart, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-// D fp32, A and B bf16, both K-major, M x N tile
-__device__ __forceinline__ uint32_t instr_desc(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-struct Run { int s, g, t0, count, n_hist, seg_tile0, tiles_seg; };
-
-// A run = consecutive tiles of one segment inside the CTA's range [begin, end).  Forward walks (pass 1)
-// name a run by its first tile, backward walks (pass 2) by its last one.
-__device__ __forceinline__ Run locate(const TcArgs& a, int pos, int begin, int end, bool REV) {
-  int lo = 0, hi = a.n_seqs;                       // last s with Hkv*tile_off[s] <= pos
-  while (hi - lo > 1) {
-    int mid = (lo + hi) >> 1;
-    if (a.n_kv_heads * a.tab.tile_at(mid) <= pos) lo = mid; else hi = mid;
-  }
-  Run r;
-  r.s = lo;
-  r.tiles_seg = a.tab.tile_at(lo + 1) - a.tab.tile_at(lo);
-  const int rel = pos - a.n_kv_heads * a.tab.tile_at(lo);
-  r.g = rel / r.tiles_seg;
-  const int t = rel - r.g * r.tiles_seg;
-  r.seg_tile0 = pos - t;
-  if (REV) {
-    r.t0 = max(r.seg_tile0, begin) - r.seg_tile0;
-    r.count = t - r.t0 + 1;
-  } else {
-    r.t0 = t;
-    r.count = min(end - pos, r.tiles_seg - t);
-  }
-  r.n_hist = max(a.tab.cu_at(lo + 1) - a.tab.cu_at(lo) - a.window, 0);
-  return r;
-}
-
-// sum_e 2^(v_e * sc - m) over 32 accumulator values, four independent chains
-__device__ __forceinline__ float sum_ex2_32(const uint32_t (&r)[32], float sc, float m) {
-  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-  for (int e = 0; e < 32; e += 4) {
-    s0 += ex2(fmaf(__uint_as_float(r[e]), sc, -m));
-    s1 += ex2(fmaf(__uint_as_float(r[e + 1]), sc, -m));
-    s2 += ex2(fmaf(__uint_as_float(r[e + 2]), sc, -m));
-    s3 += ex2_fma(fmaf(__uint_as_float(r[e + 3]), sc, -m), true);
-  }
-  return (s0 + s1) + (s2 + s3);
-}
-__device__ __forceinline__ float max_32(const uint32_t (&r)[32], int n_valid_here) {
-  float t[32];
-#pragma unroll
-  for (int e = 0; e < 32; ++e) t[e] = e < n_valid_here ? __uint_as_float(r[e]) : -INFINITY;
-#pragma unroll
-  for (int w = 16; w >= 1; w >>= 1)
-#pragma unroll
-    for (int e = 0; e < w; ++e) t[e] = fmaxf(t[e], t[e + w]);
-  return t[0];
-}
-
-// Pass 1, exact path for one 128-row accumulator: running maximum and rescaled sum over the tile's first n_valid
-// keys.  Used for a segment's ragged last tile and when the fast path over- or underflows.  A function of its
-// own (not inlined) so that a CTA which will need it can run it once before the K stream starts: fetching
-// these instructions for the first time while the stream saturates the memory system stalled the tile for
-// microseconds.
-__device__ __noinline__ void tile_row_stats_exact(uint32_t tcol, float sc, int n_valid, float& m_io, float& z_io) {
-  uint32_t ra[32];
-  float m = m_io, z = z_io;
-#pragma unroll 1
-  for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
-    if (c0 >= n_valid) break;
-    tc_ld32_issue(tcol + c0, ra);
-    tc_ld_wait(ra);
-    const float mn = fmaxf(m, max_32(ra, n_valid - c0) * sc);
-    z *= ex2(m - mn);
-    m = mn;
-    float zc = 0.f;
-#pragma unroll
-    for (int e = 0; e < 32; ++e)
-      if (e < n_valid - c0) zc += ex2(fmaf(__uint_as_float(ra[e]), sc, -m));
-    z += zc;
-  }
-  m_io = m; z_io = z;
-}
 
 // Grid-wide barrier of the fused kernel (both passes in one launch): one arrival counter per launch, taken in
 // turn from a small table in the module's globals (zero at load).  atom.inc wraps the counter back to zero with
@@ -732,20 +510,22 @@ bool tensor_path_supported(const slkv_params& p) {
 
 int tensor_slot_stride(const Problem& pb) { return (pb.max_hist + kTileKeys - 1) / kTileKeys + 2; }
 
-cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, cudaStream_t st,
-                                int* launches) {
+cudaError_t plan_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, TcPlan* plan) {
+  plan->n_cta = 0;
   if (pb.max_hist <= 0) return cudaSuccess;
   EncodeTiledFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
   const slkv_params& p = pb.p;
   const Schedule sc = schedule_of(pb, cu_host);
   if (sc.n_cta == 0) return cudaSuccess;
+  CUtensorMap& tm_q = plan->tm_q;
+  CUtensorMap& tm_k = plan->tm_k;
+  TcArgs& a = plan->a;
 
   // Tensor-map dimensions go from the smallest stride to the largest.  The order of the G*w query rows
   // inside the Q tile follows from it (head-fastest or window-row-fastest); the scores do not depend on it.
   const int q_head_inner = p.q_stride_head <= p.q_stride_row;
   const int k_head_inner = p.k_stride_head <= p.k_stride_tok;
-  CUtensorMap tm_q, tm_k;
   {
     cuuint64_t dims[4] = {(cuuint64_t)p.head_dim, (cuuint64_t)p.window, (cuuint64_t)p.n_q_heads, (cuuint64_t)p.n_seqs};
     cuuint64_t strides[3] = {(cuuint64_t)p.q_stride_row * 2, (cuuint64_t)p.q_stride_head * 2, (cuuint64_t)p.q_stride_seq * 2};
@@ -777,7 +557,6 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
       return cudaErrorInvalidValue;
   }
 
-  TcArgs a;
   a.tab = pb.tab;
   a.part_m = pb.part_m; a.part_z = pb.part_z; a.vote = pb.vote; a.status = status;
   a.trace = nullptr;
@@ -792,6 +571,22 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
   const size_t q_bytes = (size_t)a.MT * 2 * 128 * 128;
   a.n_stages = (int)((kSmemLimit - kTailBytes - q_bytes) / kStageBytes);
   if (a.n_stages > kMaxStages) a.n_stages = kMaxStages;
+  plan->n_cta = sc.n_cta;
+  return cudaSuccess;
+}
+
+unsigned long long* tensor_trace_buffer(int half, int n_cta) { return trace_buffer(half + 1, n_cta); }
+
+cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, cudaStream_t st,
+                                int* launches) {
+  TcPlan plan;
+  cudaError_t pe = plan_score_tensor(pb, cu_host, status, &plan);
+  if (pe != cudaSuccess || plan.n_cta == 0) return pe;
+  const CUtensorMap& tm_q = plan.tm_q;
+  const CUtensorMap& tm_k = plan.tm_k;
+  TcArgs& a = plan.a;
+  struct { int n_cta; } sc = {plan.n_cta};
+  const size_t q_bytes = (size_t)a.MT * 2 * 128 * 128;
   const size_t smem = q_bytes + (size_t)a.n_stages * kStageBytes + kTailBytes;
   static thread_local int configured_dev = -1;
   int dev = 0;

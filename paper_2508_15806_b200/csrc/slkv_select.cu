@@ -244,17 +244,19 @@ cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t*
 }
 
 cudaError_t launch_gather(const Problem& pb, const int32_t* offsets, const int32_t* kept_idx, void* k_out,
-                          void* v_out, int64_t capacity, cudaStream_t st, int* launches) {
+                          void* v_out, int64_t capacity, cudaStream_t st, int* launches, int block_threads) {
   (void)kept_idx;
   const int row_bytes = pb.p.head_dim * pb.elem;
-  const int rows_per_cta = 256 / (row_bytes >> 4);
+  if (block_threads != 128) block_threads = 256;
+  const int rows_per_cta = block_threads / (row_bytes >> 4);
   long long max_rows = (long long)pb.p.n_kv_heads * pb.total_tokens;
   if (capacity < max_rows) max_rows = capacity;
   if (max_rows <= 0) return cudaSuccess;
   long long want = (max_rows + rows_per_cta - 1) / rows_per_cta;
-  int grid = (int)(want < 148 * 8 ? want : 148 * 8);
+  const int max_grid = 148 * 8 * (256 / block_threads);
+  int grid = (int)(want < max_grid ? want : max_grid);
   LaunchScope scope(KID_GATHER, st, launches);
-  return launch_pdl(k_gather, dim3(grid), dim3(256), 0, st, 1, (const unsigned char*)pb.k,
+  return launch_pdl(k_gather, dim3(grid), dim3(block_threads), 0, st, 1, (const unsigned char*)pb.k,
                     (const unsigned char*)pb.v, (unsigned char*)k_out, (unsigned char*)v_out, offsets,
                     (const int32_t*)pb.gather_src, pb.n_seg, pb.p.n_kv_heads, row_bytes,
                     (long long)(pb.p.k_stride_tok * pb.elem), (long long)(pb.p.k_stride_head * pb.elem),
