@@ -149,29 +149,47 @@ __device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& 
       ok = __all_sync(0xffffffffu, ok) != 0;                  // the TMEM loads below need the whole warp
       if (!ok) continue;
       tc_fence_after();
+      if (et == 0 && it == 0) trace_mark(a.trace, 2);
       const int key0 = (r.t0 + i) * kTileKeys;
       const int n_valid = min(r.n_hist - key0, kTileKeys);
       const uint32_t tcol = c.tmem0 + lane_sel + (uint32_t)(b * 128);
-      bool exact = n_valid < kTileKeys;
-      if (!exact) {
-        uint32_t ra[32], rb[32];
-        float zt = z;
-        tc_ld32_issue(tcol, ra);
-#pragma unroll 1
-        for (int c0 = 0; c0 < kTileKeys; c0 += 64) {
-          tc_ld_wait(ra);
-          tc_ld32_issue(tcol + c0 + 32, rb);
-          zt += sum_ex2_32(ra, sc, m);
-          tc_ld_wait(rb);
-          if (c0 + 64 < kTileKeys) tc_ld32_issue(tcol + c0 + 64, ra);
-          zt += sum_ex2_32(rb, sc, m);
+      // A fixed reference m per row (0 until a fallback moves it) instead of a running maximum: any reference gives
+      // the same log-sum-exp as long as nothing overflows and not everything underflows.  A chunk whose sum is not
+      // finite and positive is redone exactly from the registers, which moves the reference.  Keys past the
+      // segment's end (its ragged last tile) are left out chunk by chunk.
+      uint32_t ra[32], rb[32];
+      auto add_chunk = [&](const uint32_t (&rr)[32], int nv) {
+        if (nv >= 32) {
+          const float zc = sum_ex2_32(rr, sc, m);
+          const float zn = z + zc;
+          if (zn < INFINITY && zc > 0.f) { z = zn; return; }
         }
-        if (zt < INFINITY && zt > 0.f) z = zt; else exact = true;
+        // rare: a copy goes through the stack so that the chunk registers themselves never have to
+        uint32_t tmp[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) tmp[e] = rr[e];
+        chunk_stats_exact(tmp, sc, nv < 32 ? nv : 32, m, z);
+      };
+      tc_ld32_issue(tcol, ra);
+#pragma unroll 1
+      for (int c0 = 0; c0 < kTileKeys; c0 += 64) {
+        const bool last = c0 + 64 >= kTileKeys;
+        tc_ld_wait(ra);
+        tc_ld32_issue(tcol + c0 + 32, rb);
+        if (last) {
+          // the whole accumulator is in registers (or on its way): hand the TMEM buffer back before the arithmetic
+          tc_ld_wait(rb);
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(c.acce_bar(b));
+        }
+        add_chunk(ra, n_valid - c0);
+        if (!last) {
+          tc_ld_wait(rb);
+          tc_ld32_issue(tcol + c0 + 64, ra);
+        }
+        add_chunk(rb, n_valid - c0 - 32);
       }
-      if (exact) tile_row_stats_exact(tcol, sc, n_valid, m, z);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(c.acce_bar(b));
     }
     // combine the two warpgroups' statistics and publish this CTA's partial for the segment
     const int slot = blockIdx.x - first_cta;
@@ -179,9 +197,11 @@ __device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& 
     named_bar(1);
     if (wg == 0 && row < R) {
       const float m1 = stat_m[row], z1 = stat_z[row];
-      const float M = fmaxf(m, m1);
+      const bool h0 = z > 0.f, h1 = z1 > 0.f;                  // a warpgroup without a tile in this run has z = 0
+      const float M = h0 && h1 ? fmaxf(m, m1) : (h0 ? m : m1);
       float Z = 0.f;
-      if (M > -INFINITY) Z = z * ex2(m - M) + z1 * ex2(m1 - M);
+      if (h0) Z += z * ex2(m - M);
+      if (h1) Z += z1 * ex2(m1 - M);
       a.part_m[((long long)seg * a.slot_stride + slot) * R + row] = M;
       a.part_z[((long long)seg * a.slot_stride + slot) * R + row] = Z;
     }
@@ -239,7 +259,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
           }
 #pragma unroll
           for (int u = 0; u < 12; ++u)
-            if (m12[u] > -INFINITY) {
+            if (z12[u] > 0.f) {                                       // empty partials carry z = 0
               const float Mn = fmaxf(M, m12[u]);
               Z = Z * ex2(M - Mn) + z12[u] * ex2(m12[u] - Mn);      // ex2(-inf) = 0 covers the first term
               M = Mn;
@@ -254,6 +274,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
       if (half == 0 && rr >= 0) lse[rr] = Mn + log2f(Zt);
     }
     named_bar(2);
+    if (et == 0 && run_idx == 0) trace_mark(a.trace, 3);
     for (int i = 0; i < r.count; ++i, ++it) {
       if ((it & 1) != wg) continue;
       const int b = it & 1;
@@ -265,22 +286,25 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
       const uint32_t tb = c.tmem0 + lane_sel + (uint32_t)(b * 128);
       uint32_t ra[32], rb[32];
       float acc = 0.f;
+      auto release = [&]() {
+        // the accumulator is in registers: hand its TMEM buffer back before the arithmetic and the vote's store
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(c.acce_bar(b));
+      };
       tc_ld32_issue(tb, ra);
 #pragma unroll 1
       for (int c0 = 0; c0 < R; c0 += 64) {
         tc_ld_wait(ra);
         if (c0 + 32 < R) tc_ld32_issue(tb + c0 + 32, rb);
+        if (c0 + 32 >= R) release();
+        else if (c0 + 64 >= R) { tc_ld_wait(rb); release(); }
         acc += vote_chunk(ra, sc, lse + c0);
         if (c0 + 32 < R) {
-          tc_ld_wait(rb);
-          if (c0 + 64 < R) tc_ld32_issue(tb + c0 + 64, ra);
+          if (c0 + 64 < R) { tc_ld_wait(rb); tc_ld32_issue(tb + c0 + 64, ra); }
           acc += vote_chunk(rb, sc, lse + c0 + 32);
         }
       }
-      // The accumulator is in registers now: hand its TMEM buffer back before the vote leaves for global memory.
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(c.acce_bar(b));
       const int j = key0 + row;
       if (j < r.n_hist) a.vote[a.tab.hist_at(r.s) * a.n_kv_heads + (long long)r.g * r.n_hist + j] = acc * inv_g;
     }
@@ -375,24 +399,15 @@ k_score_pipe(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ 
     if (lane == 0 && has_b) issuer<true>(cb, pa.b);
   } else if (warp < 12) {
     if (has_a) {
-      bool ragged = false;                                            // a segment's ragged last tile in this CTA's range?
-      for (int pos = ca.begin; pos < ca.end;) {
-        const Run r = locate(pa.a, pos, ca.begin, ca.end, false);
-        ragged |= r.t0 + r.count == r.tiles_seg && (r.n_hist & (kTileKeys - 1)) != 0;
-        pos += r.count;
-      }
-      if (ragged) {                                                   // instruction-cache warm-up, results unused
-        float mw = 0.f, zw = 0.f;
-        tile_row_stats_exact(ca.tmem0 + ((uint32_t)((warp & 3) * 32) << 16), 0.f, kTileKeys - 1, mw, zw);
-        if (zw == 12345.f) abort_sh = 0;                              // keeps the call alive; writes what is there
-      }
       pdl_wait();
+      if (tid == 128) trace_mark(trace, 1);
       epilogue_rows(ca, pa.a, tid - 128, warp, stat_m, stat_z);
       if (tid == 128) trace_mark(trace, 5);
     }
   } else {
     if (has_b) {
       pdl_wait();
+      if (tid == 384) trace_mark(trace, 7);
       epilogue_votes(cb, pa.b, tid - 384, warp, lse2);
       if (tid == 384) trace_mark(trace, 6);
     }

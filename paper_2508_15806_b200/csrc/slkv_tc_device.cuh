@@ -20,7 +20,9 @@ constexpr int kThreads = 384;                  // warps 0-3: TMA, MMA, 2 idle; w
 constexpr int kEpiThreads = 256;
 constexpr int kTraceSlots = 64;               // per CTA: 0 start, 1 set-up done, 2 Q landed, 3 first K landed,
                                                // 4 end; 5 / 6 grid barrier reached / passed, 7 first log-sum-exp merged; 8+2i / 9+2i = epilogue of the
-                                               // CTA's i-th tile begins / ends
+                                               // CTA's i-th tile begins / ends.  Two-layer kernel: 0 start, 1 / 7 stream A / B
+                                               // past its wait for the launch before, 2 first accumulator of A ready,
+                                               // 3 first log-sum-exps of B merged, 5 / 6 epilogue of A / B done, 4 end
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per wait
 
 
@@ -185,6 +187,22 @@ __device__ __forceinline__ float sum_ex2_32(const uint32_t (&r)[32], float sc, f
     s3 += ex2_fma(fmaf(__uint_as_float(r[e + 3]), sc, -m), true);
   }
   return (s0 + s1) + (s2 + s3);
+}
+// Adds one chunk of 32 accumulator values (the first nv of them) to a row's (reference m, sum z) pair exactly:
+// the reference moves to the running maximum and the sum is rescaled.  Taken when the fixed-reference sum of the
+// chunk over- or underflowed; works on the registers, so the accumulator may already be back with the tensor pipe.
+__device__ __noinline__ void chunk_stats_exact(const uint32_t (&r)[32], float sc, int nv, float& m_io, float& z_io) {
+  float mx = -INFINITY;
+#pragma unroll
+  for (int e = 0; e < 32; ++e)
+    if (e < nv) mx = fmaxf(mx, __uint_as_float(r[e]) * sc);
+  if (!(mx > -INFINITY)) return;                       // nothing valid (or only -inf scores)
+  const float m_new = z_io > 0.f ? fmaxf(m_io, mx) : mx;
+  float z = z_io > 0.f ? z_io * ex2(m_io - m_new) : 0.f;
+#pragma unroll
+  for (int e = 0; e < 32; ++e)
+    if (e < nv) z += ex2(fmaf(__uint_as_float(r[e]), sc, -m_new));
+  m_io = m_new; z_io = z;
 }
 __device__ __forceinline__ float max_32(const uint32_t (&r)[32], int n_valid_here) {
   float t[32];
