@@ -199,7 +199,7 @@ def run_cuda(args):
                  L["offsets"], L["kept"], ws, None, status, stream)
             n += B.slkv_last_launch_count()
         B.slkv_join(stream)
-        launches_per_step = n
+        launches_per_step = n + B.slkv_last_launch_count()
 
     def barrier():
         torch.cuda.synchronize()
@@ -222,6 +222,26 @@ def run_cuda(args):
         step()
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "device status word set during warm-up"
+    eager_step = step
+    if args.graph:
+        # The calls of a step are stream-ordered and allocate nothing: capture them once (the side streams of the
+        # overlapped calls fork from and rejoin the captured stream) and replay the graph per step.
+        cap = torch.cuda.Stream()
+        stream = cap
+        with torch.cuda.stream(cap):
+            eager_step()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=cap):
+            eager_step()
+        stream = torch.cuda.current_stream()
+
+        def step():
+            graph.replay()
+        for _ in range(2):
+            step()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
     steps = args.steps
     if steps is None:                                   # aim at ~3 s of timed work
         one = timed(1, step)
@@ -235,7 +255,7 @@ def run_cuda(args):
     barrier()
     prof_steps = min(steps, 50)
     for _ in range(prof_steps):
-        step()
+        eager_step()
     torch.cuda.synchronize()
     per_kernel = B.slkv_profile_collect()
     B.slkv_profile_enable(False)
@@ -435,6 +455,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="use fewer layers (profiling captures only)")
     ap.add_argument("--workload", type=int, default=0, choices=[0, 1, 2, 3, 4, 5],
                     help="time another of the five workloads (default: the 32k-context one); the others are parity cases")
+    ap.add_argument("--graph", action="store_true", help="capture a step's calls in a CUDA graph and replay it")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="one layer at a time (slkv_compress) instead of overlapped calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -41,8 +41,9 @@ int cuda_fail(cudaError_t e) {
   return SLKV_ERR_CUDA;
 }
 
+constexpr int kLaySlots = 2 * kPipeMaxLayers + 2;   // overlapped calls: layers in flight at once
 struct Layout {
-  size_t hist_off, tile_off, vote[3], pooled, part_m[2], part_z[2], flags, gather_src[3], total;
+  size_t hist_off, tile_off, vote[kLaySlots], pooled, part_m[kLaySlots], part_z[kLaySlots], flags, gather_src[kLaySlots], total;
 };
 
 // Validates p and cu_seqlens_host and fills the host-known fields of `pb`.
@@ -115,27 +116,27 @@ Layout layout_of(const Problem& pb, bool overlapped = false) {
   size_t o = 0;
   L.hist_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int64_t));
   L.tile_off = o; o = align_up(o + (size_t)(pb.p.n_seqs + 1) * sizeof(int32_t));
-  // Overlapped calls keep up to three layers in flight: the votes and the source-row list of a layer are read by
-  // its selection and its gather while the score kernels of the next two layers run; the per-CTA row statistics
-  // live from one launch to the next (two sets).  Ordinary calls use the first of each.
+  // Overlapped calls keep many layers in flight (the score kernel takes a list of layers per launch, selections and
+  // gathers trail behind): each has its own votes, source-row list and per-CTA row statistics.  Ordinary calls use
+  // the first of each.
   const size_t votes = (size_t)pb.p.n_kv_heads * (size_t)pb.total_hist * sizeof(float);
-  const int n_slots = overlapped ? 3 : 1, n_parts = overlapped ? 2 : 1;
-  for (int i = 0; i < 3; ++i) {
+  const int n_slots = overlapped ? kLaySlots : 1;
+  for (int i = 0; i < kLaySlots; ++i) {
     L.vote[i] = i < n_slots ? o : L.vote[0];
     if (i < n_slots) o = align_up(o + votes);
   }
   L.pooled = o; o = align_up(o + votes);
   const size_t nchunks = (size_t)(pb.max_hist + kMinChunkKeys - 1) / kMinChunkKeys + 2;
   const size_t parts = (size_t)pb.n_seg * pb.R * nchunks * sizeof(float);
-  for (int i = 0; i < 2; ++i) {
-    L.part_m[i] = i < n_parts ? o : L.part_m[0];
-    if (i < n_parts) o = align_up(o + parts);
-    L.part_z[i] = i < n_parts ? o : L.part_z[0];
-    if (i < n_parts) o = align_up(o + parts);
+  for (int i = 0; i < kLaySlots; ++i) {
+    L.part_m[i] = i < n_slots ? o : L.part_m[0];
+    if (i < n_slots) o = align_up(o + parts);
+    L.part_z[i] = i < n_slots ? o : L.part_z[0];
+    if (i < n_slots) o = align_up(o + parts);
   }
   L.flags = o; o = align_up(o + 8 * sizeof(int32_t));
   const size_t srcs = (size_t)pb.p.n_kv_heads * (size_t)pb.total_tokens * sizeof(int32_t);
-  for (int i = 0; i < 3; ++i) {
+  for (int i = 0; i < kLaySlots; ++i) {
     L.gather_src[i] = i < n_slots ? o : L.gather_src[0];
     if (i < n_slots) o = align_up(o + srcs);
   }
@@ -154,9 +155,8 @@ int resolve_path(const Problem& pb, int* path) {
   return SLKV_OK;
 }
 
-// slot: which of the three vote arrays / source-row lists (overlapped calls), part: which set of row statistics
-int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overlapped = false, int slot = 0,
-                   int part = 0) {
+// slot: which of the vote arrays / source-row lists / sets of row statistics (overlapped calls)
+int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overlapped = false, int slot = 0) {
   if (!ws) return SLKV_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) % kAlign != 0) return SLKV_ERR_BAD_ALIGN;
   Layout L = layout_of(*pb, overlapped);
@@ -168,8 +168,8 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overla
   pb->tab.hist_ptr = reinterpret_cast<const long long*>(pb->hist_off);
   pb->vote = reinterpret_cast<float*>(b + L.vote[slot]);
   pb->pooled_ws = reinterpret_cast<float*>(b + L.pooled);
-  pb->part_m = reinterpret_cast<float*>(b + L.part_m[part]);
-  pb->part_z = reinterpret_cast<float*>(b + L.part_z[part]);
+  pb->part_m = reinterpret_cast<float*>(b + L.part_m[slot]);
+  pb->part_z = reinterpret_cast<float*>(b + L.part_z[slot]);
   pb->dev_flags = reinterpret_cast<int32_t*>(b + L.flags);
   pb->gather_src = reinterpret_cast<int32_t*>(b + L.gather_src[slot]);
   pb->chunk_keys = path == SLKV_PATH_TENSOR ? 128 : simt_chunk_keys();
@@ -194,7 +194,7 @@ int enqueue_votes(const Problem& pb, int path, const int32_t* cu_host, int32_t* 
 // The selection and the gather of a layer run on side streams while the score kernels of the following layers
 // run on the caller's stream.  Where the two-layer score kernel takes the shape, a call enqueues pass 1 of its
 // own layer together with pass 2 of the layer before (which stays "pending" until the next call or a join).
-constexpr int kSlots = 3;
+constexpr int kSlots = 2 * kPipeMaxLayers + 2;     // layers whose votes / source rows / row statistics are live at once
 struct PendingCall {
   bool valid = false;
   Problem pb;
@@ -227,7 +227,8 @@ struct OverlapState {
   cudaEvent_t done[kSlots] = {};         // recorded on the gather stream after the gather
   bool in_flight[kSlots] = {};
   unsigned seq = 0;
-  PendingCall pending;
+  std::vector<PendingCall> queue;        // layers whose score kernel is not launched yet (at most kPipeMaxLayers + 1)
+  PendingCall pending;                   // pass 1 launched, pass 2 not
   ShapeSig sig;
 };
 constexpr int kMaxDevices = 64;
@@ -292,26 +293,41 @@ cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pip
   return cudaSuccess;
 }
 
-// Pass 2, selection and gather of the pending layer (no layer after it yet).
-cudaError_t flush_pending(OverlapState* os, int* launches) {
-  if (!os->pending.valid) return cudaSuccess;
-  cudaError_t e = launch_score_pipe(nullptr, &os->pending.plan, os->pending.st, launches);
-  if (e == cudaSuccess) e = enqueue_tail(os, os->pending, true, launches);
+// Launches the score kernel for the first n queued layers (pass 1) together with pass 2 of the pending layer and of
+// all but the last of them -- of all of them when `finish` is set -- then the selections and gathers of the
+// layers whose votes that gives.
+cudaError_t launch_queue(OverlapState* os, int n, bool finish, int* launches) {
+  if (n > (int)os->queue.size()) n = (int)os->queue.size();
+  if (n == 0 && !(finish && os->pending.valid)) return cudaSuccess;
+  const TcPlan* plans[kPipeMaxLayers];
+  for (int i = 0; i < n; ++i) plans[i] = &os->queue[i].plan;
+  cudaStream_t st = n > 0 ? os->queue[0].st : os->pending.st;
+  cudaError_t e = launch_score_pipe(os->pending.valid ? &os->pending.plan : nullptr, plans, n, finish, st, launches);
+  if (e == cudaSuccess && os->pending.valid) e = enqueue_tail(os, os->pending, true, launches);
   os->pending.valid = false;
+  const int n_voted = finish ? n : n - 1;
+  for (int i = 0; i < n_voted && e == cudaSuccess; ++i) e = enqueue_tail(os, os->queue[i], true, launches);
+  if (!finish && n > 0) os->pending = os->queue[n - 1];
+  os->queue.erase(os->queue.begin(), os->queue.begin() + n);
+  return e;
+}
+cudaError_t flush_pending(OverlapState* os, int* launches) {
+  cudaError_t e = cudaSuccess;
+  while (!os->queue.empty() && (int)os->queue.size() > kPipeMaxLayers && e == cudaSuccess)
+    e = launch_queue(os, kPipeMaxLayers, false, launches);
+  if (e == cudaSuccess) e = launch_queue(os, (int)os->queue.size(), true, launches);
   return e;
 }
 
 // Makes `st` wait for every overlapped call still in flight on this device (no host wait).
-cudaError_t join_overlapped(cudaStream_t st) {
+cudaError_t join_overlapped(cudaStream_t st, int* launches) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaSuccess;
   std::lock_guard<std::mutex> lock(g_overlap_mu);
   OverlapState& s = g_overlap[dev];
-  int launches = 0;
-  e = flush_pending(&s, &launches);
-  g_last_launches += launches;
+  e = flush_pending(&s, launches);
   if (e != cudaSuccess) return e;
   for (int h = 0; h < kSlots; ++h)
     if (s.in_flight[h]) {
@@ -341,15 +357,15 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
   // pooling, offsets and selection run in one kernel when the segments fit it: one CTA per segment up to
   // 32768 history positions (overlapped calls), a thread-block cluster per segment otherwise
   const bool one_cta = overlapped && select_cta_supported(pb) && pb.tab.n_inline > 0;
+  int launches = 0;
   if (!one_cta) {
     // ordinary call (or shapes the overlapped path does not take): everything on the caller's stream, after
     // whatever overlapped calls are still in flight
-    cudaError_t je = join_overlapped(st);
+    cudaError_t je = join_overlapped(st, &launches);
     if (je != cudaSuccess) return cuda_fail(je);
     overlapped = false;
   }
   cudaError_t e = cudaSuccess;
-  int launches = 0;
   if (overlapped) {
     std::lock_guard<std::mutex> lock(g_overlap_mu);
     OverlapState* os = nullptr;
@@ -369,8 +385,8 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
       if (e != cudaSuccess) return cuda_fail(e);
       os->sig = sig;
     }
-    const int slot = (int)(os->seq % kSlots), part = (int)(os->seq & 1u);
-    rc = bind_workspace(&pb, ws, ws_bytes, path, true, slot, part);
+    const int slot = (int)(os->seq % kSlots);
+    rc = bind_workspace(&pb, ws, ws_bytes, path, true, slot);
     if (rc != SLKV_OK) return rc;
     ++os->seq;
     pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
@@ -385,24 +401,27 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
     cur.valid = true; cur.pb = pb; cur.slot = slot; cur.budgets = budgets; cur.k_out = k_out; cur.v_out = v_out;
     cur.capacity = capacity; cur.offsets = offsets; cur.kept_idx = kept_idx; cur.pooled_opt = pooled_opt;
     cur.status = status; cur.st = st;
-    const bool pipe = path == SLKV_PATH_TENSOR && score_pipe_supported(pb);
-    if (os->pending.valid && (!pipe || os->pending.st != st)) {
+    bool pipe = path == SLKV_PATH_TENSOR && score_pipe_supported(pb);
+    if (pipe) {
+      e = plan_score_tensor(pb, cu_host, status, &cur.plan);
+      if (e != cudaSuccess) return cuda_fail(e);
+      if (cur.plan.n_cta == 0) pipe = false;                        // no history: nothing to score
+    }
+    const bool queued = !os->queue.empty() || os->pending.valid;
+    if (queued && (!pipe || (os->queue.empty() ? os->pending.st : os->queue[0].st) != st)) {
       e = flush_pending(os, &launches);
       if (e != cudaSuccess) return cuda_fail(e);
     }
     e = claim_slot(os, slot, st);
     if (e != cudaSuccess) return cuda_fail(e);
     if (pipe) {
-      // pass 1 of this layer beside pass 2 of the layer before; this layer's votes come with the next call
-      e = plan_score_tensor(pb, cu_host, status, &cur.plan);
-      if (e != cudaSuccess) return cuda_fail(e);
-      e = launch_score_pipe(&cur.plan, os->pending.valid ? &os->pending.plan : nullptr, st, &launches);
-      if (e != cudaSuccess) return cuda_fail(e);
-      if (os->pending.valid) {
-        e = enqueue_tail(os, os->pending, true, &launches);
+      // Queue the layer; the score kernel takes a list of layers per launch (pass 1 of each beside pass 2 of the
+      // one before) and goes out when the list is full and one more layer has come, or at a join.
+      os->queue.push_back(cur);
+      if ((int)os->queue.size() > kPipeMaxLayers) {
+        e = launch_queue(os, kPipeMaxLayers, false, &launches);
         if (e != cudaSuccess) return cuda_fail(e);
       }
-      os->pending = cur;
     } else {
       rc = enqueue_votes(pb, path, cu_host, status, st, &launches);
       if (rc != SLKV_OK) return rc;
@@ -560,7 +579,9 @@ int slkv_compress_overlapped(const slkv_params* p, const void* q_win, const void
 }
 
 int slkv_join(void* stream) {
-  cudaError_t e = join_overlapped((cudaStream_t)stream);
+  int launches = 0;
+  cudaError_t e = join_overlapped((cudaStream_t)stream, &launches);
+  g_last_launches = launches;
   if (e != cudaSuccess) return cuda_fail(e);
   return SLKV_OK;
 }
@@ -595,7 +616,7 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
   pb.tab.cu_ptr = cu_seqlens_dev;
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
-  cudaError_t e = join_overlapped(st);             // the workspace may still serve an overlapped call
+  cudaError_t e = join_overlapped(st, &launches);  // the workspace may still serve an overlapped call
   if (e != cudaSuccess) return cuda_fail(e);
   if (pb.tab.n_inline == 0) {
     e = launch_setup(pb, nullptr, nullptr, 0, nullptr, st, &launches);

@@ -159,8 +159,12 @@ cudaError_t plan_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t
 // Timeline buffer of this thread (diagnostics), or null: half 0 / 1, kTraceSlots words per CTA.
 unsigned long long* tensor_trace_buffer(int half, int n_cta);
 
-// Two layers per launch: pass 1 of plan `a` beside pass 2 of plan `b` (either may be null).  The shapes it takes:
+// Several layers per launch, pass 1 of one layer beside pass 2 of the layer before: pass 1 of a[0..n_a), pass 2 of
+// `pending` (pass 1 done by an earlier launch; may be null) and of a[0..n_a-1), or of all of a[] when `finish`.
+// All plans share one shape.  The shapes it takes:
 bool score_pipe_supported(const Problem& pb);
-cudaError_t launch_score_pipe(const TcPlan* a, const TcPlan* b, cudaStream_t st, int* launches);
+constexpr int kPipeMaxLayers = 8;
+cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int n_a, bool finish, cudaStream_t st,
+                              int* launches);
 
 }  // namespace slkv

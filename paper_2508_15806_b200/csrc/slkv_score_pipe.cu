@@ -10,9 +10,17 @@
 // Each stream has its own TMA producer thread, MMA issuer thread, K ring, Q tile, two TMEM accumulators and two
 // epilogue warpgroups; the special-function and FMA pipes, which bound both passes, never wait for one stream's
 // barrier, merge, ramp-up or load latency while the other has tiles ready.
+// A launch takes a list of layers: stream A walks pass 1 of layers 1..n, stream B pass 2 of layers 0..n-1 (layer 0
+// is the one whose pass 1 the launch before did) or 0..n.  Pass 2 of a layer of the same launch waits until every
+// CTA has published that layer's row statistics (one counter per layer, all CTAs resident: cooperative launch);
+// stream A never waits for anything, so the ramp-up, the launch gap and the stragglers of a launch are paid once per
+// list, not once per layer.
 // Shapes: bf16, head_dim 128, G * w <= 128 query rows per KV head.  Every wait is bounded (1 s), as in the
 // single-layer kernels: SLKV_ERR_DEVICE_TIMEOUT in the status words, TMEM freed, return.
 #include <cuda.h>
+
+#include <atomic>
+#include <cstring>
 
 #include "slkv_internal.cuh"
 #include "slkv_tc_device.cuh"
@@ -30,11 +38,28 @@ constexpr int kPipeTail = 512 + 1024 + 1024;   // mbarriers + flags, stat_m/stat
 constexpr int kPipeSmem = 2 * kQBytes + (kStagesA + kStagesB) * kStageBytes + kPipeTail;
 static_assert(kPipeSmem <= kSmemLimit, "shared memory of the two-stream kernel");
 
-struct PipeArgs {
-  TcArgs a;        // stream A: pass 1 of this layer
-  TcArgs b;        // stream B: pass 2 of this layer
-  int has_a, has_b;
+constexpr int kMaxLay = kPipeMaxLayers + 1;     // the layer pending from the launch before + this launch's layers
+constexpr int kCountSlots = 64;                 // launches whose counters are live at once
+
+struct LayerDesc {
+  alignas(64) CUtensorMap tm_q;
+  alignas(64) CUtensorMap tm_k;
+  float* part_m;
+  float* part_z;
+  float* vote;
+  int32_t* status;
 };
+struct PipeArgs {
+  TcArgs base;                 // tables, shapes, schedule, scale: the same for every layer of the launch
+  LayerDesc lay[kMaxLay];
+  int a_first, a_last;         // stream A: pass 1 of layers a_first..a_last (none if a_first > a_last)
+  int b_first, b_last;         // stream B: pass 2 of layers b_first..b_last
+  unsigned* counters;          // [kMaxLay] CTAs that have published the layer's row statistics (running totals)
+  unsigned target[kMaxLay];    // value a layer's counter reaches when all CTAs of this launch have
+};
+
+// Running totals, never reset: a launch waits for the value its host-side bookkeeping says the counter will have.
+__device__ unsigned g_layer_published[kCountSlots * kMaxLay];
 
 // One stream's resources inside the CTA.
 struct StreamCtx {
@@ -53,47 +78,53 @@ __device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, %
 
 // ---- one thread: TMA loads of the stream's Q tiles and K tiles ------------------------------------------
 template <bool REV>
-__device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, const CUtensorMap* tm_q, const CUtensorMap* tm_k) {
+__device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, const LayerDesc* lay, int first, int last,
+                                         int new_from) {
   int it = 0, run_idx = 0, st = 0;
   uint32_t st_phase = 0;
   bool ok = true;
-  for (int pos = REV ? c.end - 1 : c.begin; (REV ? pos >= c.begin : pos < c.end) && ok;) {
-    const Run r = locate(a, pos, c.begin, c.end, REV);
-    ok = mbar_wait(c.qempty_bar(), (run_idx & 1) ^ 1, c.abort_flag);        // the run before is done with Q
-    if (!ok) break;
-    mbar_expect_tx(c.qfull_bar(), 2u * (uint32_t)a.R * 128u);
-    const int qy = a.q_head_inner ? r.g * a.G : 0, qz = a.q_head_inner ? 0 : r.g * a.G;
-    tma_load_4d(c.q_smem, tm_q, 0, qy, qz, r.s, c.qfull_bar());
-    tma_load_4d(c.q_smem + kHalfBytes, tm_q, 64, qy, qz, r.s, c.qfull_bar());
-    int tok = a.tab.cu_at(r.s) + (r.t0 + (REV ? r.count - 1 : 0)) * kTileKeys;
-    const int tok_step = REV ? -kTileKeys : kTileKeys;
-    for (int i = 0; i < r.count; ++i, ++it, tok += tok_step) {
-      ok = mbar_wait(c.empty_bar(st), st_phase ^ 1u, c.abort_flag);
+  for (int j = first; j <= last && ok; ++j) {
+    if (j == new_from || (j == first && j > new_from)) pdl_wait();   // inputs this launch is the first to read
+    const CUtensorMap* tm_q = &lay[j].tm_q;
+    const CUtensorMap* tm_k = &lay[j].tm_k;
+    for (int pos = REV ? c.end - 1 : c.begin; (REV ? pos >= c.begin : pos < c.end) && ok;) {
+      const Run r = locate(a, pos, c.begin, c.end, REV);
+      ok = mbar_wait(c.qempty_bar(), (run_idx & 1) ^ 1, c.abort_flag);        // the run before is done with Q
       if (!ok) break;
-      const uint32_t fb = c.full_bar(st), dst = c.k_smem + (uint32_t)st * kStageBytes;
-      mbar_expect_tx(fb, kStageBytes);
-      const int ky = a.k_head_inner ? r.g : tok, kz = a.k_head_inner ? tok : r.g;
-      tma_load_3d(dst, tm_k, 0, ky, kz, fb);
-      tma_load_3d(dst + kHalfBytes, tm_k, 64, ky, kz, fb);
-      if (++st == c.n_stages) { st = 0; st_phase ^= 1u; }
+      mbar_expect_tx(c.qfull_bar(), 2u * (uint32_t)a.R * 128u);
+      const int qy = a.q_head_inner ? r.g * a.G : 0, qz = a.q_head_inner ? 0 : r.g * a.G;
+      tma_load_4d(c.q_smem, tm_q, 0, qy, qz, r.s, c.qfull_bar());
+      tma_load_4d(c.q_smem + kHalfBytes, tm_q, 64, qy, qz, r.s, c.qfull_bar());
+      int tok = a.tab.cu_at(r.s) + (r.t0 + (REV ? r.count - 1 : 0)) * kTileKeys;
+      const int tok_step = REV ? -kTileKeys : kTileKeys;
+      for (int i = 0; i < r.count; ++i, ++it, tok += tok_step) {
+        ok = mbar_wait(c.empty_bar(st), st_phase ^ 1u, c.abort_flag);
+        if (!ok) break;
+        const uint32_t fb = c.full_bar(st), dst = c.k_smem + (uint32_t)st * kStageBytes;
+        mbar_expect_tx(fb, kStageBytes);
+        const int ky = a.k_head_inner ? r.g : tok, kz = a.k_head_inner ? tok : r.g;
+        tma_load_3d(dst, tm_k, 0, ky, kz, fb);
+        tma_load_3d(dst + kHalfBytes, tm_k, 64, ky, kz, fb);
+        if (++st == c.n_stages) { st = 0; st_phase ^= 1u; }
+      }
+      pos = REV ? pos - r.count : pos + r.count;
+      ++run_idx;
     }
-    pos = REV ? pos - r.count : pos + r.count;
-    ++run_idx;
   }
   if (!ok) {
     // give loads already in flight a bounded chance to land before the CTA's shared memory goes away
     const unsigned long long t0 = now_ns();
     for (int s2 = 0; s2 < c.n_stages; ++s2) {
-      const int last = it - 1 - ((it - 1 - s2) % c.n_stages + c.n_stages) % c.n_stages;   // last issue into stage s2
-      if (it == 0 || last < 0) continue;
-      while (!mbar_try(c.full_bar(s2), (last / c.n_stages) & 1) && now_ns() - t0 < kWaitLimitNs) {}
+      const int last_it = it - 1 - ((it - 1 - s2) % c.n_stages + c.n_stages) % c.n_stages;   // last issue into stage s2
+      if (it == 0 || last_it < 0) continue;
+      while (!mbar_try(c.full_bar(s2), (last_it / c.n_stages) & 1) && now_ns() - t0 < kWaitLimitNs) {}
     }
   }
 }
 
 // ---- one thread: the stream's MMAs, one 128 x 128 x 128 product per tile into one of two accumulators --------
 template <bool REV>
-__device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a) {
+__device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int first, int last) {
   // pass 1: D[row, key] = Q K^T (A = Q, B = K); pass 2: D[key, row] = K Q^T (A = K, B = Q, N = R)
   const uint32_t idesc = REV ? instr_desc(kTileKeys, a.R) : instr_desc(128, kTileKeys);
   const uint64_t q_desc0 = smem_desc(c.q_smem), k_desc0 = smem_desc(c.k_smem);
@@ -102,6 +133,7 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a) {
   uint32_t st_phase = 0, b_phase = 0;
   uint64_t k_desc = k_desc0;
   bool ok = true;
+  for (int j = first; j <= last && ok; ++j)
   for (int pos = REV ? c.end - 1 : c.begin; (REV ? pos >= c.begin : pos < c.end) && ok;) {
     const Run r = locate(a, pos, c.begin, c.end, REV);
     ok = mbar_wait(c.qfull_bar(), run_idx & 1, c.abort_flag);
@@ -130,13 +162,16 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a) {
 }
 
 // ---- 256 threads: pass 1, row statistics (stream A) ----------------------------------------------------------
-__device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& a, int et, int warp, float* stat_m, float* stat_z) {
+__device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& a, const PipeArgs& pa, int et, int warp,
+                                              float* stat_m, float* stat_z) {
   const int wg = et >> 7, row = et & 127, lane = et & 31;
   const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
   const float sc = a.scale_log2;
   const int R = a.R;
   int it = 0;
   bool ok = true;
+  for (int j = pa.a_first; j <= pa.a_last; ++j) {
+  const LayerDesc& L = pa.lay[j];
   for (int pos = c.begin; pos < c.end;) {
     const Run r = locate(a, pos, c.begin, c.end, false);
     const int seg = r.s * a.n_kv_heads + r.g;
@@ -202,11 +237,16 @@ __device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& 
       float Z = 0.f;
       if (h0) Z += z * ex2(m - M);
       if (h1) Z += z1 * ex2(m1 - M);
-      a.part_m[((long long)seg * a.slot_stride + slot) * R + row] = M;
-      a.part_z[((long long)seg * a.slot_stride + slot) * R + row] = Z;
+      L.part_m[((long long)seg * a.slot_stride + slot) * R + row] = M;
+      L.part_z[((long long)seg * a.slot_stride + slot) * R + row] = Z;
     }
     named_bar(1);
     pos += r.count;
+  }
+  // This CTA's row statistics of layer j are written (the barrier above orders the other threads' stores before
+  // this thread's release): one more CTA has published.
+  if (et == 0 && ok) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(pa.counters + j) : "memory");
+  if (et == 0 && j < 24) trace_mark(a.trace, 8 + 2 * j);
   }
 }
 
@@ -225,7 +265,8 @@ __device__ __forceinline__ float vote_chunk(const uint32_t (&r)[32], float sc, c
 }
 
 // ---- 256 threads: pass 2, votes (stream B) ---------------------------------------------------------------------
-__device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs& a, int et, int warp, float* lse2) {
+__device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs& a, const PipeArgs& pa, int et, int warp,
+                                               float* lse2) {
   const int wg = et >> 7, row = et & 127, lane = et & 31;
   const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
   const float sc = a.scale_log2;
@@ -233,6 +274,25 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
   const int R = a.R;
   int it = 0, run_idx = 0;
   bool ok = true;
+  for (int j = pa.b_first; j <= pa.b_last; ++j) {
+  const LayerDesc& L = pa.lay[j];
+  if (j >= pa.a_first && j <= pa.a_last) {
+    // the layer's pass 1 is part of this launch: wait until every CTA has published its row statistics (all CTAs
+    // are resident, and stream A waits for nothing, so the count gets there; bounded all the same)
+    if (et == 0 && ok) {
+      const unsigned long long t0 = now_ns();
+      for (unsigned spin = 1;; ++spin) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(pa.counters + j) : "memory");
+        if ((int)(v - pa.target[j]) >= 0) break;
+        if ((spin & 63u) == 0 && (*c.abort_flag || now_ns() - t0 > kWaitLimitNs)) { *c.abort_flag = 1; break; }
+        __nanosleep(64);
+      }
+    }
+    named_bar(2);
+    ok = ok && *c.abort_flag == 0;
+  }
+  if (et == 0 && j < 24) trace_mark(a.trace, 9 + 2 * j);
   for (int pos = c.end - 1; pos >= c.begin;) {
     const Run r = locate(a, pos, c.begin, c.end, true);
     const int seg = r.s * a.n_kv_heads + r.g;
@@ -246,8 +306,8 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
       const int half = et & 1;
       float M = -INFINITY, Z = 0.f;
       if (rr >= 0) {
-        const float* pm = a.part_m + (long long)seg * a.slot_stride * R + rr;      // [segment][slot][row]
-        const float* pz = a.part_z + (long long)seg * a.slot_stride * R + rr;
+        const float* pm = L.part_m + (long long)seg * a.slot_stride * R + rr;      // [segment][slot][row]
+        const float* pz = L.part_z + (long long)seg * a.slot_stride * R + rr;
         for (int c0 = half; c0 < n_slots; c0 += 24) {
           float m12[12], z12[12];
 #pragma unroll
@@ -305,18 +365,17 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
           acc += vote_chunk(rb, sc, lse + c0 + 32);
         }
       }
-      const int j = key0 + row;
-      if (j < r.n_hist) a.vote[a.tab.hist_at(r.s) * a.n_kv_heads + (long long)r.g * r.n_hist + j] = acc * inv_g;
+      const int jk = key0 + row;
+      if (jk < r.n_hist) L.vote[a.tab.hist_at(r.s) * a.n_kv_heads + (long long)r.g * r.n_hist + jk] = acc * inv_g;
     }
     pos -= r.count;
     ++run_idx;
   }
+  }
 }
 
 __global__ void __launch_bounds__(kPipeThreads, 1)
-k_score_pipe(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ CUtensorMap tm_ka,
-             const __grid_constant__ CUtensorMap tm_qb, const __grid_constant__ CUtensorMap tm_kb,
-             const __grid_constant__ PipeArgs pa) {
+k_score_pipe(const __grid_constant__ PipeArgs pa) {
   // Shared memory, all dynamic and 1024-byte aligned (the swizzled tiles need it):
   //   [Q of A 32 KB][Q of B 32 KB][K ring of A 3 x 32 KB][K ring of B 2 x 32 KB][mbarriers, flags 512 B]
   //   [stat_m, stat_z of A 1 KB][log-sum-exp rows of B 2 x 512 B]
@@ -328,12 +387,14 @@ k_score_pipe(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ 
   float* stat_m = reinterpret_cast<float*>(tail + 512);
   float* stat_z = stat_m + 128;
   float* lse2 = stat_m + 256;
-  const bool has_a = pa.has_a != 0, has_b = pa.has_b != 0;
-  int32_t* status_a = has_a ? pa.a.status : nullptr;
-  int32_t* status_b = has_b ? pa.b.status : nullptr;
+  const TcArgs& a = pa.base;
+  const bool has_a = pa.a_first <= pa.a_last, has_b = pa.b_first <= pa.b_last;
+  const int lay_lo = has_b ? min(pa.b_first, has_a ? pa.a_first : pa.b_first) : pa.a_first;
+  const int lay_hi = has_a ? max(pa.a_last, has_b ? pa.b_last : pa.a_last) : pa.b_last;
   if ((smem_u32(smem) & 1023u) != 0) {                      // never run on a skewed layout (uniform over the CTA)
-    if (tid == 0 && status_a) atomicExch(status_a, (int)SLKV_ERR_BAD_ALIGN);
-    if (tid == 0 && status_b) atomicExch(status_b, (int)SLKV_ERR_BAD_ALIGN);
+    if (tid == 0)
+      for (int j = lay_lo; j <= lay_hi; ++j)
+        if (pa.lay[j].status) atomicExch(pa.lay[j].status, (int)SLKV_ERR_BAD_ALIGN);
     return;
   }
   StreamCtx ca, cb;
@@ -346,18 +407,15 @@ k_score_pipe(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ 
   ca.n_stages = kStagesA;
   cb.n_stages = kStagesB;
   ca.abort_flag = cb.abort_flag = &abort_sh;
-  ca.begin = has_a ? min(blockIdx.x * pa.a.tiles_per_cta, pa.a.total_tiles) : 0;
-  ca.end = has_a ? min(ca.begin + pa.a.tiles_per_cta, pa.a.total_tiles) : 0;
-  cb.begin = has_b ? min(blockIdx.x * pa.b.tiles_per_cta, pa.b.total_tiles) : 0;
-  cb.end = has_b ? min(cb.begin + pa.b.tiles_per_cta, pa.b.total_tiles) : 0;
+  ca.begin = cb.begin = min(blockIdx.x * a.tiles_per_cta, a.total_tiles);
+  ca.end = cb.end = min(ca.begin + a.tiles_per_cta, a.total_tiles);
 
-  unsigned long long* trace = has_a ? pa.a.trace : pa.b.trace;
-  if (tid == 0) trace_mark(trace, 0);
+  if (tid == 0) trace_mark(a.trace, 0);
   if (tid == 0) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_ka)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_kb)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_qa)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_qb)) : "memory");
+    if (has_a) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&pa.lay[pa.a_first].tm_k)) : "memory");
+    if (has_b) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&pa.lay[pa.b_first].tm_k)) : "memory");
+    if (has_a) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&pa.lay[pa.a_first].tm_q)) : "memory");
+    if (has_b) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&pa.lay[pa.b_first].tm_q)) : "memory");
     abort_sh = 0;
     for (int s = 0; s < 2; ++s) {
       const StreamCtx& c = s ? cb : ca;
@@ -369,7 +427,7 @@ k_score_pipe(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // rows of a Q tile beyond R are never written by TMA: keep them zero
-  if ((has_a && pa.a.R != 128) || (has_b && pa.b.R != 128)) {
+  if (a.R != 128) {
     for (int i = tid; i < 2 * kQBytes / 16; i += kPipeThreads) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -385,41 +443,40 @@ k_score_pipe(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ 
   cb.tmem0 = tmem_base + 256;
   pdl_launch_dependents();
 
-  // Stream A reads this layer's Q and K for the first time and overwrites partials the launch before may still be
-  // merging: all its roles wait for the work before this launch.  Stream B's loads and MMAs need only Q and K of
-  // the layer before, which the launch before this one has read: they start at once; its epilogue needs that
-  // launch's partials and waits.
+  // Stream A reads its layers' Q and K for the first time and overwrites row statistics an earlier launch may still
+  // be merging: all its roles wait for the work before this launch.  Stream B's loads and MMAs need only Q and K,
+  // which are inputs, and for the pending layer have been read by the launch before: they start at once; its
+  // epilogue needs that launch's row statistics and waits.
   if (warp == 0) {
-    if (lane == 0 && has_a) { pdl_wait(); producer<false>(ca, pa.a, &tm_qa, &tm_ka); }
+    if (lane == 0 && has_a) producer<false>(ca, a, pa.lay, pa.a_first, pa.a_last, pa.a_first);
   } else if (warp == 1) {
-    if (lane == 0 && has_a) issuer<false>(ca, pa.a);
+    if (lane == 0 && has_a) issuer<false>(ca, a, pa.a_first, pa.a_last);
   } else if (warp == 2) {
-    if (lane == 0 && has_b) producer<true>(cb, pa.b, &tm_qb, &tm_kb);
+    if (lane == 0 && has_b) producer<true>(cb, a, pa.lay, pa.b_first, pa.b_last, 1);   // layer 0 was read before
   } else if (warp == 3) {
-    if (lane == 0 && has_b) issuer<true>(cb, pa.b);
+    if (lane == 0 && has_b) issuer<true>(cb, a, pa.b_first, pa.b_last);
   } else if (warp < 12) {
     if (has_a) {
       pdl_wait();
-      if (tid == 128) trace_mark(trace, 1);
-      epilogue_rows(ca, pa.a, tid - 128, warp, stat_m, stat_z);
-      if (tid == 128) trace_mark(trace, 5);
+      if (tid == 128) trace_mark(a.trace, 1);
+      epilogue_rows(ca, a, pa, tid - 128, warp, stat_m, stat_z);
+      if (tid == 128) trace_mark(a.trace, 5);
     }
   } else {
     if (has_b) {
       pdl_wait();
-      if (tid == 384) trace_mark(trace, 7);
-      epilogue_votes(cb, pa.b, tid - 384, warp, lse2);
-      if (tid == 384) trace_mark(trace, 6);
+      if (tid == 384) trace_mark(a.trace, 7);
+      epilogue_votes(cb, a, pa, tid - 384, warp, lse2);
+      if (tid == 384) trace_mark(a.trace, 6);
     }
   }
 
   tc_fence_before();
   __syncthreads();
-  if (abort_sh && tid == 0) {
-    if (status_a) atomicExch(status_a, (int)SLKV_ERR_DEVICE_TIMEOUT);
-    if (status_b) atomicExch(status_b, (int)SLKV_ERR_DEVICE_TIMEOUT);
-  }
-  if (tid == 0) trace_mark(trace, 4);
+  if (abort_sh && tid == 0)
+    for (int j = lay_lo; j <= lay_hi; ++j)
+      if (pa.lay[j].status) atomicExch(pa.lay[j].status, (int)SLKV_ERR_DEVICE_TIMEOUT);
+  if (tid == 0) trace_mark(a.trace, 4);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -432,33 +489,82 @@ bool score_pipe_supported(const Problem& pb) {
   return tensor_path_supported(pb.p) && pb.R <= 128;
 }
 
-// One launch: pass 1 of plan `a` (or null) and pass 2 of plan `b` (or null).
-cudaError_t launch_score_pipe(const TcPlan* a, const TcPlan* b, cudaStream_t st, int* launches) {
-  const bool has_a = a && a->n_cta > 0, has_b = b && b->n_cta > 0;
-  if (!has_a && !has_b) return cudaSuccess;
+// One launch: pass 1 of plans a[0..n_a) beside pass 2 of `pending` (the layer whose pass 1 an earlier launch did;
+// may be null) and of a[0..n_a-1), or of all of a[] when `finish` is set.  The plans share one shape and schedule.
+cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int n_a, bool finish, cudaStream_t st,
+                              int* launches) {
+  if (n_a > kPipeMaxLayers) return cudaErrorInvalidValue;
+  const TcPlan* any = pending && pending->n_cta > 0 ? pending : nullptr;
+  for (int i = 0; i < n_a && !any; ++i)
+    if (a[i]->n_cta > 0) any = a[i];
+  if (!any) return cudaSuccess;                       // no history anywhere: nothing to score
   static thread_local int configured_dev = -1;
+  static thread_local unsigned* counters_base = nullptr;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (configured_dev != dev) {
     e = cudaFuncSetAttribute(k_score_pipe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem);
     if (e != cudaSuccess) return e;
+    void* sym = nullptr;
+    e = cudaGetSymbolAddress(&sym, g_layer_published);
+    if (e != cudaSuccess) return e;
+    counters_base = static_cast<unsigned*>(sym);
     configured_dev = dev;
   }
   PipeArgs pa;
-  const TcPlan* any = has_a ? a : b;
-  pa.a = has_a ? a->a : any->a;
-  pa.b = has_b ? b->a : any->a;
-  pa.has_a = has_a; pa.has_b = has_b;
-  int n_cta = 0;
-  if (has_a) n_cta = a->n_cta;
-  if (has_b && b->n_cta > n_cta) n_cta = b->n_cta;
-  unsigned long long* tr = tensor_trace_buffer(0, n_cta);
-  pa.a.trace = tr; pa.b.trace = tr;
+  std::memset(&pa, 0, sizeof(pa));
+  pa.base = any->a;
+  pa.base.part_m = pa.base.part_z = pa.base.vote = nullptr;
+  pa.base.status = nullptr;
+  auto fill = [&](int j, const TcPlan* p) {
+    pa.lay[j].tm_q = p->tm_q; pa.lay[j].tm_k = p->tm_k;
+    pa.lay[j].part_m = p->a.part_m; pa.lay[j].part_z = p->a.part_z; pa.lay[j].vote = p->a.vote;
+    pa.lay[j].status = p->a.status;
+  };
+  const bool has_pending = pending && pending->n_cta > 0;
+  if (has_pending) fill(0, pending);
+  int n_live = 0;
+  for (int i = 0; i < n_a; ++i)
+    if (a[i]->n_cta > 0) fill(++n_live, a[i]);      // layers without history take no part
+  pa.a_first = 1; pa.a_last = n_live;
+  pa.b_first = has_pending ? 0 : 1;
+  pa.b_last = finish ? n_live : n_live - 1;
+  if (pa.a_first > pa.a_last && pa.b_first > pa.b_last) return cudaSuccess;
+  const int n_cta = any->n_cta;
+  pa.base.trace = tensor_trace_buffer(0, n_cta);
+  // counters of this launch: a slot of the table, zeroed on the stream before the kernel
+  static std::atomic<unsigned> launch_seq{0};
+  pa.counters = counters_base + (size_t)(launch_seq.fetch_add(1) % kCountSlots) * kMaxLay;
+  for (int j = 0; j < kMaxLay; ++j) pa.target[j] = (unsigned)n_cta;
+  const bool waits_inside = pa.b_last >= pa.a_first && pa.a_last >= pa.a_first;   // a layer's two passes in one launch
+  if (waits_inside) {
+    e = cudaMemsetAsync(pa.counters, 0, kMaxLay * sizeof(unsigned), st);
+    if (e != cudaSuccess) return e;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_cta);
+  cfg.blockDim = dim3(kPipeThreads);
+  cfg.dynamicSmemBytes = kPipeSmem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (waits_inside) {                                 // CTAs wait for one another: all of them must be resident
+    attr[n].id = cudaLaunchAttributeCooperative;
+    attr[n].val.cooperative = 1;
+    ++n;
+  } else {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
   LaunchScope scope(KID_SCORE_PIPE, st, launches);
-  return launch_pdl(k_score_pipe, dim3(n_cta), dim3(kPipeThreads), (size_t)kPipeSmem, st, 1,
-                    has_a ? a->tm_q : any->tm_q, has_a ? a->tm_k : any->tm_k,
-                    has_b ? b->tm_q : any->tm_q, has_b ? b->tm_k : any->tm_k, pa);
+  return cudaLaunchKernelEx(&cfg, k_score_pipe, pa);
 }
+
+// The most layers one launch takes (pass 1); callers that queue layers launch when they have this many.
+int score_pipe_max_layers() { return kPipeMaxLayers; }
 
 }  // namespace slkv
