@@ -30,6 +30,7 @@ namespace {
 
 constexpr int kPipeThreads = 640;        // warps 0-3: producer A, issuer A, producer B, issuer B;
                                          // warps 4-11: epilogue of stream A; warps 12-19: epilogue of stream B
+constexpr unsigned kPollNs = 64;          // pause between two polls of an mbarrier
 constexpr int kStagesA = 3;              // K tiles in flight from HBM
 constexpr int kStagesB = 2;              // K tiles in flight from L2
 constexpr int kQBytes = 2 * kHalfBytes;  // one 128-row Q tile
@@ -66,6 +67,7 @@ struct StreamCtx {
   uint32_t q_smem, k_smem, bar0, tmem0;
   int n_stages, begin, end;
   volatile int* abort_flag;
+  volatile int* b_layer;       // CTA-wide: the layer whose pass 2 this CTA's epilogue has begun
   __device__ __forceinline__ uint32_t full_bar(int st) const { return bar0 + 8u * st; }
   __device__ __forceinline__ uint32_t empty_bar(int st) const { return bar0 + 8u * (3 + st); }
   __device__ __forceinline__ uint32_t accf_bar(int b) const { return bar0 + 8u * (6 + b); }
@@ -85,11 +87,22 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
   bool ok = true;
   for (int j = first; j <= last && ok; ++j) {
     if (j == new_from || (j == first && j > new_from)) pdl_wait();   // inputs this launch is the first to read
+    if (!REV) {
+      // Pass 1 stays at most one layer ahead of this CTA's pass 2 (which needs the other CTAs' pass 1 of the layer
+      // before, so it cannot deadlock): the two streams then share the SM to the end instead of pass 2 running on
+      // alone, on half the epilogue warps, after pass 1 has raced through the list.
+      const unsigned long long t0 = now_ns();
+      for (unsigned spin = 1; *c.b_layer < j - 2; ++spin) {
+        if ((spin & 63u) == 0 && (*c.abort_flag || now_ns() - t0 > kWaitLimitNs)) { *c.abort_flag = 1; ok = false; break; }
+        __nanosleep(100);
+      }
+      if (!ok) break;
+    }
     const CUtensorMap* tm_q = &lay[j].tm_q;
     const CUtensorMap* tm_k = &lay[j].tm_k;
     for (int pos = REV ? c.end - 1 : c.begin; (REV ? pos >= c.begin : pos < c.end) && ok;) {
       const Run r = locate(a, pos, c.begin, c.end, REV);
-      ok = mbar_wait(c.qempty_bar(), (run_idx & 1) ^ 1, c.abort_flag);        // the run before is done with Q
+      ok = mbar_wait(c.qempty_bar(), (run_idx & 1) ^ 1, c.abort_flag, kPollNs);        // the run before is done with Q
       if (!ok) break;
       mbar_expect_tx(c.qfull_bar(), 2u * (uint32_t)a.R * 128u);
       const int qy = a.q_head_inner ? r.g * a.G : 0, qz = a.q_head_inner ? 0 : r.g * a.G;
@@ -98,7 +111,7 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
       int tok = a.tab.cu_at(r.s) + (r.t0 + (REV ? r.count - 1 : 0)) * kTileKeys;
       const int tok_step = REV ? -kTileKeys : kTileKeys;
       for (int i = 0; i < r.count; ++i, ++it, tok += tok_step) {
-        ok = mbar_wait(c.empty_bar(st), st_phase ^ 1u, c.abort_flag);
+        ok = mbar_wait(c.empty_bar(st), st_phase ^ 1u, c.abort_flag, kPollNs);
         if (!ok) break;
         const uint32_t fb = c.full_bar(st), dst = c.k_smem + (uint32_t)st * kStageBytes;
         mbar_expect_tx(fb, kStageBytes);
@@ -136,10 +149,10 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int 
   for (int j = first; j <= last && ok; ++j)
   for (int pos = REV ? c.end - 1 : c.begin; (REV ? pos >= c.begin : pos < c.end) && ok;) {
     const Run r = locate(a, pos, c.begin, c.end, REV);
-    ok = mbar_wait(c.qfull_bar(), run_idx & 1, c.abort_flag);
+    ok = mbar_wait(c.qfull_bar(), run_idx & 1, c.abort_flag, kPollNs);
     if (!ok) break;
     for (int i = 0; i < r.count; ++i, ++it) {
-      ok = mbar_wait(c.full_bar(st), st_phase, c.abort_flag) && mbar_wait(c.acce_bar(b), b_phase ^ 1u, c.abort_flag);
+      ok = mbar_wait(c.full_bar(st), st_phase, c.abort_flag, kPollNs) && mbar_wait(c.acce_bar(b), b_phase ^ 1u, c.abort_flag, kPollNs);
       if (!ok) break;
       tc_fence_after();
       const uint32_t d0 = c.tmem0 + (uint32_t)(b * 128);
@@ -180,7 +193,7 @@ __device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& 
     for (int i = 0; i < r.count; ++i, ++it) {
       if ((it & 1) != wg) continue;
       const int b = it & 1;
-      if (ok) ok = mbar_wait(c.accf_bar(b), (it >> 1) & 1, c.abort_flag);
+      if (ok) ok = mbar_wait(c.accf_bar(b), (it >> 1) & 1, c.abort_flag, kPollNs);
       ok = __all_sync(0xffffffffu, ok) != 0;                  // the TMEM loads below need the whole warp
       if (!ok) continue;
       tc_fence_after();
@@ -292,6 +305,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
     named_bar(2);
     ok = ok && *c.abort_flag == 0;
   }
+  if (et == 0) *c.b_layer = j;
   if (et == 0 && j < 24) trace_mark(a.trace, 9 + 2 * j);
   for (int pos = c.end - 1; pos >= c.begin;) {
     const Run r = locate(a, pos, c.begin, c.end, true);
@@ -338,7 +352,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
     for (int i = 0; i < r.count; ++i, ++it) {
       if ((it & 1) != wg) continue;
       const int b = it & 1;
-      if (ok) ok = mbar_wait(c.accf_bar(b), (it >> 1) & 1, c.abort_flag);
+      if (ok) ok = mbar_wait(c.accf_bar(b), (it >> 1) & 1, c.abort_flag, kPollNs);
       ok = __all_sync(0xffffffffu, ok) != 0;
       if (!ok) continue;
       tc_fence_after();
@@ -384,6 +398,7 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   unsigned char* tail = smem + 2 * kQBytes + (kStagesA + kStagesB) * kStageBytes;
   uint32_t& tmem_base_sh = *reinterpret_cast<uint32_t*>(tail + 256);
   int& abort_sh = *reinterpret_cast<int*>(tail + 260);
+  int& b_layer_sh = *reinterpret_cast<int*>(tail + 264);   // the layer stream B's epilogue has begun
   float* stat_m = reinterpret_cast<float*>(tail + 512);
   float* stat_z = stat_m + 128;
   float* lse2 = stat_m + 256;
@@ -407,6 +422,7 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   ca.n_stages = kStagesA;
   cb.n_stages = kStagesB;
   ca.abort_flag = cb.abort_flag = &abort_sh;
+  ca.b_layer = cb.b_layer = &b_layer_sh;
   ca.begin = cb.begin = min(blockIdx.x * a.tiles_per_cta, a.total_tiles);
   ca.end = cb.end = min(ca.begin + a.tiles_per_cta, a.total_tiles);
 
@@ -417,6 +433,7 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
     if (has_a) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&pa.lay[pa.a_first].tm_q)) : "memory");
     if (has_b) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&pa.lay[pa.b_first].tm_q)) : "memory");
     abort_sh = 0;
+    b_layer_sh = has_b ? pa.b_first - 1 : 1 << 30;
     for (int s = 0; s < 2; ++s) {
       const StreamCtx& c = s ? cb : ca;
       for (int st = 0; st < 3; ++st) { mbar_init(c.full_bar(st), 1); mbar_init(c.empty_bar(st), 1); }

@@ -57,10 +57,12 @@ __device__ __forceinline__ void trace_mark(const unsigned long long* base, int s
   if (base) const_cast<unsigned long long*>(base)[(size_t)blockIdx.x * kTraceSlots + slot] = now_ns();
 }
 // Waits for the phase with the given parity.  false = gave up (limit reached or another thread did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// backoff_ns > 0: sleep that long between polls, so that a waiting warp leaves the issue slots to the working ones.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned backoff_ns = 0) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = now_ns();
   for (unsigned it = 1;; ++it) {
+    if (backoff_ns) __nanosleep(backoff_ns);
     if (mbar_try(bar, parity)) return true;
     if ((it & 63u) == 0) {
       if (*abort_flag) return false;
