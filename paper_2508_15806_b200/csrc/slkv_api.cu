@@ -195,6 +195,7 @@ int enqueue_votes(const Problem& pb, int path, const int32_t* cu_host, int32_t* 
 // run on the caller's stream.  Where the two-layer score kernel takes the shape, a call enqueues pass 1 of its
 // own layer together with pass 2 of the layer before (which stays "pending" until the next call or a join).
 constexpr int kSlots = 2 * kPipeMaxLayers + 2;     // layers whose votes / source rows / row statistics are live at once
+constexpr int kSideStreams = 8;   // after the last launch of a list the selections of its layers run side by side
 struct PendingCall {
   bool valid = false;
   Problem pb;
@@ -221,7 +222,7 @@ struct ShapeSig {                                  // calls in flight together m
   }
 };
 struct OverlapState {
-  cudaStream_t side_select[2] = {nullptr, nullptr}, side_gather = nullptr;
+  cudaStream_t side_select[kSideStreams] = {}, side_gather[kSideStreams] = {};   // slot s uses streams s % kSideStreams
   cudaEvent_t scored[kSlots] = {};       // recorded on the caller's stream after the vote pass of the slot's layer
   cudaEvent_t selected[kSlots] = {};     // recorded on a selection stream after the selection
   cudaEvent_t done[kSlots] = {};         // recorded on the gather stream after the gather
@@ -242,13 +243,13 @@ cudaError_t overlap_state(OverlapState** out) {
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   OverlapState& s = g_overlap[dev];
-  if (!s.side_gather) {
-    for (int i = 0; i < 2; ++i) {
+  if (!s.side_gather[kSideStreams - 1]) {
+    for (int i = 0; i < kSideStreams; ++i) {
       e = cudaStreamCreateWithFlags(&s.side_select[i], cudaStreamNonBlocking);
       if (e != cudaSuccess) return e;
+      e = cudaStreamCreateWithFlags(&s.side_gather[i], cudaStreamNonBlocking);
+      if (e != cudaSuccess) return e;
     }
-    e = cudaStreamCreateWithFlags(&s.side_gather, cudaStreamNonBlocking);
-    if (e != cudaSuccess) return e;
     for (int h = 0; h < kSlots; ++h) {
       e = cudaEventCreateWithFlags(&s.scored[h], cudaEventDisableTiming);
       if (e != cudaSuccess) return e;
@@ -267,27 +268,27 @@ cudaError_t overlap_state(OverlapState** out) {
 cudaError_t claim_slot(OverlapState* os, int slot, cudaStream_t st) {
   if (!os->in_flight[slot]) return cudaSuccess;
   cudaError_t e = cudaStreamWaitEvent(st, os->selected[slot], 0);
-  if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_select[slot & 1], os->done[slot], 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_select[slot % kSideStreams], os->done[slot], 0);
   return e;
 }
 
 // The votes of layer `c` are enqueued on c.st: selection on a side stream, gather on another.
 cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pipe, int* launches) {
   const int slot = c.slot;
-  cudaStream_t sel = os->side_select[slot & 1];
+  cudaStream_t sel = os->side_select[slot % kSideStreams], gat = os->side_gather[slot % kSideStreams];
   cudaError_t e = cudaEventRecord(os->scored[slot], c.st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(sel, os->scored[slot], 0);
   if (e != cudaSuccess) return e;
   e = launch_select_cta(c.pb, c.pooled_opt, c.budgets, c.offsets, c.kept_idx, c.capacity, c.status, sel, launches);
   if (e != cudaSuccess) return e;
   e = cudaEventRecord(os->selected[slot], sel);
-  if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_gather, os->selected[slot], 0);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(gat, os->selected[slot], 0);
   if (e != cudaSuccess) return e;
   // beside the two-layer score kernel an SM has registers left for one 128-thread gather CTA
-  e = launch_gather(c.pb, c.offsets, c.kept_idx, c.k_out, c.v_out, c.capacity, os->side_gather, launches,
+  e = launch_gather(c.pb, c.offsets, c.kept_idx, c.k_out, c.v_out, c.capacity, gat, launches,
                     beside_pipe ? 128 : 256);
   if (e != cudaSuccess) return e;
-  e = cudaEventRecord(os->done[slot], os->side_gather);
+  e = cudaEventRecord(os->done[slot], gat);
   if (e != cudaSuccess) return e;
   os->in_flight[slot] = true;
   return cudaSuccess;

@@ -76,6 +76,19 @@ struct StreamCtx {
   __device__ __forceinline__ uint32_t qempty_bar() const { return bar0 + 8u * 11; }
 };
 
+// sum_e 2^(v_e * sc - m) over 32 accumulator values.  All exponentials on the special-function unit: with sixteen
+// epilogue warps at 96 registers the polynomial share the single-layer kernels use made this kernel slower.
+__device__ __forceinline__ float sum_ex2_32_mufu(const uint32_t (&r)[32], float sc, float m) {
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < 32; e += 4) {
+    s0 += ex2(fmaf(__uint_as_float(r[e]), sc, -m));
+    s1 += ex2(fmaf(__uint_as_float(r[e + 1]), sc, -m));
+    s2 += ex2(fmaf(__uint_as_float(r[e + 2]), sc, -m));
+    s3 += ex2(fmaf(__uint_as_float(r[e + 3]), sc, -m));
+  }
+  return (s0 + s1) + (s2 + s3);
+}
 __device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(kEpiThreads) : "memory"); }
 
 // ---- one thread: TMA loads of the stream's Q tiles and K tiles ------------------------------------------
@@ -208,7 +221,7 @@ __device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& 
       uint32_t ra[32], rb[32];
       auto add_chunk = [&](const uint32_t (&rr)[32], int nv) {
         if (nv >= 32) {
-          const float zc = sum_ex2_32(rr, sc, m);
+          const float zc = sum_ex2_32_mufu(rr, sc, m);
           const float zn = z + zc;
           if (zn < INFINITY && zc > 0.f) { z = zn; return; }
         }
@@ -272,7 +285,7 @@ __device__ __forceinline__ float vote_chunk(const uint32_t (&r)[32], float sc, c
     s0 += ex2(fmaf(__uint_as_float(r[e]), sc, -l4.x));
     s1 += ex2(fmaf(__uint_as_float(r[e + 1]), sc, -l4.y));
     s2 += ex2(fmaf(__uint_as_float(r[e + 2]), sc, -l4.z));
-    s3 += ex2_fma(fmaf(__uint_as_float(r[e + 3]), sc, -l4.w), false);
+    s3 += ex2(fmaf(__uint_as_float(r[e + 3]), sc, -l4.w));
   }
   return (s0 + s1) + (s2 + s3);
 }
