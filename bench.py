@@ -223,7 +223,9 @@ def run_cuda(args):
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "device status word set during warm-up"
     eager_step = step
-    if args.graph:
+    eager_us_per_layer = None
+    if overlap and not args.no_graph:
+        eager_us_per_layer = timed(10, eager_step) / 10 * 1e3 / nl
         # The calls of a step are stream-ordered and allocate nothing: capture them once (the side streams of the
         # overlapped calls fork from and rejoin the captured stream) and replay the graph per step.
         cap = torch.cuda.Stream()
@@ -356,13 +358,16 @@ def run_cuda(args):
 
     if rank == 0:
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-               "ms_per_step": ms_per_step, "us_per_layer": t_layer_us, "higher_is_better": True, "scaling": "weak",
+               "ms_per_step": ms_per_step, "us_per_layer": t_layer_us, "us_per_layer_without_graph": eager_us_per_layer,
+               "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
                "config": {"workload": wl.name, "n_layers": nl, "n_q_heads": wl.n_q_heads, "n_kv_heads": hkv,
                           "head_dim": d, "seq_lens": wl.seq_lens, "window": w, "pool_kernel": wl.pool_kernel,
                           "avg_budget_per_kv_head": total // (nl * hkv), "fixed": wl.fixed, "parallelism":
                           f"dp{world} (one sequence batch per GPU, no collective)",
-                          "api": "slkv_compress_overlapped + slkv_join per step" if overlap else "slkv_compress",
+                          "api": ("slkv_compress_overlapped + slkv_join per step" +
+                                  (", captured once in a CUDA graph and replayed" if eager_us_per_layer is not None else ""))
+                          if overlap else "slkv_compress",
                           "l2": "inputs larger than L2: every layer has its own Q/K/V (%.1f GB per step)" %
                                 (nl * (2 * T * hkv * d * e) / 1e9)},
                "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * steps,
@@ -455,7 +460,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="use fewer layers (profiling captures only)")
     ap.add_argument("--workload", type=int, default=0, choices=[0, 1, 2, 3, 4, 5],
                     help="time another of the five workloads (default: the 32k-context one); the others are parity cases")
-    ap.add_argument("--graph", action="store_true", help="capture a step's calls in a CUDA graph and replay it")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="issue the calls of every step (default: capture a step's calls in a CUDA graph once and replay it)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="one layer at a time (slkv_compress) instead of overlapped calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")

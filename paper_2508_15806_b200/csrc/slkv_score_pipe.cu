@@ -40,6 +40,7 @@ constexpr int kPipeSmem = 2 * kQBytes + (kStagesA + kStagesB) * kStageBytes + kP
 static_assert(kPipeSmem <= kSmemLimit, "shared memory of the two-stream kernel");
 
 constexpr int kMaxLay = kPipeMaxLayers + 1;     // the layer pending from the launch before + this launch's layers
+constexpr int kCountWords = kMaxLay + 1;        // per launch: one publish counter per layer + one exit counter
 constexpr int kCountSlots = 64;                 // launches whose counters are live at once
 
 struct LayerDesc {
@@ -55,12 +56,13 @@ struct PipeArgs {
   LayerDesc lay[kMaxLay];
   int a_first, a_last;         // stream A: pass 1 of layers a_first..a_last (none if a_first > a_last)
   int b_first, b_last;         // stream B: pass 2 of layers b_first..b_last
-  unsigned* counters;          // [kMaxLay] CTAs that have published the layer's row statistics (running totals)
-  unsigned target[kMaxLay];    // value a layer's counter reaches when all CTAs of this launch have
+  unsigned* counters;          // [kMaxLay] CTAs that have published the layer's row statistics, then [1] CTAs that are done
+  unsigned target[kMaxLay];    // value a layer's counter reaches when all CTAs of this launch have published
 };
 
-// Running totals, never reset: a launch waits for the value its host-side bookkeeping says the counter will have.
-__device__ unsigned g_layer_published[kCountSlots * kMaxLay];
+// Counter sets, taken in turn by the launches (zero at load).  The last CTA of a launch to finish puts its set back to
+// zero, so the set is clean for its next user 64 launches later; no memset sits between two launches.
+__device__ unsigned g_layer_published[kCountSlots * kCountWords];
 
 // One stream's resources inside the CTA.
 struct StreamCtx {
@@ -220,6 +222,7 @@ __device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& 
       // segment's end (its ragged last tile) are left out chunk by chunk.
       uint32_t ra[32], rb[32];
       auto add_chunk = [&](const uint32_t (&rr)[32], int nv) {
+        if (nv <= 0) return;                                   // wholly past the segment's end
         if (nv >= 32) {
           const float zc = sum_ex2_32_mufu(rr, sc, m);
           const float zn = z + zc;
@@ -440,6 +443,7 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   ca.end = cb.end = min(ca.begin + a.tiles_per_cta, a.total_tiles);
 
   if (tid == 0) trace_mark(a.trace, 0);
+  if (tid == 0 && a.trace) a.trace[(size_t)blockIdx.x * kTraceSlots + 60] = (unsigned long long)clock64();
   if (tid == 0) {
     if (has_a) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&pa.lay[pa.a_first].tm_k)) : "memory");
     if (has_b) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&pa.lay[pa.b_first].tm_k)) : "memory");
@@ -507,6 +511,16 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
     for (int j = lay_lo; j <= lay_hi; ++j)
       if (pa.lay[j].status) atomicExch(pa.lay[j].status, (int)SLKV_ERR_DEVICE_TIMEOUT);
   if (tid == 0) trace_mark(a.trace, 4);
+  if (tid == 0 && a.trace) a.trace[(size_t)blockIdx.x * kTraceSlots + 61] = (unsigned long long)clock64();
+  if (tid == 0) {
+    // every thread of this CTA is past its last use of the counters (the barrier above)
+    unsigned prev;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(pa.counters + kMaxLay) : "memory");
+    if (prev == gridDim.x - 1) {
+      for (int j = 0; j <= kMaxLay; ++j) pa.counters[j] = 0;
+      __threadfence();
+    }
+  }
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -565,33 +579,49 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
   pa.base.trace = tensor_trace_buffer(0, n_cta);
   // counters of this launch: a slot of the table, zeroed on the stream before the kernel
   static std::atomic<unsigned> launch_seq{0};
-  pa.counters = counters_base + (size_t)(launch_seq.fetch_add(1) % kCountSlots) * kMaxLay;
+  pa.counters = counters_base + (size_t)(launch_seq.fetch_add(1) % kCountSlots) * kCountWords;
   for (int j = 0; j < kMaxLay; ++j) pa.target[j] = (unsigned)n_cta;
   const bool waits_inside = pa.b_last >= pa.a_first && pa.a_last >= pa.a_first;   // a layer's two passes in one launch
-  if (waits_inside) {
-    e = cudaMemsetAsync(pa.counters, 0, kMaxLay * sizeof(unsigned), st);
-    if (e != cudaSuccess) return e;
+  // CTAs that wait for one another must all be resident: cooperative launch.  Dependent launch on top where the
+  // device takes both (the kernel waits for the launch before it exactly where it needs that launch's results).
+  static thread_local int pdl_with_coop[64] = {};     // per device: 0 untried, 1 works, -1 refused
+  int& pc = pdl_with_coop[dev < 64 ? dev : 0];
+  for (int attempt = 0; attempt < 2; ++attempt) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_cta);
+    cfg.blockDim = dim3(kPipeThreads);
+    cfg.dynamicSmemBytes = kPipeSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (waits_inside) {
+      attr[n].id = cudaLaunchAttributeCooperative;
+      attr[n].val.cooperative = 1;
+      ++n;
+    }
+    const bool with_pdl = !waits_inside || pc >= 0;
+    if (with_pdl) {
+      attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[n].val.programmaticStreamSerializationAllowed = 1;
+      ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    cudaError_t le;
+    {
+      LaunchScope scope(KID_SCORE_PIPE, st, launches);
+      le = cudaLaunchKernelEx(&cfg, k_score_pipe, pa);
+    }
+    if (le == cudaSuccess) {
+      if (waits_inside && with_pdl) pc = 1;
+      return cudaSuccess;
+    }
+    if (!(waits_inside && with_pdl) || pc == 1) return le;
+    (void)cudaGetLastError();                         // not a sticky error: the launch was refused
+    --*launches;
+    pc = -1;                                          // once more without dependent launch
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(n_cta);
-  cfg.blockDim = dim3(kPipeThreads);
-  cfg.dynamicSmemBytes = kPipeSmem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[2];
-  int n = 0;
-  if (waits_inside) {                                 // CTAs wait for one another: all of them must be resident
-    attr[n].id = cudaLaunchAttributeCooperative;
-    attr[n].val.cooperative = 1;
-    ++n;
-  } else {
-    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[n].val.programmaticStreamSerializationAllowed = 1;
-    ++n;
-  }
-  cfg.attrs = attr;
-  cfg.numAttrs = n;
-  LaunchScope scope(KID_SCORE_PIPE, st, launches);
-  return cudaLaunchKernelEx(&cfg, k_score_pipe, pa);
+  return cudaErrorLaunchFailure;
 }
 
 // The most layers one launch takes (pass 1); callers that queue layers launch when they have this many.

@@ -490,6 +490,20 @@ Schedule schedule_of(const Problem& pb, const int32_t* cu_host) {
   int sms = sm_count();
   if (pb.max_score_ctas > 0 && pb.max_score_ctas < sms) sms = pb.max_score_ctas;
   sc.tiles_per_cta = sc.total_tiles > 0 ? (sc.total_tiles + sms - 1) / sms : 1;
+  // A CTA whose range straddles two segments reloads Q in mid-stream (a pipeline bubble of a few microseconds) and
+  // holds everybody else up wherever CTAs wait for one another.  When all segments have the same number of tiles
+  // and a slightly larger share per CTA divides it, the ranges line up with the segments.
+  if (pb.p.n_seqs > 0 && sc.total_tiles > 0) {
+    const long long per_seg = tiles / pb.p.n_seqs;
+    bool equal = per_seg * pb.p.n_seqs == tiles;
+    for (int s = 0; s < pb.p.n_seqs && equal; ++s) {
+      long long nh = (long long)cu_host[s + 1] - cu_host[s] - pb.p.window;
+      equal = nh > 0 && (nh + kTileKeys - 1) / kTileKeys == per_seg;
+    }
+    if (equal && per_seg >= sc.tiles_per_cta)
+      for (int t = sc.tiles_per_cta; t <= sc.tiles_per_cta + sc.tiles_per_cta / 8 + 1; ++t)
+        if (per_seg % t == 0) { sc.tiles_per_cta = t; break; }
+  }
   sc.n_cta = sc.total_tiles > 0 ? (sc.total_tiles + sc.tiles_per_cta - 1) / sc.tiles_per_cta : 0;
   return sc;
 }

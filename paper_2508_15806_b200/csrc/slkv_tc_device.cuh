@@ -22,7 +22,8 @@ constexpr int kTraceSlots = 64;               // per CTA: 0 start, 1 set-up done
                                                // 4 end; 5 / 6 grid barrier reached / passed, 7 first log-sum-exp merged; 8+2i / 9+2i = epilogue of the
                                                // CTA's i-th tile begins / ends.  Two-layer kernel: 0 start, 1 / 7 stream A / B
                                                // past its wait for the launch before, 2 first accumulator of A ready,
-                                               // 3 first log-sum-exps of B merged, 5 / 6 epilogue of A / B done, 4 end
+                                               // 3 first log-sum-exps of B merged, 5 / 6 epilogue of A / B done, 4 end,
+                                               // 8+2j / 9+2j layer j published by A / begun by B, 60 / 61 SM cycle counter at start / end
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per wait
 
 
