@@ -111,6 +111,12 @@ int describe(const slkv_params* p, const int32_t* cu_host, Problem* pb) {
   return SLKV_OK;
 }
 
+// Layers an overlapped call sequence keeps in flight: many where the score kernel takes lists of layers, three
+// otherwise (one being scored, one being selected, one being gathered).
+int overlapped_slots(const Problem& pb) {
+  return tensor_path_supported(pb.p) && score_pipe_supported(pb) && pb.p.score_path != SLKV_PATH_SIMT ? kLaySlots : 3;
+}
+
 Layout layout_of(const Problem& pb, bool overlapped = false) {
   Layout L;
   size_t o = 0;
@@ -120,7 +126,7 @@ Layout layout_of(const Problem& pb, bool overlapped = false) {
   // gathers trail behind): each has its own votes, source-row list and per-CTA row statistics.  Ordinary calls use
   // the first of each.
   const size_t votes = (size_t)pb.p.n_kv_heads * (size_t)pb.total_hist * sizeof(float);
-  const int n_slots = overlapped ? kLaySlots : 1;
+  const int n_slots = overlapped ? overlapped_slots(pb) : 1;
   for (int i = 0; i < kLaySlots; ++i) {
     L.vote[i] = i < n_slots ? o : L.vote[0];
     if (i < n_slots) o = align_up(o + votes);
@@ -276,6 +282,7 @@ cudaError_t claim_slot(OverlapState* os, int slot, cudaStream_t st) {
 cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pipe, int* launches) {
   const int slot = c.slot;
   cudaStream_t sel = os->side_select[slot % kSideStreams], gat = os->side_gather[slot % kSideStreams];
+  if (g_prof_on) sel = gat = c.st;       // per-kernel timing: one stream, so that the event pairs do not overlap
   cudaError_t e = cudaEventRecord(os->scored[slot], c.st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(sel, os->scored[slot], 0);
   if (e != cudaSuccess) return e;
@@ -386,7 +393,7 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
       if (e != cudaSuccess) return cuda_fail(e);
       os->sig = sig;
     }
-    const int slot = (int)(os->seq % kSlots);
+    const int slot = (int)(os->seq % (unsigned)overlapped_slots(pb));
     rc = bind_workspace(&pb, ws, ws_bytes, path, true, slot);
     if (rc != SLKV_OK) return rc;
     ++os->seq;

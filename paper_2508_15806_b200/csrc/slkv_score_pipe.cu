@@ -94,15 +94,18 @@ __device__ __forceinline__ float sum_ex2_32_mufu(const uint32_t (&r)[32], float 
 __device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(kEpiThreads) : "memory"); }
 
 // ---- one thread: TMA loads of the stream's Q tiles and K tiles ------------------------------------------
-template <bool REV>
+template <bool VOTE>
 __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, const LayerDesc* lay, int first, int last,
                                          int new_from) {
   int it = 0, run_idx = 0, st = 0;
   uint32_t st_phase = 0;
   bool ok = true;
+  // Every K tile is read twice, by pass 1 and a layer later by pass 2, in the same order: pass 1 asks L2 to keep the
+  // lines, pass 2 to drop them first, so that about one layer's K is live in L2 and pass 2 need not go to HBM.
+  const uint64_t policy = VOTE ? l2_policy_evict_first() : l2_policy_evict_last();
   for (int j = first; j <= last && ok; ++j) {
     if (j == new_from || (j == first && j > new_from)) pdl_wait();   // inputs this launch is the first to read
-    if (!REV) {
+    if (!VOTE) {
       // Pass 1 stays at most one layer ahead of this CTA's pass 2 (which needs the other CTAs' pass 1 of the layer
       // before, so it cannot deadlock): the two streams then share the SM to the end instead of pass 2 running on
       // alone, on half the epilogue warps, after pass 1 has raced through the list.
@@ -115,27 +118,26 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
     }
     const CUtensorMap* tm_q = &lay[j].tm_q;
     const CUtensorMap* tm_k = &lay[j].tm_k;
-    for (int pos = REV ? c.end - 1 : c.begin; (REV ? pos >= c.begin : pos < c.end) && ok;) {
-      const Run r = locate(a, pos, c.begin, c.end, REV);
+    for (int pos = c.begin; pos < c.end && ok;) {
+      const Run r = locate(a, pos, c.begin, c.end, false);
       ok = mbar_wait(c.qempty_bar(), (run_idx & 1) ^ 1, c.abort_flag, kPollNs);        // the run before is done with Q
       if (!ok) break;
       mbar_expect_tx(c.qfull_bar(), 2u * (uint32_t)a.R * 128u);
       const int qy = a.q_head_inner ? r.g * a.G : 0, qz = a.q_head_inner ? 0 : r.g * a.G;
       tma_load_4d(c.q_smem, tm_q, 0, qy, qz, r.s, c.qfull_bar());
       tma_load_4d(c.q_smem + kHalfBytes, tm_q, 64, qy, qz, r.s, c.qfull_bar());
-      int tok = a.tab.cu_at(r.s) + (r.t0 + (REV ? r.count - 1 : 0)) * kTileKeys;
-      const int tok_step = REV ? -kTileKeys : kTileKeys;
-      for (int i = 0; i < r.count; ++i, ++it, tok += tok_step) {
+      int tok = a.tab.cu_at(r.s) + r.t0 * kTileKeys;
+      for (int i = 0; i < r.count; ++i, ++it, tok += kTileKeys) {
         ok = mbar_wait(c.empty_bar(st), st_phase ^ 1u, c.abort_flag, kPollNs);
         if (!ok) break;
         const uint32_t fb = c.full_bar(st), dst = c.k_smem + (uint32_t)st * kStageBytes;
         mbar_expect_tx(fb, kStageBytes);
         const int ky = a.k_head_inner ? r.g : tok, kz = a.k_head_inner ? tok : r.g;
-        tma_load_3d(dst, tm_k, 0, ky, kz, fb);
-        tma_load_3d(dst + kHalfBytes, tm_k, 64, ky, kz, fb);
+        tma_load_3d_hint(dst, tm_k, 0, ky, kz, fb, policy);
+        tma_load_3d_hint(dst + kHalfBytes, tm_k, 64, ky, kz, fb, policy);
         if (++st == c.n_stages) { st = 0; st_phase ^= 1u; }
       }
-      pos = REV ? pos - r.count : pos + r.count;
+      pos += r.count;
       ++run_idx;
     }
   }
@@ -151,10 +153,10 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
 }
 
 // ---- one thread: the stream's MMAs, one 128 x 128 x 128 product per tile into one of two accumulators --------
-template <bool REV>
+template <bool VOTE>
 __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int first, int last) {
   // pass 1: D[row, key] = Q K^T (A = Q, B = K); pass 2: D[key, row] = K Q^T (A = K, B = Q, N = R)
-  const uint32_t idesc = REV ? instr_desc(kTileKeys, a.R) : instr_desc(128, kTileKeys);
+  const uint32_t idesc = VOTE ? instr_desc(kTileKeys, a.R) : instr_desc(128, kTileKeys);
   const uint64_t q_desc0 = smem_desc(c.q_smem), k_desc0 = smem_desc(c.k_smem);
   const uint64_t hi = (uint64_t)(kHalfBytes >> 4);
   int it = 0, run_idx = 0, st = 0, b = 0;
@@ -162,8 +164,8 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int 
   uint64_t k_desc = k_desc0;
   bool ok = true;
   for (int j = first; j <= last && ok; ++j)
-  for (int pos = REV ? c.end - 1 : c.begin; (REV ? pos >= c.begin : pos < c.end) && ok;) {
-    const Run r = locate(a, pos, c.begin, c.end, REV);
+  for (int pos = c.begin; pos < c.end && ok;) {
+    const Run r = locate(a, pos, c.begin, c.end, false);
     ok = mbar_wait(c.qfull_bar(), run_idx & 1, c.abort_flag, kPollNs);
     if (!ok) break;
     for (int i = 0; i < r.count; ++i, ++it) {
@@ -174,7 +176,7 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int 
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const uint64_t off = (uint64_t)((ks & 3) * 2) + (ks >> 2) * hi;
-        if (REV) tc_mma(d0, k_desc + off, q_desc0 + off, idesc, ks > 0);
+        if (VOTE) tc_mma(d0, k_desc + off, q_desc0 + off, idesc, ks > 0);
         else tc_mma(d0, q_desc0 + off, k_desc + off, idesc, ks > 0);
       }
       tc_commit(c.empty_bar(st));       // K stage free once these MMAs have read it
@@ -184,7 +186,7 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int 
       if (++b == 2) { b = 0; b_phase ^= 1u; }
     }
     tc_commit(c.qempty_bar());          // Q tile free once the run's MMAs are done
-    pos = REV ? pos - r.count : pos + r.count;
+    pos += r.count;
     ++run_idx;
   }
 }
@@ -323,8 +325,8 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
   }
   if (et == 0) *c.b_layer = j;
   if (et == 0 && j < 24) trace_mark(a.trace, 9 + 2 * j);
-  for (int pos = c.end - 1; pos >= c.begin;) {
-    const Run r = locate(a, pos, c.begin, c.end, true);
+  for (int pos = c.begin; pos < c.end;) {
+    const Run r = locate(a, pos, c.begin, c.end, false);
     const int seg = r.s * a.n_kv_heads + r.g;
     const int first_cta = r.seg_tile0 / a.tiles_per_cta;
     float* lse = lse2 + 128 * (run_idx & 1);
@@ -372,7 +374,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
       ok = __all_sync(0xffffffffu, ok) != 0;
       if (!ok) continue;
       tc_fence_after();
-      const int key0 = (r.t0 + r.count - 1 - i) * kTileKeys;
+      const int key0 = (r.t0 + i) * kTileKeys;
       const uint32_t tb = c.tmem0 + lane_sel + (uint32_t)(b * 128);
       uint32_t ra[32], rb[32];
       float acc = 0.f;
@@ -398,7 +400,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
       const int jk = key0 + row;
       if (jk < r.n_hist) L.vote[a.tab.hist_at(r.s) * a.n_kv_heads + (long long)r.g * r.n_hist + jk] = acc * inv_g;
     }
-    pos -= r.count;
+    pos += r.count;
     ++run_idx;
   }
   }
