@@ -234,3 +234,51 @@ def test_overlapped_calls_match_ordinary_calls():
     torch.cuda.synchronize()
     n = int(a[1]["offsets"][-1].item())
     assert torch.equal(o["kept"][:n], a[1]["kept"][:n]) and torch.equal(b[0]["kept"][:int(a[0]["offsets"][-1])], a[0]["kept"][:int(a[0]["offsets"][-1])])
+
+
+def test_overlapped_calls_of_changing_shapes_and_streams():
+    # layers of two different shapes through one workspace, queued in lists by the overlapped entry point: a change
+    # of shape drains what is in flight before the workspace is carved up anew; results equal one call at a time
+    dev = torch.device("cuda:0")
+    base = synth.workloads()[2]
+    shapes = [synth.small_variant(base, [5000], n_layers=3, totals=[3 * 8 * 200]),
+              synth.small_variant(base, [2100, 900], n_layers=3, totals=[3 * 8 * 300])]
+    cases = []
+    for wl in shapes:
+        budgets = O.alloc_budgets(synth.inf_sc(wl).numpy(), wl.fixed, wl.totals[0])
+        for l in range(3):
+            x = synth.layer_inputs(wl, l, device=dev)
+            cases.append((wl, x, torch.tensor(budgets[l].tolist(), dtype=torch.int32, device=dev)))
+    ws_bytes = 0
+    prepared = []
+    for wl, x, bud in cases:
+        params = B.make_params(x.q_win, x.k, x.v, wl.window, wl.pool_kernel)
+        cu = wl.cu_seqlens
+        ws_bytes = max(ws_bytes, B.slkv_workspace_bytes_overlapped(params, cu))
+        cap = B.slkv_packed_rows_upper_bound(params, cu)
+        n_seg = (len(cu) - 1) * wl.n_kv_heads
+        prepared.append((params, x, cu, torch.tensor(cu, dtype=torch.int32, device=dev), bud, cap, n_seg))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+
+    def outputs():
+        return [dict(k=torch.zeros(cap, 128, dtype=torch.bfloat16, device=dev), v=torch.zeros(cap, 128, dtype=torch.bfloat16, device=dev),
+                     off=torch.zeros(n_seg + 1, dtype=torch.int32, device=dev), kept=torch.full((cap,), -1, dtype=torch.int32, device=dev),
+                     status=torch.zeros(1, dtype=torch.int32, device=dev)) for (_, _, _, _, _, cap, n_seg) in prepared]
+
+    def run(fn, outs, order):
+        for i in order:
+            params, x, cu, cu_dev, bud, cap, n_seg = prepared[i]
+            o = outs[i]
+            fn(params, x.q_win, x.k, x.v, cu_dev, cu, bud, o["k"], o["v"], o["off"], o["kept"], ws, None, o["status"])
+        B.slkv_join()
+        torch.cuda.synchronize()
+
+    order = [0, 1, 3, 4, 2, 5, 0, 3]                  # shapes alternate in runs of different lengths
+    a, b = outputs(), outputs()
+    run(B.slkv_compress, a, order)
+    run(B.slkv_compress_overlapped, b, order)
+    for i in range(len(prepared)):
+        assert int(b[i]["status"].item()) == 0
+        n = int(a[i]["off"][-1].item())
+        assert torch.equal(a[i]["off"], b[i]["off"]) and torch.equal(a[i]["kept"][:n], b[i]["kept"][:n])
+        assert torch.equal(a[i]["k"][:n], b[i]["k"][:n]) and torch.equal(a[i]["v"][:n], b[i]["v"][:n])
