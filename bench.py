@@ -35,8 +35,11 @@ TOTAL_INDEX = 1             # average budget 512 per KV head
 # DRAM bytes per key row (256 B of K) of one launch, from an ncu capture of the kernel as it stands; a kernel
 # that has changed since its capture has no entry (traffic is then reported as null)
 DRAM_TRAFFIC_PER_KEY_ROW = {
-    "k_score_fused": {"bytes": 261.7, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch "
-                      "(68.54 MB) / (8 KV heads x 32736 history rows): profiles/k_score_fused_cfg3_4layers.txt"},
+    "k_score_fused": {"bytes": 262.1, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch "
+                      "(68.65 MB) / (8 KV heads x 32736 history rows): profiles/k_score_fused_cfg3_4layers.txt"},
+    "k_score_pipe": {"bytes": 441.7, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of 8 "
+                     "layers (925.4 MB) / (8 layers x 8 KV heads x 32736 history rows): "
+                     "profiles/k_score_pipe_cfg3_8layers.txt; a launch's traffic is this x the layers it takes"},
 }
 
 
@@ -320,7 +323,10 @@ def run_cuda(args):
         kern[name] = {"launches_per_step": cnt / prof_steps, "avg_us": ms * 1e3 / cnt, "share": ms / prof_total}
     top = max(per_kernel, key=lambda n: per_kernel[n][0])
     top_us = kern[top]["avg_us"]
-    achieved = alg[top] / (top_us * 1e-6) / 1e9
+    # the two-layer score kernel takes a list of layers per launch: a launch's units are those of all its layers
+    layers_per_launch = nl / kern[top]["launches_per_step"] if top == "k_score_pipe" else 1.0
+    alg_top = alg[top] * layers_per_launch
+    achieved = alg_top / (top_us * 1e-6) / 1e9
     layer_bytes = k_scan + q_bytes + 4 * rows_avg * d * e
     flops_layer = 2 * 2.0 * wl.n_q_heads * w * n_hist * d           # two softmax passes
     exps_layer = 2.0 * wl.n_q_heads * w * n_hist
@@ -331,7 +337,7 @@ def run_cuda(args):
                 "t_ex2_us": exps_layer / (148 * 16 * f_sm) * 1e6}
     roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
-                "alg_bytes_per_launch": alg[top], "avg_launch_us": top_us,
+                "alg_bytes_per_launch": alg_top, "layers_per_launch": layers_per_launch, "avg_launch_us": top_us,
                 "layer": {"alg_bytes": layer_bytes, "us": t_layer_us,
                           "achieved": layer_bytes / (t_layer_us * 1e-6) / 1e9,
                           "frac": layer_bytes / (t_layer_us * 1e-6) / 1e9 / peaks["hbm_gbs"],
@@ -340,14 +346,14 @@ def run_cuda(args):
     # The score kernel's own ceiling is the special-function unit, not HBM: two exponentials per (query row, key)
     # at 16 ex2.approx per clock per SM need longer than streaming K once.  Reported beside the HBM figures.
     if top.startswith("k_score"):
-        n_exp = exps_layer if top in ("k_score_fused", "k_score_pipe") else exps_layer / 2
+        n_exp = (exps_layer if top in ("k_score_fused", "k_score_pipe") else exps_layer / 2) * layers_per_launch
         peak_gexp = 148 * 16 * 1965e6 / 1e9
         roofline["alu"] = {"bound": "alu", "unit": "Gexp/s", "achieved": n_exp / (top_us * 1e-6) / 1e9, "peak": peak_gexp,
                            "frac": n_exp / (top_us * 1e-6) / 1e9 / peak_gexp, "exps_per_launch": n_exp,
                            "peak_source": "148 SMs x 16 ex2.approx per clock x 1965 MHz (nominal unit count and maximum clock)"}
     tr = DRAM_TRAFFIC_PER_KEY_ROW.get(top)
     if tr:
-        roofline["traffic"] = tr["bytes"] * hkv * n_hist
+        roofline["traffic"] = tr["bytes"] * hkv * n_hist * layers_per_launch
         roofline["traffic_source"] = tr["source"]
 
     # ---- the oracle on the host cores (rank 0, N=1 only): a reported baseline, not a target

@@ -155,20 +155,30 @@ int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const 
 /*
  * slkv_compress with the calls of successive layers overlapped on the GPU (Algorithm 3, same results).
  *
- * The selection and the gather of a layer are latency-bound and need few SMs; the score kernels of the next
- * layer are bandwidth-bound and do not depend on them.  This entry point enqueues the score kernels on
- * `stream` and the selection + gather on a stream of the library's own, ordered after them by an event, so
- * that the next call's score kernels (which leave a few SMs free) run beside them.  Consequences:
- *   - The outputs of a call (k_out, v_out, offsets, kept_idx, pooled_opt, status) are NOT ordered on `stream`
- *     when the call returns.  slkv_join(stream) makes `stream` wait for every overlapped call enqueued so far
- *     on the current device (no host wait); consume outputs, or free / overwrite any input, output or
- *     workspace buffer, only behind it.  Any other slkv_* call that uses a workspace joins by itself first.
- *   - workspace must hold slkv_workspace_bytes_overlapped (two vote arrays and two source-row lists: successive calls alternate).
- *     Successive calls may share one workspace; q_win, k, v, budgets and the outputs of calls that may be in
- *     flight together must not alias each other's outputs.
- *   - The first call on a device creates two side streams and six events (no device memory).
- *   - Shapes the overlapped path does not take (more than 64 sequences, a segment with more than 32768
- *     history positions, pool_kernel > 9) run as slkv_compress does, on `stream`, after a join.
+ * The layers of a prefill are independent problems, and inside one layer the vote pass needs every key's row
+ * statistics first (the softmax of Eq. 7 runs over all keys).  This entry point therefore works on several layers
+ * at once: the score kernel takes a LIST of layers per launch and runs, in every CTA, the row-statistics pass of a
+ * layer beside the vote pass of the layer before it; the selection and the gather of a layer run on side streams
+ * of the library's own while the score kernel works on later layers.  A call queues its layer; the score kernel
+ * goes out when eight layers are queued and a ninth arrives, or at slkv_join.  Consequences:
+ *   - Nothing of a call needs to have been enqueued when it returns, and its outputs (k_out, v_out, offsets,
+ *     kept_idx, pooled_opt, status) are NOT ordered on `stream`.  slkv_join(stream) enqueues whatever is still
+ *     queued and makes `stream` wait for every overlapped call made so far on the current device (no host wait);
+ *     consume outputs, or free / overwrite any input, output or workspace buffer -- q_win, k, v, cu_seqlens_dev
+ *     and budgets included -- only behind it.  cu_seqlens_host is read during the call only.  Any other slkv_*
+ *     call that uses a workspace joins by itself first.
+ *   - workspace must hold slkv_workspace_bytes_overlapped: votes, source-row lists and row statistics for up to
+ *     eighteen layers in flight (77 MB for 8 KV heads x 32k keys; three layers' worth for shapes the list kernel
+ *     does not take).  Successive calls share one workspace; a call with another shape or workspace first drains
+ *     what is in flight.  q_win, k, v, budgets and the outputs of calls that may be in flight together must not
+ *     alias each other's outputs.
+ *   - The first call on a device creates sixteen side streams and 54 events (no device memory).
+ *   - The call sequence is stream-ordered and allocates nothing, so a step's calls plus the join can be captured
+ *     in a CUDA graph (the side streams fork from and rejoin `stream`).
+ *   - The list kernel takes bf16, head_dim 128, (n_q_heads / n_kv_heads) * window <= 128 and a multiple of 32,
+ *     at most 64 sequences, segments of at most 32768 history positions, pool_kernel <= 9.  Other shapes that the
+ *     one-CTA selection takes run one layer per score launch with the selection and gather on the side streams;
+ *     the rest run as slkv_compress does, on `stream`, after a join.
  * Arguments, results and error codes otherwise as slkv_compress.
  */
 int slkv_compress_overlapped(const slkv_params* p, const void* q_win, const void* k, const void* v,
@@ -177,7 +187,8 @@ int slkv_compress_overlapped(const slkv_params* p, const void* q_win, const void
                              int32_t* kept_idx, float* pooled_opt, int32_t* status, void* workspace,
                              size_t workspace_bytes, void* stream);
 size_t slkv_workspace_bytes_overlapped(const slkv_params* p, const int32_t* cu_seqlens_host);
-/* Orders `stream` after every overlapped call enqueued so far on the current device (see above). */
+/* Enqueues the layers still queued by slkv_compress_overlapped and orders `stream` after every overlapped call made
+ * so far on the current device (see above). */
 int slkv_join(void* stream);
 
 /* Bytes of device arena slkv_compress_host needs (inputs, outputs and workspace; 0 on invalid arguments). */
