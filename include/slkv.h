@@ -172,7 +172,7 @@ int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const 
  *     does not take).  Successive calls share one workspace; a call with another shape or workspace first drains
  *     what is in flight.  q_win, k, v, budgets and the outputs of calls that may be in flight together must not
  *     alias each other's outputs.
- *   - The first call on a device creates sixteen side streams and 54 events (no device memory).
+ *   - The first call on a device creates eighteen side streams and 54 events (no device memory).
  *   - The call sequence is stream-ordered and allocates nothing, so a step's calls plus the join can be captured
  *     in a CUDA graph (the side streams fork from and rejoin `stream`).
  *   - The list kernel takes bf16, head_dim 128, (n_q_heads / n_kv_heads) * window <= 128 and a multiple of 32,

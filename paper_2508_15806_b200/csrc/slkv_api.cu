@@ -201,7 +201,7 @@ int enqueue_votes(const Problem& pb, int path, const int32_t* cu_host, int32_t* 
 // run on the caller's stream.  Where the two-layer score kernel takes the shape, a call enqueues pass 1 of its
 // own layer together with pass 2 of the layer before (which stays "pending" until the next call or a join).
 constexpr int kSlots = 2 * kPipeMaxLayers + 2;     // layers whose votes / source rows / row statistics are live at once
-constexpr int kSideStreams = 8;   // after the last launch of a list the selections of its layers run side by side
+constexpr int kSideStreams = 9;   // after the last launch of a list the selections of its layers run side by side
 struct PendingCall {
   bool valid = false;
   Problem pb;
