@@ -30,6 +30,7 @@ namespace {
 
 constexpr int kPipeThreads = 640;        // warps 0-3: producer A, issuer A, producer B, issuer B;
                                          // warps 4-11: epilogue of stream A; warps 12-19: epilogue of stream B
+constexpr int kLeadEntries = 2;           // entries pass 1 may be ahead of the entry pass 2 has begun
 constexpr unsigned kPollNs = 64;          // pause between two polls of an mbarrier
 constexpr int kStagesA = 3;              // K tiles in flight from HBM
 constexpr int kStagesB = 2;              // K tiles in flight from L2
@@ -39,10 +40,17 @@ constexpr int kPipeTail = 512 + 1024 + 1024;   // mbarriers + flags, stat_m/stat
 constexpr int kPipeSmem = 2 * kQBytes + (kStagesA + kStagesB) * kStageBytes + kPipeTail;
 static_assert(kPipeSmem <= kSmemLimit, "shared memory of the two-stream kernel");
 
-constexpr int kMaxLay = kPipeMaxLayers + 1;     // the layer pending from the launch before + this launch's layers
+// Entries a layer may be split into (1 or 2).  Two halves the K that lies between pass 1 and pass 2, and pass 2 then
+// finds it in L2 (measured: 299 B of DRAM traffic per key row instead of 442, SM clock 1.82 instead of 1.64 GHz under
+// the power cap) but pays for twice the merges, Q reloads and waits for the other CTAs: 35.7 against 34.3 us per
+// layer.  One it is.
+constexpr int kMaxGroups = 1;
+constexpr int kMaxLay = kPipeMaxLayers * kMaxGroups + 1;   // the entry pending from the launch before + this launch's
 constexpr int kCountWords = kMaxLay + 1;        // per launch: one publish counter per layer + one exit counter
 constexpr int kCountSlots = 64;                 // launches whose counters are live at once
 
+// One entry of a launch's list: a layer, or one group of consecutive segments of a layer (a range of the layer's
+// flat tile list).  Smaller entries keep less K between pass 1 and pass 2.
 struct LayerDesc {
   alignas(64) CUtensorMap tm_q;
   alignas(64) CUtensorMap tm_k;
@@ -50,6 +58,8 @@ struct LayerDesc {
   float* part_z;
   float* vote;
   int32_t* status;
+  int tile_begin, tile_end;    // the entry's tiles in the layer's tile list; CTA b takes tiles_per_cta of them from
+                               // tile_begin + b * tiles_per_cta
 };
 struct PipeArgs {
   TcArgs base;                 // tables, shapes, schedule, scale: the same for every layer of the launch
@@ -67,7 +77,7 @@ __device__ unsigned g_layer_published[kCountSlots * kCountWords];
 // One stream's resources inside the CTA.
 struct StreamCtx {
   uint32_t q_smem, k_smem, bar0, tmem0;
-  int n_stages, begin, end;
+  int n_stages;
   volatile int* abort_flag;
   volatile int* b_layer;       // CTA-wide: the layer whose pass 2 this CTA's epilogue has begun
   __device__ __forceinline__ uint32_t full_bar(int st) const { return bar0 + 8u * st; }
@@ -91,6 +101,11 @@ __device__ __forceinline__ float sum_ex2_32_mufu(const uint32_t (&r)[32], float 
   }
   return (s0 + s1) + (s2 + s3);
 }
+// this CTA's tiles of an entry
+__device__ __forceinline__ void entry_range(const TcArgs& a, const LayerDesc& L, int& begin, int& end) {
+  begin = min(L.tile_begin + (int)blockIdx.x * a.tiles_per_cta, L.tile_end);
+  end = min(begin + a.tiles_per_cta, L.tile_end);
+}
 __device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(kEpiThreads) : "memory"); }
 
 // ---- one thread: TMA loads of the stream's Q tiles and K tiles ------------------------------------------
@@ -110,7 +125,7 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
       // before, so it cannot deadlock): the two streams then share the SM to the end instead of pass 2 running on
       // alone, on half the epilogue warps, after pass 1 has raced through the list.
       const unsigned long long t0 = now_ns();
-      for (unsigned spin = 1; *c.b_layer < j - 2; ++spin) {
+      for (unsigned spin = 1; *c.b_layer < j - kLeadEntries; ++spin) {
         if ((spin & 63u) == 0 && (*c.abort_flag || now_ns() - t0 > kWaitLimitNs)) { *c.abort_flag = 1; ok = false; break; }
         __nanosleep(100);
       }
@@ -118,8 +133,10 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
     }
     const CUtensorMap* tm_q = &lay[j].tm_q;
     const CUtensorMap* tm_k = &lay[j].tm_k;
-    for (int pos = c.begin; pos < c.end && ok;) {
-      const Run r = locate(a, pos, c.begin, c.end, false);
+    int begin, end;
+    entry_range(a, lay[j], begin, end);
+    for (int pos = begin; pos < end && ok;) {
+      const Run r = locate(a, pos, begin, end, false);
       ok = mbar_wait(c.qempty_bar(), (run_idx & 1) ^ 1, c.abort_flag, kPollNs);        // the run before is done with Q
       if (!ok) break;
       mbar_expect_tx(c.qfull_bar(), 2u * (uint32_t)a.R * 128u);
@@ -154,7 +171,7 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
 
 // ---- one thread: the stream's MMAs, one 128 x 128 x 128 product per tile into one of two accumulators --------
 template <bool VOTE>
-__device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int first, int last) {
+__device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, const LayerDesc* lay, int first, int last) {
   // pass 1: D[row, key] = Q K^T (A = Q, B = K); pass 2: D[key, row] = K Q^T (A = K, B = Q, N = R)
   const uint32_t idesc = VOTE ? instr_desc(kTileKeys, a.R) : instr_desc(128, kTileKeys);
   const uint64_t q_desc0 = smem_desc(c.q_smem), k_desc0 = smem_desc(c.k_smem);
@@ -163,9 +180,11 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int 
   uint32_t st_phase = 0, b_phase = 0;
   uint64_t k_desc = k_desc0;
   bool ok = true;
-  for (int j = first; j <= last && ok; ++j)
-  for (int pos = c.begin; pos < c.end && ok;) {
-    const Run r = locate(a, pos, c.begin, c.end, false);
+  for (int j = first; j <= last && ok; ++j) {
+  int begin, end;
+  entry_range(a, lay[j], begin, end);
+  for (int pos = begin; pos < end && ok;) {
+    const Run r = locate(a, pos, begin, end, false);
     ok = mbar_wait(c.qfull_bar(), run_idx & 1, c.abort_flag, kPollNs);
     if (!ok) break;
     for (int i = 0; i < r.count; ++i, ++it) {
@@ -189,6 +208,7 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, int 
     pos += r.count;
     ++run_idx;
   }
+  }
 }
 
 // ---- 256 threads: pass 1, row statistics (stream A) ----------------------------------------------------------
@@ -202,10 +222,12 @@ __device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& 
   bool ok = true;
   for (int j = pa.a_first; j <= pa.a_last; ++j) {
   const LayerDesc& L = pa.lay[j];
-  for (int pos = c.begin; pos < c.end;) {
-    const Run r = locate(a, pos, c.begin, c.end, false);
+  int begin, end;
+  entry_range(a, L, begin, end);
+  for (int pos = begin; pos < end;) {
+    const Run r = locate(a, pos, begin, end, false);
     const int seg = r.s * a.n_kv_heads + r.g;
-    const int first_cta = r.seg_tile0 / a.tiles_per_cta;
+    const int first_cta = (r.seg_tile0 - L.tile_begin) / a.tiles_per_cta;
     float m = 0.f, z = 0.f;                                   // fixed reference 0 on the fast path
     for (int i = 0; i < r.count; ++i, ++it) {
       if ((it & 1) != wg) continue;
@@ -325,15 +347,17 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
   }
   if (et == 0) *c.b_layer = j;
   if (et == 0 && j < 24) trace_mark(a.trace, 9 + 2 * j);
-  for (int pos = c.begin; pos < c.end;) {
-    const Run r = locate(a, pos, c.begin, c.end, false);
+  int begin, end;
+  entry_range(a, L, begin, end);
+  for (int pos = begin; pos < end;) {
+    const Run r = locate(a, pos, begin, end, false);
     const int seg = r.s * a.n_kv_heads + r.g;
-    const int first_cta = r.seg_tile0 / a.tiles_per_cta;
+    const int first_cta = (r.seg_tile0 - L.tile_begin) / a.tiles_per_cta;
     float* lse = lse2 + 128 * (run_idx & 1);
     {
       // merge the per-CTA partials of this segment into the rows' log-sum-exp (log2 units): two neighbouring
       // lanes share a row (even / odd slots), all loads in flight before the first use
-      const int n_slots = (r.seg_tile0 + r.tiles_seg - 1) / a.tiles_per_cta - first_cta + 1;
+      const int n_slots = (r.seg_tile0 - L.tile_begin + r.tiles_seg - 1) / a.tiles_per_cta - first_cta + 1;
       const int rr = (et >> 1) < R ? (et >> 1) : -1;
       const int half = et & 1;
       float M = -INFINITY, Z = 0.f;
@@ -441,8 +465,6 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   cb.n_stages = kStagesB;
   ca.abort_flag = cb.abort_flag = &abort_sh;
   ca.b_layer = cb.b_layer = &b_layer_sh;
-  ca.begin = cb.begin = min(blockIdx.x * a.tiles_per_cta, a.total_tiles);
-  ca.end = cb.end = min(ca.begin + a.tiles_per_cta, a.total_tiles);
 
   if (tid == 0) trace_mark(a.trace, 0);
   if (tid == 0 && a.trace) a.trace[(size_t)blockIdx.x * kTraceSlots + 60] = (unsigned long long)clock64();
@@ -486,11 +508,11 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   if (warp == 0) {
     if (lane == 0 && has_a) producer<false>(ca, a, pa.lay, pa.a_first, pa.a_last, pa.a_first);
   } else if (warp == 1) {
-    if (lane == 0 && has_a) issuer<false>(ca, a, pa.a_first, pa.a_last);
+    if (lane == 0 && has_a) issuer<false>(ca, a, pa.lay, pa.a_first, pa.a_last);
   } else if (warp == 2) {
     if (lane == 0 && has_b) producer<true>(cb, a, pa.lay, pa.b_first, pa.b_last, 1);   // layer 0 was read before
   } else if (warp == 3) {
-    if (lane == 0 && has_b) issuer<true>(cb, a, pa.b_first, pa.b_last);
+    if (lane == 0 && has_b) issuer<true>(cb, a, pa.lay, pa.b_first, pa.b_last);
   } else if (warp < 12) {
     if (has_a) {
       pdl_wait();
@@ -563,21 +585,43 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
   pa.base = any->a;
   pa.base.part_m = pa.base.part_z = pa.base.vote = nullptr;
   pa.base.status = nullptr;
-  auto fill = [&](int j, const TcPlan* p) {
+  // A layer goes in as one entry, or as two (its first and second half of the segments) when the halves are whole
+  // segments and equal: pass 2 of an entry then follows its pass 1 after half a layer's time and half a layer's K.
+  const TcArgs& sh = any->a;
+  const int total = sh.total_tiles;
+  int groups = 1;
+  if (kMaxGroups >= 2 && total % 2 == 0 && sh.tab.n_inline > 0) {
+    const int mid = total / 2;
+    for (int q = 0; q < sh.tab.n_inline && groups == 1; ++q) {
+      const int t_seq = sh.tab.tile_off[q + 1] - sh.tab.tile_off[q];
+      for (int g = 0; g < sh.n_kv_heads; ++g)
+        if (sh.n_kv_heads * sh.tab.tile_off[q] + g * t_seq == mid) { groups = 2; break; }
+    }
+  }
+  int n_cta = any->n_cta;
+  if (groups == 2) {
+    const int per_group = total / 2;
+    int tpc = (per_group + n_cta - 1) / n_cta;
+    pa.base.tiles_per_cta = tpc;
+    n_cta = (per_group + tpc - 1) / tpc;
+  }
+  auto fill = [&](int j, const TcPlan* p, int group) {
     pa.lay[j].tm_q = p->tm_q; pa.lay[j].tm_k = p->tm_k;
     pa.lay[j].part_m = p->a.part_m; pa.lay[j].part_z = p->a.part_z; pa.lay[j].vote = p->a.vote;
     pa.lay[j].status = p->a.status;
+    pa.lay[j].tile_begin = groups == 2 ? group * (total / 2) : 0;
+    pa.lay[j].tile_end = groups == 2 ? (group + 1) * (total / 2) : total;
   };
   const bool has_pending = pending && pending->n_cta > 0;
-  if (has_pending) fill(0, pending);
+  if (has_pending) fill(0, pending, groups - 1);      // what is pending of a layer is its last group
   int n_live = 0;
   for (int i = 0; i < n_a; ++i)
-    if (a[i]->n_cta > 0) fill(++n_live, a[i]);      // layers without history take no part
+    if (a[i]->n_cta > 0)
+      for (int g = 0; g < groups; ++g) fill(++n_live, a[i], g);     // layers without history take no part
   pa.a_first = 1; pa.a_last = n_live;
   pa.b_first = has_pending ? 0 : 1;
   pa.b_last = finish ? n_live : n_live - 1;
   if (pa.a_first > pa.a_last && pa.b_first > pa.b_last) return cudaSuccess;
-  const int n_cta = any->n_cta;
   pa.base.trace = tensor_trace_buffer(0, n_cta);
   // counters of this launch: a slot of the table, zeroed on the stream before the kernel
   static std::atomic<unsigned> launch_seq{0};
