@@ -265,18 +265,27 @@ def test_overlapped_calls_of_changing_shapes_and_streams():
                      off=torch.zeros(n_seg + 1, dtype=torch.int32, device=dev), kept=torch.full((cap,), -1, dtype=torch.int32, device=dev),
                      status=torch.zeros(1, dtype=torch.int32, device=dev)) for (_, _, _, _, _, cap, n_seg) in prepared]
 
-    def run(fn, outs, order):
-        for i in order:
+    side = torch.cuda.Stream()
+
+    def run(fn, outs, order, streams):
+        torch.cuda.synchronize()
+        for n, i in enumerate(order):
             params, x, cu, cu_dev, bud, cap, n_seg = prepared[i]
             o = outs[i]
-            fn(params, x.q_win, x.k, x.v, cu_dev, cu, bud, o["k"], o["v"], o["off"], o["kept"], ws, None, o["status"])
+            fn(params, x.q_win, x.k, x.v, cu_dev, cu, bud, o["k"], o["v"], o["off"], o["kept"], ws, None, o["status"],
+               streams[n % len(streams)])
         B.slkv_join()
         torch.cuda.synchronize()
 
     order = [0, 1, 3, 4, 2, 5, 0, 3]                  # shapes alternate in runs of different lengths
-    a, b = outputs(), outputs()
-    run(B.slkv_compress, a, order)
-    run(B.slkv_compress_overlapped, b, order)
+    a, b, c = outputs(), outputs(), outputs()
+    run(B.slkv_compress, a, order, [None])
+    run(B.slkv_compress_overlapped, b, order, [None])
+    run(B.slkv_compress_overlapped, c, order, [None, None, side])     # every third call on another stream
+    for i in range(len(prepared)):
+        n = int(a[i]["off"][-1].item())
+        assert int(c[i]["status"].item()) == 0 and torch.equal(a[i]["kept"][:n], c[i]["kept"][:n])
+        assert torch.equal(a[i]["k"][:n], c[i]["k"][:n]) and torch.equal(a[i]["v"][:n], c[i]["v"][:n])
     for i in range(len(prepared)):
         assert int(b[i]["status"].item()) == 0
         n = int(a[i]["off"][-1].item())
