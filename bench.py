@@ -35,10 +35,10 @@ TOTAL_INDEX = 1             # average budget 512 per KV head
 # DRAM bytes per key row (256 B of K) of one launch, from an ncu capture of the kernel as it stands; a kernel
 # that has changed since its capture has no entry (traffic is then reported as null)
 DRAM_TRAFFIC_PER_KEY_ROW = {
-    "k_score_fused": {"bytes": 262.1, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch "
-                      "(68.65 MB) / (8 KV heads x 32736 history rows): profiles/k_score_fused_cfg3_4layers.txt"},
-    "k_score_pipe": {"bytes": 441.7, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of 8 "
-                     "layers (925.4 MB) / (8 layers x 8 KV heads x 32736 history rows): "
+    "k_score_fused": {"bytes": 261.7, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch "
+                      "(68.53 MB) / (8 KV heads x 32736 history rows): profiles/k_score_fused_cfg3_4layers.txt"},
+    "k_score_pipe": {"bytes": 442.6, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of 8 "
+                     "layers (927.4 MB) / (8 layers x 8 KV heads x 32736 history rows): "
                      "profiles/k_score_pipe_cfg3_8layers.txt; a launch's traffic is this x the layers it takes"},
 }
 
