@@ -492,7 +492,8 @@ Schedule schedule_of(const Problem& pb, const int32_t* cu_host) {
   sc.tiles_per_cta = sc.total_tiles > 0 ? (sc.total_tiles + sms - 1) / sms : 1;
   // A CTA whose range straddles two segments reloads Q in mid-stream (a pipeline bubble of a few microseconds) and
   // holds everybody else up wherever CTAs wait for one another.  When all segments have the same number of tiles
-  // and a slightly larger share per CTA divides it, the ranges line up with the segments.
+  // and a share per CTA at most 1/15 larger divides it, the ranges line up with the segments (more than that costs
+  // more than the bubbles).
   if (pb.p.n_seqs > 0 && sc.total_tiles > 0) {
     const long long per_seg = tiles / pb.p.n_seqs;
     bool equal = per_seg * pb.p.n_seqs == tiles;
@@ -501,7 +502,7 @@ Schedule schedule_of(const Problem& pb, const int32_t* cu_host) {
       equal = nh > 0 && (nh + kTileKeys - 1) / kTileKeys == per_seg;
     }
     if (equal && per_seg >= sc.tiles_per_cta)
-      for (int t = sc.tiles_per_cta; t <= sc.tiles_per_cta + sc.tiles_per_cta / 8 + 1; ++t)
+      for (int t = sc.tiles_per_cta; (t - sc.tiles_per_cta) * 15 <= sc.tiles_per_cta; ++t)      // at most 1/15 more tiles
         if (per_seg % t == 0) { sc.tiles_per_cta = t; break; }
   }
   sc.n_cta = sc.total_tiles > 0 ? (sc.total_tiles + sc.tiles_per_cta - 1) / sc.tiles_per_cta : 0;
