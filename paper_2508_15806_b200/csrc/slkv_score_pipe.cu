@@ -250,7 +250,7 @@ __device__ __forceinline__ void epilogue_rows(const StreamCtx& c, const TcArgs& 
         if (nv >= 32) {
           const float zc = sum_ex2_32_mufu(rr, sc, m);
           const float zn = z + zc;
-          if (zn < INFINITY && zc > 0.f) { z = zn; return; }
+          if (zn < INFINITY && zn > kTinySum) { z = zn; return; }
         }
         // rare: a copy goes through the stack so that the chunk registers themselves never have to
         uint32_t tmp[32];

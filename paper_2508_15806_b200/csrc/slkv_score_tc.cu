@@ -298,7 +298,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               }
 #pragma unroll
               for (int u = 0; u < 12; ++u)
-                if (m12[u] > -INFINITY) {
+                if (z12[u] > 0.f) {                                    // empty partials carry z = 0
                   const float Mn = fmaxf(M, m12[u]);
                   Z = Z * ex2(M - Mn) + z12[u] * ex2(m12[u] - Mn);      // ex2(-inf) = 0 covers the first term
                   M = Mn;
@@ -350,7 +350,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 if (c0 + 64 < kTileKeys) tc_ld32_issue(tcol + c0 + 64, ra);
                 zt += sum_ex2_32(rb, sc, m);
               }
-              if (zt < INFINITY && zt > 0.f) z = zt; else exact = true;
+              if (zt < INFINITY && zt > kTinySum) z = zt; else exact = true;
             }
             if (exact) tile_row_stats_exact(tcol, sc, n_valid, m, z);
             m_run[mt] = m; z_run[mt] = z;
@@ -414,9 +414,11 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const int rr = mt * 128 + row;
             if (rr < R) {
               const float m1 = stat_m[row], z1 = stat_z[row];
-              const float M = fmaxf(m_run[mt], m1);
+              const bool h0 = z_run[mt] > 0.f, h1 = z1 > 0.f;      // a warpgroup without a tile in this run has z = 0
+              const float M = h0 && h1 ? fmaxf(m_run[mt], m1) : (h0 ? m_run[mt] : m1);
               float Z = 0.f;
-              if (M > -INFINITY) Z = z_run[mt] * ex2(m_run[mt] - M) + z1 * ex2(m1 - M);
+              if (h0) Z += z_run[mt] * ex2(m_run[mt] - M);
+              if (h1) Z += z1 * ex2(m1 - M);
               a.part_m[((long long)seg * a.slot_stride + slot) * R + rr] = M;
               a.part_z[((long long)seg * a.slot_stride + slot) * R + rr] = Z;
             }

@@ -24,6 +24,9 @@ constexpr int kTraceSlots = 64;               // per CTA: 0 start, 1 set-up done
                                                // past its wait for the launch before, 2 first accumulator of A ready,
                                                // 3 first log-sum-exps of B merged, 5 / 6 epilogue of A / B done, 4 end,
                                                // 8+2j / 9+2j layer j published by A / begun by B, 60 / 61 SM cycle counter at start / end
+// A row sum under the fixed reference that is not above this has underflowed (terms below fp32's range are flushed
+// to zero, or clamped to 2^-125 on the polynomial path): the exact path then moves the reference.
+constexpr float kTinySum = 1e-30f;
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;   // 1 s per wait
 
 
@@ -249,8 +252,11 @@ __device__ __noinline__ void tile_row_stats_exact(uint32_t tcol, float sc, int n
     if (c0 >= n_valid) break;
     tc_ld32_issue(tcol + c0, ra);
     tc_ld_wait(ra);
-    const float mn = fmaxf(m, max_32(ra, n_valid - c0) * sc);
-    z *= ex2(m - mn);
+    // the reference a row starts with (0) is a guess, not a score: while nothing has been summed it gives way to
+    // the first maximum seen, however low
+    const float mx = max_32(ra, n_valid - c0) * sc;
+    const float mn = z > 0.f ? fmaxf(m, mx) : mx;
+    z = z > 0.f ? z * ex2(m - mn) : 0.f;
     m = mn;
     float zc = 0.f;
 #pragma unroll

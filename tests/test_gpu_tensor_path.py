@@ -72,3 +72,67 @@ def test_strided_views_on_tensor_path():
     assert int(status.item()) == 0
     ref = P.oracle_pooled(q_hm.permute(0, 2, 1, 3).contiguous(), kv[:, 0].contiguous(), cu, w, 7)
     P.assert_pooled_close(pooled.cpu().numpy(), ref, cu, Hkv, w)
+
+
+def overlapped_result(q, k, v, cu, bud, w, p, repeats=2):
+    """The layer `repeats` times through slkv_compress_overlapped + slkv_join; host results of the last call."""
+    dev = torch.device("cuda:0")
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    cu = [int(x) for x in cu]
+    params = B.make_params(qd, kd, vd, w, p, B.SLKV_POOL_MAX, B.SLKV_PATH_TENSOR)
+    cap = B.slkv_packed_rows_upper_bound(params, cu)
+    n_seg = (len(cu) - 1) * k.shape[1]
+    cu_dev = torch.tensor(cu, dtype=torch.int32, device=dev)
+    budd = torch.tensor(list(bud), dtype=torch.int32, device=dev)
+    ws = torch.empty(B.slkv_workspace_bytes_overlapped(params, cu), dtype=torch.uint8, device=dev)
+    n_pool = B.slkv_pooled_elems(params, cu)
+    outs = []
+    for _ in range(repeats):
+        o = dict(k_out=torch.zeros(cap, 128, dtype=k.dtype, device=dev), v_out=torch.zeros(cap, 128, dtype=k.dtype, device=dev),
+                 offsets=torch.full((n_seg + 1,), -1, dtype=torch.int32, device=dev),
+                 kept=torch.full((cap,), -1, dtype=torch.int32, device=dev),
+                 pooled=torch.full((n_pool,), float("nan"), dtype=torch.float32, device=dev),
+                 status=torch.zeros(1, dtype=torch.int32, device=dev))
+        B.slkv_compress_overlapped(params, qd, kd, vd, cu_dev, cu, budd, o["k_out"], o["v_out"], o["offsets"], o["kept"], ws,
+                                   o["pooled"], o["status"])
+        outs.append(o)
+    B.slkv_join()
+    torch.cuda.synchronize()
+    o = outs[-1]
+    assert int(o["status"].item()) == 0
+    return {"offsets": o["offsets"].cpu().numpy().astype(np.int64), "kept_idx": o["kept"].cpu().numpy().astype(np.int64),
+            "k_out": o["k_out"].cpu(), "v_out": o["v_out"].cpu(), "pooled": o["pooled"].cpu().numpy()}
+
+
+@pytest.mark.parametrize("kind", ["overflow", "underflow"])
+def test_extreme_logits_on_both_entry_points(kind):
+    # overflow: a few keys 120 logits above the bulk (2^x overflows fp32 under a fixed reference of 0);
+    # underflow: every logit of every row near -150 (every 2^x underflows under that reference).
+    # Both must leave the fixed-reference fast path for the exact one, in the single-layer kernel (slkv_compress)
+    # and in the two-stream kernel (slkv_compress_overlapped).
+    q, k, v, cu = rand_case(8, 2, 16, [1500, 700], seed=21)
+    qf, kf = q.float(), k.float()
+    qf[..., 0] += 41.0
+    if kind == "underflow":
+        kf[..., 0] -= 41.0                       # adds -41 * 41 / sqrt(128) = -148.6 to every logit
+    else:
+        for t in (5, 333, 1499, 1500 + 77):
+            kf[t, :, 0] += 33.0                  # +119.6 on these keys
+    q, k = qf.to(torch.bfloat16), kf.to(torch.bfloat16)
+    bud = [200, 64]
+    w, p = 16, 5
+    ref = P.oracle_pooled(q, k, cu, w, p)
+    ordinary = P.gpu_compress(q, k, v, cu, bud, w, p, score_path=B.SLKV_PATH_TENSOR)
+    assert ordinary["status"] == 0
+    overlapped = overlapped_result(q, k, v, cu, bud, w, p)
+    for gpu in (ordinary, overlapped):
+        P.assert_pooled_close(gpu["pooled"], ref, cu, k.shape[1], w)
+        if kind == "underflow":
+            P.assert_selection_valid(gpu, ref, cu, bud, w, k, v)
+        else:
+            # next to keys 120 logits up every other probability is below fp32's range (exp(-120)), so the order of
+            # the rest cannot be compared; the planted keys and their pooling neighbourhoods must be kept
+            for h in range(2):
+                a, b = gpu["offsets"][h], gpu["offsets"][h + 1]
+                kept = set(gpu["kept_idx"][a:b].tolist())
+                assert {3, 4, 5, 6, 7, 331, 332, 333, 334, 335} <= kept
