@@ -136,3 +136,23 @@ def test_extreme_logits_on_both_entry_points(kind):
                 a, b = gpu["offsets"][h], gpu["offsets"][h + 1]
                 kept = set(gpu["kept_idx"][a:b].tolist())
                 assert {3, 4, 5, 6, 7, 331, 332, 333, 334, 335} <= kept
+
+
+@pytest.mark.parametrize("lens", [
+    [5, 16, 9],                                  # no sequence longer than the window: nothing to score
+    [40 + 3 * i for i in range(70)],             # more sequences than the per-sequence tables in kernel parameters hold
+    [16 + 128 * 4, 17, 16 + 128],                # histories of whole key tiles beside a one-key history
+])
+def test_overlapped_entry_point_on_degenerate_batches(lens):
+    w, p = 16, 3
+    q, k, v, cu = rand_case(8, 2, w, lens, seed=len(lens))
+    bud = [w + 9, 3 * w]
+    ordinary = P.gpu_compress(q, k, v, cu, bud, w, p, score_path=B.SLKV_PATH_TENSOR)
+    assert ordinary["status"] == 0
+    ref = P.oracle_pooled(q, k, cu, w, p)
+    P.assert_selection_valid(ordinary, ref, cu, bud, w, k, v)
+    overlapped = overlapped_result(q, k, v, cu, bud, w, p, repeats=3)
+    n = int(ordinary["offsets"][-1])
+    assert np.array_equal(overlapped["offsets"], ordinary["offsets"])
+    assert np.array_equal(overlapped["kept_idx"][:n], ordinary["kept_idx"][:n])
+    assert torch.equal(overlapped["k_out"][:n], ordinary["k_out"][:n]) and torch.equal(overlapped["v_out"][:n], ordinary["v_out"][:n])
