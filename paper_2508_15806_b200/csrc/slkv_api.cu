@@ -216,6 +216,7 @@ struct PendingCall {
   float* pooled_opt = nullptr;
   int32_t* status = nullptr;
   cudaStream_t st = nullptr;
+  std::vector<int32_t> cu_host;          // the call's cu_seqlens_host (the caller's copy is only valid during the call)
 };
 struct ShapeSig {                                  // calls in flight together must carve the workspace alike
   const void* ws = nullptr;
@@ -307,6 +308,14 @@ cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pip
 cudaError_t launch_queue(OverlapState* os, int n, bool finish, int* launches) {
   if (n > (int)os->queue.size()) n = (int)os->queue.size();
   if (n == 0 && !(finish && os->pending.valid)) return cudaSuccess;
+  if (n == 1 && finish && !os->pending.valid) {
+    // a single layer and nothing to pair it with: both passes in the single-layer kernel
+    const PendingCall& c = os->queue[0];
+    cudaError_t e1 = launch_score_tensor(c.pb, c.cu_host.data(), c.status, c.st, launches);
+    if (e1 == cudaSuccess) e1 = enqueue_tail(os, c, false, launches);
+    os->queue.clear();
+    return e1;
+  }
   const TcPlan* plans[kPipeMaxLayers];
   for (int i = 0; i < n; ++i) plans[i] = &os->queue[i].plan;
   cudaStream_t st = n > 0 ? os->queue[0].st : os->pending.st;
@@ -409,6 +418,7 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
     cur.valid = true; cur.pb = pb; cur.slot = slot; cur.budgets = budgets; cur.k_out = k_out; cur.v_out = v_out;
     cur.capacity = capacity; cur.offsets = offsets; cur.kept_idx = kept_idx; cur.pooled_opt = pooled_opt;
     cur.status = status; cur.st = st;
+    cur.cu_host.assign(cu_host, cu_host + pb.p.n_seqs + 1);
     bool pipe = path == SLKV_PATH_TENSOR && score_pipe_supported(pb);
     if (pipe) {
       e = plan_score_tensor(pb, cu_host, status, &cur.plan);
