@@ -234,6 +234,7 @@ struct OverlapState {
   cudaEvent_t selected[kSlots] = {};     // recorded on a selection stream after the selection
   cudaEvent_t done[kSlots] = {};         // recorded on the gather stream after the gather
   bool in_flight[kSlots] = {};
+  bool wait_done[kSlots] = {};           // the slot's next selection must first wait for the gather that had the slot
   unsigned seq = 0;
   std::vector<PendingCall> queue;        // layers whose score kernel is not launched yet (at most kPipeMaxLayers + 1)
   PendingCall pending;                   // pass 1 launched, pass 2 not
@@ -274,18 +275,23 @@ cudaError_t overlap_state(OverlapState** out) {
 // its source-row list by that layer's gather.
 cudaError_t claim_slot(OverlapState* os, int slot, cudaStream_t st) {
   if (!os->in_flight[slot]) return cudaSuccess;
-  cudaError_t e = cudaStreamWaitEvent(st, os->selected[slot], 0);
-  if (e == cudaSuccess) e = cudaStreamWaitEvent(os->side_select[slot % kSideStreams], os->done[slot], 0);
-  return e;
+  os->wait_done[slot] = true;
+  return cudaStreamWaitEvent(st, os->selected[slot], 0);
 }
 
-// The votes of layer `c` are enqueued on c.st: selection on a side stream, gather on another.
-cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pipe, int* launches) {
+// The votes of layer `c` are enqueued on c.st: selection on a side stream, gather on another.  While more score
+// launches follow, two selections at a time (a selection takes one SM per segment, and a score launch whose CTAs wait
+// for one another starts only when all of them fit beside what is running); `wide`: nothing follows, all side
+// streams.
+cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pipe, bool wide, int* launches) {
   const int slot = c.slot;
-  cudaStream_t sel = os->side_select[slot % kSideStreams], gat = os->side_gather[slot % kSideStreams];
+  const int si = wide ? slot % kSideStreams : slot % 2;
+  cudaStream_t sel = os->side_select[si], gat = os->side_gather[si];
   if (g_prof_on) sel = gat = c.st;       // per-kernel timing: one stream, so that the event pairs do not overlap
   cudaError_t e = cudaEventRecord(os->scored[slot], c.st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(sel, os->scored[slot], 0);
+  if (e == cudaSuccess && os->wait_done[slot]) e = cudaStreamWaitEvent(sel, os->done[slot], 0);
+  os->wait_done[slot] = false;
   if (e != cudaSuccess) return e;
   e = launch_select_cta(c.pb, c.pooled_opt, c.budgets, c.offsets, c.kept_idx, c.capacity, c.status, sel, launches);
   if (e != cudaSuccess) return e;
@@ -312,7 +318,7 @@ cudaError_t launch_queue(OverlapState* os, int n, bool finish, int* launches) {
     // a single layer and nothing to pair it with: both passes in the single-layer kernel
     const PendingCall& c = os->queue[0];
     cudaError_t e1 = launch_score_tensor(c.pb, c.cu_host.data(), c.status, c.st, launches);
-    if (e1 == cudaSuccess) e1 = enqueue_tail(os, c, false, launches);
+    if (e1 == cudaSuccess) e1 = enqueue_tail(os, c, false, true, launches);
     os->queue.clear();
     return e1;
   }
@@ -320,10 +326,10 @@ cudaError_t launch_queue(OverlapState* os, int n, bool finish, int* launches) {
   for (int i = 0; i < n; ++i) plans[i] = &os->queue[i].plan;
   cudaStream_t st = n > 0 ? os->queue[0].st : os->pending.st;
   cudaError_t e = launch_score_pipe(os->pending.valid ? &os->pending.plan : nullptr, plans, n, finish, st, launches);
-  if (e == cudaSuccess && os->pending.valid) e = enqueue_tail(os, os->pending, true, launches);
+  if (e == cudaSuccess && os->pending.valid) e = enqueue_tail(os, os->pending, true, finish, launches);
   os->pending.valid = false;
   const int n_voted = finish ? n : n - 1;
-  for (int i = 0; i < n_voted && e == cudaSuccess; ++i) e = enqueue_tail(os, os->queue[i], true, launches);
+  for (int i = 0; i < n_voted && e == cudaSuccess; ++i) e = enqueue_tail(os, os->queue[i], true, finish, launches);
   if (!finish && n > 0) os->pending = os->queue[n - 1];
   os->queue.erase(os->queue.begin(), os->queue.begin() + n);
   return e;
@@ -443,7 +449,7 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
     } else {
       rc = enqueue_votes(pb, path, cu_host, status, st, &launches);
       if (rc != SLKV_OK) return rc;
-      e = enqueue_tail(os, cur, false, &launches);
+      e = enqueue_tail(os, cur, false, false, &launches);
       if (e != cudaSuccess) return cuda_fail(e);
     }
     g_last_launches = launches;
