@@ -20,6 +20,7 @@
 #include <cuda.h>
 
 #include <atomic>
+#include <cstdlib>
 #include <cstring>
 
 #include "slkv_internal.cuh"
@@ -562,6 +563,26 @@ bool score_pipe_supported(const Problem& pb) {
 cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int n_a, bool finish, cudaStream_t st,
                               int* launches) {
   if (n_a > kPipeMaxLayers) return cudaErrorInvalidValue;
+  // Without cooperative launches (refused once on this device) no launch may hold both passes of a layer: one layer's
+  // pass 1 per launch, beside pass 2 of the layer before.
+  static thread_local bool no_coop[64] = {};
+  static const bool env_no_coop = [] {                // SLKV_NO_COOPERATIVE=1: behave as if they were refused (tests)
+    const char* v = std::getenv("SLKV_NO_COOPERATIVE");
+    return v && v[0] == '1';
+  }();
+  {
+    int d = 0;
+    if (env_no_coop && cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < 64) no_coop[d] = true;
+    if (cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < 64 && no_coop[d] && (n_a > 1 || (n_a == 1 && finish))) {
+      const TcPlan* prev = pending;
+      for (int i = 0; i < n_a; ++i) {
+        cudaError_t e1 = launch_score_pipe(prev, a + i, 1, false, st, launches);
+        if (e1 != cudaSuccess) return e1;
+        prev = a[i];
+      }
+      return finish ? launch_score_pipe(prev, nullptr, 0, true, st, launches) : cudaSuccess;
+    }
+  }
   const TcPlan* any = pending && pending->n_cta > 0 ? pending : nullptr;
   for (int i = 0; i < n_a && !any; ++i)
     if (a[i]->n_cta > 0) any = a[i];
@@ -662,10 +683,13 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
       if (waits_inside && with_pdl) pc = 1;
       return cudaSuccess;
     }
-    if (!(waits_inside && with_pdl) || pc == 1) return le;
+    if (!waits_inside) return le;
     (void)cudaGetLastError();                         // not a sticky error: the launch was refused
     --*launches;
-    pc = -1;                                          // once more without dependent launch
+    if (with_pdl && pc != 1) { pc = -1; continue; }   // once more without dependent launch
+    // cooperative launches do not work here: the list goes out one layer per launch from now on
+    no_coop[dev < 64 ? dev : 0] = true;
+    return launch_score_pipe(pending, a, n_a, finish, st, launches);
   }
   return cudaErrorLaunchFailure;
 }

@@ -291,3 +291,19 @@ def test_overlapped_calls_of_changing_shapes_and_streams():
         n = int(a[i]["off"][-1].item())
         assert torch.equal(a[i]["off"], b[i]["off"]) and torch.equal(a[i]["kept"][:n], b[i]["kept"][:n])
         assert torch.equal(a[i]["k"][:n], b[i]["k"][:n]) and torch.equal(a[i]["v"][:n], b[i]["v"][:n])
+
+
+def test_overlapped_calls_without_cooperative_launches():
+    # where the device refuses cooperative launches the score kernel takes one layer's pass 1 per launch (beside
+    # pass 2 of the layer before); SLKV_NO_COOPERATIVE=1 makes the library behave that way.  The switch is read
+    # once per process, hence the child process.
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, SLKV_NO_COOPERATIVE="1")
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-m", "gpu", "-x",
+                        "tests/test_gpu_compress.py::test_overlapped_calls_match_ordinary_calls",
+                        "tests/test_gpu_compress.py::test_overlapped_calls_of_changing_shapes_and_streams"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
