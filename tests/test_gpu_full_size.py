@@ -52,3 +52,56 @@ def test_config5_long_context_heavy_and_fixed_only_layers():
     for layer in (heavy, fixed_only):
         _, bud, gpu, stats = full_layer(wl, layer, wl.totals[0])
         assert stats["segments"] == 8 and stats["pooled_max_rel_err"] < 1e-3
+
+
+def test_config3_full_layers_through_the_overlapped_entry_point():
+    # the launch configuration bench.py times: layers queued by slkv_compress_overlapped, the score kernel taking
+    # them a list at a time (here 10 layers: a full list of 8, then the rest at the join).  Pooled scores and the
+    # selection of two of the layers against the oracle, every layer against slkv_compress bit for bit.
+    from paper_2508_15806_b200 import binding as B
+    wl = synth.workloads()[2]
+    total = wl.totals[1]
+    dev = torch.device("cuda:0")
+    layers = [0, 1, 2, 3, 17, 18, 19, 20, 30, 31]
+    budgets = O.alloc_budgets(synth.inf_sc(wl).numpy(), wl.fixed, total)
+    xs = [synth.layer_inputs(wl, l, device=dev) for l in layers]
+    cu = wl.cu_seqlens
+    cu_dev = torch.tensor(cu, dtype=torch.int32, device=dev)
+    params = B.make_params(xs[0].q_win, xs[0].k, xs[0].v, wl.window, wl.pool_kernel)
+    ws = torch.empty(B.slkv_workspace_bytes_overlapped(params, cu), dtype=torch.uint8, device=dev)
+    cap = B.slkv_packed_rows_upper_bound(params, cu)
+    n_pool = B.slkv_pooled_elems(params, cu)
+    buds = [torch.tensor(budgets[l].tolist(), dtype=torch.int32, device=dev) for l in layers]
+
+    def outputs():
+        return [dict(k_out=torch.zeros(cap, 128, dtype=torch.bfloat16, device=dev),
+                     v_out=torch.zeros(cap, 128, dtype=torch.bfloat16, device=dev),
+                     offsets=torch.zeros(9, dtype=torch.int32, device=dev),
+                     kept=torch.full((cap,), -1, dtype=torch.int32, device=dev),
+                     pooled=torch.full((n_pool,), float("nan"), dtype=torch.float32, device=dev),
+                     status=torch.zeros(1, dtype=torch.int32, device=dev)) for _ in layers]
+
+    def run(fn, outs):
+        for x, bud, o in zip(xs, buds, outs):
+            fn(params, x.q_win, x.k, x.v, cu_dev, cu, bud, o["k_out"], o["v_out"], o["offsets"], o["kept"], ws,
+               o["pooled"], o["status"])
+        B.slkv_join()
+        torch.cuda.synchronize()
+
+    a, b = outputs(), outputs()
+    run(B.slkv_compress, a)
+    run(B.slkv_compress_overlapped, b)
+    for i, l in enumerate(layers):
+        assert int(b[i]["status"].item()) == 0
+        n = int(a[i]["offsets"][-1].item())
+        assert n == int(budgets[l].clip(wl.window, 32768).sum())
+        assert torch.equal(a[i]["offsets"], b[i]["offsets"]) and torch.equal(a[i]["kept"][:n], b[i]["kept"][:n])
+        assert torch.equal(a[i]["k_out"][:n], b[i]["k_out"][:n]) and torch.equal(a[i]["v_out"][:n], b[i]["v_out"][:n])
+    for i in (1, 9):                                  # layer 1 (three near-zero heads) and layer 31
+        x = xs[i]
+        q, k, v = x.q_win.cpu(), x.k.cpu(), x.v.cpu()
+        ref = P.oracle_pooled(q, k, cu, wl.window, wl.pool_kernel)
+        gpu = {"offsets": b[i]["offsets"].cpu().numpy().astype(np.int64), "kept_idx": b[i]["kept"].cpu().numpy().astype(np.int64),
+               "k_out": b[i]["k_out"].cpu(), "v_out": b[i]["v_out"].cpu()}
+        P.assert_pooled_close(b[i]["pooled"].cpu().numpy(), ref, cu, wl.n_kv_heads, wl.window)
+        P.assert_selection_valid(gpu, ref, cu, budgets[layers[i]].tolist(), wl.window, k, v)
