@@ -263,8 +263,14 @@ int slkv_kernel_count(void);
  * With a device buffer set on the calling thread, every CTA of the two score kernels stores %globaltimer
  * nanosecond stamps into it: 64 uint64 slots per CTA, pass 1 first (n_cta * 64 entries), pass 2 after
  * it.  Slots: 0 CTA start, 1 set-up done, 2 query tile landed, 3 first key tile landed, 4 CTA end,
- * 8+2i / 9+2i start / end of the softmax arithmetic on the CTA's i-th tile (i < 28).  The buffer must hold
- * 2 * n_cta * 64 * 8 bytes (n_cta <= number of SMs); smaller buffers switch tracing off.  NULL switches it off.
+ * 8+2i / 9+2i start / end of the softmax arithmetic on the CTA's i-th tile (i < 28).  The score kernel of the
+ * overlapped entry point (a list of layers per launch, two streams per CTA) writes: 0 CTA start, 1 / 7 stream
+ * A / B past its wait for the launch before, 2 first accumulator of stream A ready, 3 first log-sum-exps of
+ * stream B merged, 5 / 6 stream A / B done, 4 CTA end, 8+2j / 9+2j list entry j published by stream A / begun by
+ * stream B, 60 / 61 the SM cycle counter at CTA start / end.  The buffer that is set when a launch is enqueued is
+ * the one it writes (the overlapped entry point enqueues a list when it is full and one more layer has come, or at
+ * a join).  The buffer must hold 2 * n_cta * 64 * 8 bytes (n_cta <= number of SMs); smaller buffers switch tracing
+ * off.  NULL switches it off.  python -m paper_2508_15806_b200.trace_timeline prints a step's timeline from it.
  */
 int slkv_trace_set_buffer(void* dev_buf, size_t bytes);
 
