@@ -7,12 +7,16 @@
  *   slkv_compress        score -> top-(C - window) history rows + window, gather (Sec. 3.4, Eq. 8, Algorithm 3)
  *   slkv_compress_host   the same, from/to host buffers (copies included)
  *   slkv_compress_overlapped / slkv_join   the same, successive layers overlapped on the GPU
+ *   slkv_row_lse         the window rows' log-sum-exp over their softmax domain       (Eq. 3-4, Eq. 7)
  *
  * Conventions
  *   - "dev" pointers are device memory of the current CUDA device, "host" pointers are host memory.
  *   - The caller owns every buffer.  The library allocates no device memory; scratch comes from the
  *     caller's `workspace` (size from slkv_workspace_bytes) and must stay untouched until the enqueued
- *     work has finished.  Nothing is freed or retained by the library.
+ *     work has finished.  Nothing is freed or retained by the library.  One exception, for callers that
+ *     have no workspace to give: slkv_score_noalloc works in a fixed array of SLKV_NOALLOC_SCRATCH_BYTES
+ *     that is part of the library's device image (see there for when it comes into being and how long it
+ *     lives).
  *   - All device work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
  *     No call synchronises the device except slkv_compress_host, which returns after its results are
  *     in the host buffers.
@@ -61,7 +65,9 @@ typedef enum slkv_status {
 
 enum { SLKV_F32 = 0, SLKV_BF16 = 1 };                 /* slkv_params.dtype */
 enum { SLKV_POOL_MAX = 0, SLKV_POOL_AVG = 1 };        /* slkv_params.pool_mode */
-enum { SLKV_HISTORY = 0 };                            /* slkv_params.softmax_domain: softmax over history keys */
+enum { SLKV_HISTORY = 0,                              /* slkv_params.softmax_domain: softmax over the history keys */
+       SLKV_ALL_CAUSAL = 1 };                         /*   over every key a window query sees causally */
+enum { SLKV_LSE_LN = 0, SLKV_LSE_LOG2 = 1 };          /* slkv_params.lse_units: natural log / base-2 log */
 enum { SLKV_PATH_AUTO = 0,                            /* slkv_params.score_path */
        SLKV_PATH_SIMT = 1,                            /*   fp32 FMA kernels (any dtype, head_dim 64/128) */
        SLKV_PATH_TENSOR = 2 };                        /*   tcgen05 + TMA kernels (bf16, head_dim 128) */
@@ -76,8 +82,10 @@ typedef struct slkv_params {
   int32_t pool_kernel;     /* odd >= 1 (1 = no pooling) */
   int32_t dtype;           /* SLKV_F32 | SLKV_BF16: element type of Q_win, K, V and the packed outputs */
   int32_t pool_mode;       /* SLKV_POOL_MAX | SLKV_POOL_AVG */
-  int32_t softmax_domain;  /* SLKV_HISTORY */
+  int32_t softmax_domain;  /* SLKV_HISTORY | SLKV_ALL_CAUSAL: the keys a window row's softmax runs over */
   int32_t score_path;      /* SLKV_PATH_AUTO picks TENSOR when the shape allows it, else SIMT */
+  int32_t lse_units;       /* SLKV_LSE_LN | SLKV_LSE_LOG2: units of lse_opt / slkv_row_lse's output */
+  int32_t reserved;        /* must be 0 */
   int64_t k_stride_tok, k_stride_head;
   int64_t v_stride_tok, v_stride_head;
   int64_t q_stride_seq, q_stride_row, q_stride_head;
@@ -118,20 +126,41 @@ int64_t slkv_packed_rows_upper_bound(const slkv_params* p, const int32_t* cu_seq
 /*
  * Relevance scores (Sec. 3.4, Eq. 7; Algorithm 3 lines 4-6; scale and softmax axis from Eq. 3-4).
  * For every sequence s, KV head g and history key j < n_hist_s:
- *     vote[j]   = (1/G) * sum_{query heads h of group g} sum_{window rows i} softmax_j(q_i . k_j / sqrt(head_dim))
+ *     vote[j]   = (1/G) * sum_{query heads h of group g} sum_{window rows i} exp(q_i . k_j / sqrt(head_dim) - lse_i)
  *     pooled[j] = max (or zero-padded mean) of vote over [j - pool_kernel/2, j + pool_kernel/2] within the history
- * with the softmax taken over the history keys only.  (The paper leaves the reduction over the window
+ * where lse_i is the log-sum-exp of row i's scaled scores over its softmax domain: the history keys
+ * (SLKV_HISTORY: Eq. 7 and Algorithm 3 as printed) or the history keys plus the window keys up to the
+ * row's own position (SLKV_ALL_CAUSAL: the prefill attention's own softmax, the reading of the prior work
+ * Sec. 3.4 refers to; the window columns get no vote).  (The paper leaves the reduction over the window
  * rows, the GQA reduction and the pooling to prior work; this is the reading used here.)
  *   q_win, k         dev, layouts above
  *   cu_seqlens_dev   dev, int32[n_seqs+1];  cu_seqlens_host: the same values on the host (sizes the launch)
+ *   lse_opt          dev, optional, float[n_seqs][n_q_heads][window] in p->lse_units: the rows' log-sum-exp
+ *                    when the caller has it already (a prefill attention kernel that keeps its softmax
+ *                    statistics has exactly the SLKV_ALL_CAUSAL one).  NULL: computed here, which costs a
+ *                    second pass over K.  The values are used as given, whatever softmax_domain says.
  *   pooled           dev, out, float[slkv_pooled_elems]
  *   status           dev, optional: SLKV_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel ran out
  *                    (pooled is then incomplete)
  * Accuracy: fp32 accumulation; relative error of pooled <= 1e-3 of the exact value.
  */
 int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
-               const int32_t* cu_seqlens_host, float* pooled, int32_t* status, void* workspace,
-               size_t workspace_bytes, void* stream);
+               const int32_t* cu_seqlens_host, const float* lse_opt, float* pooled, int32_t* status,
+               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The row statistics alone (Eq. 3-4 with Eq. 7's key set): lse_out[s][h][i] = log sum_j exp(q_i . k_j /
+ * sqrt(head_dim)) over the softmax domain of p->softmax_domain, in p->lse_units, for the window rows of
+ * every sequence longer than the window (rows of shorter sequences are left untouched).  It is what
+ * slkv_score computes first when lse_opt is NULL; fed back as lse_opt it reproduces that call bit for bit
+ * with SLKV_LSE_LOG2 (the kernels' own unit), and to rounding with SLKV_LSE_LN.  Callers that shard the
+ * keys of one sequence over several devices merge these per shard and pass the result as lse_opt.
+ *   lse_out   dev, out, float[n_seqs][n_q_heads][window]
+ * Other arguments and errors as slkv_score.
+ */
+int slkv_row_lse(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+                 const int32_t* cu_seqlens_host, float* lse_out, int32_t* status, void* workspace,
+                 size_t workspace_bytes, void* stream);
 
 /*
  * KV entry selection and gather for one layer (Sec. 3.4, Eq. 8; Algorithm 3).
@@ -139,6 +168,7 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
  * everything if len_s <= C (Alg. 3 l.1-3), else the window rows plus the kept - window history positions
  * with the largest pooled score (ties: lower position first), in ascending position order (l.7-10).
  *   budgets            dev, int32[n_kv_heads]: this layer's row of slkv_alloc_budgets' output
+ *   lse_opt            dev, optional: as in slkv_score
  *   k_out, v_out       dev, out, [out_capacity_rows, head_dim] elements of p->dtype
  *   offsets            dev, out, int32[n_seqs*n_kv_heads + 1]
  *   kept_idx           dev, out, int32[out_capacity_rows]
@@ -149,7 +179,7 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
  */
 int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const void* v,
                   const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
-                  void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx,
+                  const float* lse_opt, void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx,
                   float* pooled_opt, int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
@@ -183,7 +213,7 @@ int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const 
  */
 int slkv_compress_overlapped(const slkv_params* p, const void* q_win, const void* k, const void* v,
                              const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
-                             void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets,
+                             const float* lse_opt, void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets,
                              int32_t* kept_idx, float* pooled_opt, int32_t* status, void* workspace,
                              size_t workspace_bytes, void* stream);
 size_t slkv_workspace_bytes_overlapped(const slkv_params* p, const int32_t* cu_seqlens_host);
@@ -227,8 +257,10 @@ int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, c
  *   - Shapes whose slkv_workspace_bytes exceed the array are rejected with SLKV_ERR_WORKSPACE before anything
  *     is enqueued (32k tokens x 8 KV heads x 128 score rows needs about 5.3 MB).
  *   - The first call on each device looks up the array's device address (a CUDA runtime query, made with that
- *     device current) and keeps it; make that first call outside any stream capture.
- *   - No cudaMalloc, cudaFree or other allocating routine is called, on the first call or later.
+ *     device current) and keeps it.  With the CUDA runtime's lazy module loading the array comes into being at
+ *     that query, not when the library is loaded: make the first call at start-up, while SLKV_NOALLOC_SCRATCH_BYTES
+ *     of device memory are still free (otherwise it returns SLKV_ERR_CUDA), and outside any stream capture.
+ *   - The library itself calls no cudaMalloc, cudaFree or other allocating routine, on the first call or later.
  *   - All calls on a device share the one array.  It keeps whatever the previous call left; nothing in it has
  *     to be zero, each call overwrites what it reads.  Two calls whose kernels may overlap on the GPU
  *     (different streams, no ordering between them) race on it: order them.
@@ -237,7 +269,8 @@ int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, c
  */
 #define SLKV_NOALLOC_SCRATCH_BYTES (8u << 20)
 int slkv_score_noalloc(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
-                       const int32_t* cu_seqlens_host, float* pooled, int32_t* status, void* stream);
+                       const int32_t* cu_seqlens_host, const float* lse_opt, float* pooled, int32_t* status,
+                       void* stream);
 size_t slkv_noalloc_scratch_bytes(void);      /* = SLKV_NOALLOC_SCRATCH_BYTES */
 int slkv_noalloc_last_cuda_error(void);
 
@@ -273,6 +306,17 @@ int slkv_kernel_count(void);
  * off.  NULL switches it off.  python -m paper_2508_15806_b200.trace_timeline prints a step's timeline from it.
  */
 int slkv_trace_set_buffer(void* dev_buf, size_t bytes);
+
+/*
+ * Test hook for the bounded waits (no counterpart in the paper).  Where the CTAs of a launch wait for one another
+ * (the grid-wide barrier between the two passes of slkv_score / slkv_compress, the per-layer counters of the list
+ * kernel behind slkv_compress_overlapped), every wait gives up after one second, sets SLKV_ERR_DEVICE_TIMEOUT in the
+ * call's status word, releases what the CTA holds and returns.  With the hook armed (on != 0) the next such launch made
+ * by the calling thread waits for one arrival more than there are CTAs, so that exactly this path runs: the call's
+ * results are then incomplete and its status word says so; the calls after it are unaffected.  One-shot: the launch
+ * that takes it disarms it.
+ */
+int slkv_debug_expire_next_wait(int on);
 
 /* Library version, major*10000 + minor*100 + patch. */
 int slkv_version(void);

@@ -10,6 +10,7 @@ What follows which passage of the paper:
   alloc_budgets         Algorithm 2's weights (0.01 + L_i) * S_ij, normalised so the dynamic parts sum to
                         the dynamic pool exactly (largest-remainder rounding) -- the paper concedes that its
                         own formula "does not strictly conform to mathematical normalization" (Sec. 3.3).
+  row_lse               Eq. 3-4's row normaliser over Eq. 7's key set (the log of the softmax denominator).
   window_votes          Eq. 7 / Algorithm 3 line 6: softmax over the history keys of Q_window H^T / sqrt(d_k)
                         (Eq. 3-4 fix the scale and the softmax axis), then -- the paper does not say how the
                         w rows are reduced -- summed over the window rows and averaged over a GQA group.
@@ -155,15 +156,44 @@ def behavior_scores(W: np.ndarray, needle_idx: Sequence[int], topk_idx: Sequence
 # ----------------------------------------------------------------------------------------------
 # Prefill: scores -> pool -> select -> gather
 # ----------------------------------------------------------------------------------------------
+def row_lse(q_win: np.ndarray, k: np.ndarray, cu_seqlens: Sequence[int], window: int,
+            domain: str = "history") -> np.ndarray:
+    """lse[s][h][i] = log sum_j exp(q_i . k_j / sqrt(d)) over row i's softmax domain (Eq. 3-4's denominator with
+    Eq. 7's key set): the history keys, or with domain="all_causal" the history plus the window keys up to the
+    row's own position.  fp64 [n_seqs, n_q_heads, window]; NaN for sequences without history."""
+    q_win = np.asarray(q_win, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    B, w, Hq, d = q_win.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    out = np.full((B, Hq, w), np.nan)
+    for s in range(B):
+        t0, t1 = int(cu_seqlens[s]), int(cu_seqlens[s + 1])
+        n_hist = max(t1 - t0 - w, 0)
+        if n_hist == 0:
+            continue
+        for h in range(Hq):
+            g = h // G
+            for i in range(w):
+                n_keys = n_hist if domain == "history" else n_hist + i + 1
+                if domain not in ("history", "all_causal"):
+                    raise ValueError(domain)
+                x = (k[t0:t0 + n_keys, g, :] @ q_win[s, i, h, :]) / math.sqrt(d)
+                m = x.max()
+                out[s, h, i] = m + math.log(np.exp(x - m).sum())
+    return out
+
+
 def window_votes(q_win: np.ndarray, k: np.ndarray, cu_seqlens: Sequence[int], window: int,
-                 domain: str = "history") -> List[np.ndarray]:
+                 domain: str = "history", lse: np.ndarray = None) -> List[np.ndarray]:
     """Per sequence: vote[g][j] = (1/G) sum_{h in group g} sum_{i in window} A^h_ij, fp64 [n_kv_heads, n_hist].
 
     q_win [n_seqs, window, n_q_heads, d] holds the queries of each sequence's last `window` tokens,
     k [total_tokens, n_kv_heads, d] the keys.  A^h = softmax_j(q_i . k_j / sqrt(d)) over the history keys
     j < n_hist = len - window (domain="history", Eq. 7 / Algorithm 3 line 6), or over all keys a window query
     may see causally (domain="all_causal": history plus window keys up to the query's own position), the
-    window columns being dropped afterwards.
+    window columns being dropped afterwards.  With `lse` ([n_seqs, n_q_heads, window], natural log) the rows'
+    normalisers are taken from it as given: A^h_ij = exp(q_i . k_j / sqrt(d) - lse[s][h][i]).
     """
     q_win = np.asarray(q_win, dtype=np.float64)
     k = np.asarray(k, dtype=np.float64)
@@ -182,7 +212,9 @@ def window_votes(q_win: np.ndarray, k: np.ndarray, cu_seqlens: Sequence[int], wi
                 for h in range(g * G, (g + 1) * G):
                     Qw = q_win[s, :, h, :]                                   # [w, d]
                     S = (Qw @ Hist.T) / math.sqrt(d)                         # Eq. 3
-                    if domain == "history":
+                    if lse is not None:
+                        A = np.exp(S - np.asarray(lse, dtype=np.float64)[s, h][:, None])
+                    elif domain == "history":
                         m = S.max(axis=1, keepdims=True)
                         E = np.exp(S - m)
                         A = E / E.sum(axis=1, keepdims=True)                 # Eq. 4, keys = history

@@ -19,13 +19,15 @@ ERR = {"NULL_PTR": -1, "BAD_SHAPE": -2, "BAD_DTYPE": -3, "BAD_ALIGN": -4, "BUDGE
        "CAPACITY": -7, "WORKSPACE": -8, "CUDA": -9, "DEVICE_TIMEOUT": -10}
 SLKV_F32, SLKV_BF16 = 0, 1
 SLKV_POOL_MAX, SLKV_POOL_AVG = 0, 1
-SLKV_HISTORY = 0
+SLKV_HISTORY, SLKV_ALL_CAUSAL = 0, 1
+SLKV_LSE_LN, SLKV_LSE_LOG2 = 0, 1
 SLKV_PATH_AUTO, SLKV_PATH_SIMT, SLKV_PATH_TENSOR = 0, 1, 2
 
 
 class SlkvParams(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_seqs", "n_q_heads", "n_kv_heads", "head_dim", "window", "pool_kernel",
-                                         "dtype", "pool_mode", "softmax_domain", "score_path")] + \
+                                         "dtype", "pool_mode", "softmax_domain", "score_path", "lse_units",
+                                         "reserved")] + \
                [(n, C.c_int64) for n in ("k_stride_tok", "k_stride_head", "v_stride_tok", "v_stride_head",
                                          "q_stride_seq", "q_stride_row", "q_stride_head")]
 
@@ -66,9 +68,13 @@ def lib() -> C.CDLL:
         L.slkv_packed_rows_upper_bound.restype = i64
         L.slkv_packed_rows_upper_bound.argtypes = [pp, i32p]
         L.slkv_score.restype = C.c_int
-        L.slkv_score.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, sz, vp]
+        L.slkv_score.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, vp, sz, vp]
+        L.slkv_row_lse.restype = C.c_int
+        L.slkv_row_lse.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, sz, vp]
+        L.slkv_debug_expire_next_wait.restype = C.c_int
+        L.slkv_debug_expire_next_wait.argtypes = [C.c_int]
         L.slkv_compress.restype = C.c_int
-        L.slkv_compress.argtypes = [pp, vp, vp, vp, vp, i32p, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+        L.slkv_compress.argtypes = [pp, vp, vp, vp, vp, i32p, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
         L.slkv_compress_overlapped.restype = C.c_int
         L.slkv_compress_overlapped.argtypes = L.slkv_compress.argtypes
         L.slkv_workspace_bytes_overlapped.restype = sz
@@ -81,7 +87,7 @@ def lib() -> C.CDLL:
         L.slkv_compress_host.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, i64, vp, vp, C.POINTER(C.c_int64),
                                          vp, sz, vp]
         L.slkv_score_noalloc.restype = C.c_int
-        L.slkv_score_noalloc.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp]
+        L.slkv_score_noalloc.argtypes = [pp, vp, vp, vp, i32p, vp, vp, vp, vp]
         L.slkv_noalloc_scratch_bytes.restype = sz
         L.slkv_noalloc_last_cuda_error.restype = C.c_int
         L.slkv_profile_enable.restype = C.c_int
@@ -112,7 +118,8 @@ def _cu_host(cu_seqlens: Sequence[int]):
 
 
 def make_params(q_win: torch.Tensor, k: torch.Tensor, v: Optional[torch.Tensor], window: int, pool_kernel: int,
-                pool_mode: int = SLKV_POOL_MAX, score_path: int = SLKV_PATH_AUTO) -> SlkvParams:
+                pool_mode: int = SLKV_POOL_MAX, score_path: int = SLKV_PATH_AUTO,
+                softmax_domain: int = SLKV_HISTORY, lse_units: int = SLKV_LSE_LN) -> SlkvParams:
     """Shapes and strides from the tensors: q_win [n_seqs, w, Hq, d], k / v [T, Hkv, d] (last dim contiguous)."""
     assert q_win.dim() == 4 and k.dim() == 3 and q_win.stride(3) == 1 and k.stride(2) == 1
     if v is None:
@@ -121,7 +128,7 @@ def make_params(q_win: torch.Tensor, k: torch.Tensor, v: Optional[torch.Tensor],
     assert q_win.dtype == k.dtype == v.dtype
     return SlkvParams(n_seqs=q_win.shape[0], n_q_heads=q_win.shape[2], n_kv_heads=k.shape[1], head_dim=k.shape[2],
                       window=window, pool_kernel=pool_kernel, dtype=dt, pool_mode=pool_mode,
-                      softmax_domain=SLKV_HISTORY, score_path=score_path,
+                      softmax_domain=softmax_domain, score_path=score_path, lse_units=lse_units, reserved=0,
                       k_stride_tok=k.stride(0), k_stride_head=k.stride(1),
                       v_stride_tok=v.stride(0), v_stride_head=v.stride(1),
                       q_stride_seq=q_win.stride(0), q_stride_row=q_win.stride(1), q_stride_head=q_win.stride(2))
@@ -167,23 +174,49 @@ def new_workspace(params: SlkvParams, cu_seqlens: Sequence[int], device) -> torc
     return torch.empty(n, dtype=torch.uint8, device=device)
 
 
+def _lse(lse: Optional[torch.Tensor], params: SlkvParams) -> Optional[int]:
+    if lse is None:
+        return None
+    assert lse.is_cuda and lse.dtype == torch.float32 and lse.is_contiguous()
+    assert lse.numel() == params.n_seqs * params.n_q_heads * params.window, "lse is [n_seqs, n_q_heads, window]"
+    return lse.data_ptr()
+
+
 def slkv_score(params: SlkvParams, q_win: torch.Tensor, k: torch.Tensor, cu_dev: torch.Tensor,
                cu_seqlens: Sequence[int], pooled: torch.Tensor, workspace: torch.Tensor,
-               status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+               status: Optional[torch.Tensor] = None, stream=None, lse: Optional[torch.Tensor] = None) -> torch.Tensor:
     rc = lib().slkv_score(C.byref(params), q_win.data_ptr(), k.data_ptr(), cu_dev.data_ptr(), _cu_host(cu_seqlens),
-                          pooled.data_ptr(), _ptr(status), workspace.data_ptr(), workspace.numel(), _stream(stream))
+                          _lse(lse, params), pooled.data_ptr(), _ptr(status), workspace.data_ptr(), workspace.numel(),
+                          _stream(stream))
     if rc != SLKV_OK:
         raise SlkvError(rc, "slkv_score")
     return pooled
 
 
+def slkv_row_lse(params: SlkvParams, q_win: torch.Tensor, k: torch.Tensor, cu_dev: torch.Tensor,
+                 cu_seqlens: Sequence[int], lse_out: torch.Tensor, workspace: torch.Tensor,
+                 status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """lse_out: CUDA float32 [n_seqs, n_q_heads, window], the window rows' log-sum-exp in params.lse_units."""
+    _lse(lse_out, params)
+    rc = lib().slkv_row_lse(C.byref(params), q_win.data_ptr(), k.data_ptr(), cu_dev.data_ptr(), _cu_host(cu_seqlens),
+                            lse_out.data_ptr(), _ptr(status), workspace.data_ptr(), workspace.numel(), _stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_row_lse")
+    return lse_out
+
+
+def slkv_debug_expire_next_wait(on: bool = True) -> None:
+    lib().slkv_debug_expire_next_wait(1 if on else 0)
+
+
 def slkv_score_noalloc(params: SlkvParams, q_win: torch.Tensor, k: torch.Tensor, cu_dev: torch.Tensor,
                        cu_seqlens: Sequence[int], pooled: torch.Tensor, status: Optional[torch.Tensor] = None,
-                       stream=None) -> torch.Tensor:
+                       stream=None, lse: Optional[torch.Tensor] = None) -> torch.Tensor:
     """slkv_score for callers that cannot allocate: the scratch is a fixed array inside the library
     (slkv_noalloc_scratch_bytes() bytes); larger shapes raise SLKV_ERR_WORKSPACE."""
     rc = lib().slkv_score_noalloc(C.byref(params), q_win.data_ptr(), k.data_ptr(), cu_dev.data_ptr(),
-                                  _cu_host(cu_seqlens), pooled.data_ptr(), _ptr(status), _stream(stream))
+                                  _cu_host(cu_seqlens), _lse(lse, params), pooled.data_ptr(), _ptr(status),
+                                  _stream(stream))
     if rc != SLKV_OK:
         raise SlkvError(rc, "slkv_score_noalloc")
     return pooled
@@ -195,9 +228,10 @@ def slkv_noalloc_scratch_bytes() -> int:
 
 def slkv_compress(params: SlkvParams, q_win, k, v, cu_dev, cu_seqlens: Sequence[int], budgets, k_out, v_out,
                   offsets, kept_idx, workspace, pooled: Optional[torch.Tensor] = None,
-                  status: Optional[torch.Tensor] = None, stream=None) -> None:
+                  status: Optional[torch.Tensor] = None, stream=None, lse: Optional[torch.Tensor] = None) -> None:
     rc = lib().slkv_compress(C.byref(params), q_win.data_ptr(), k.data_ptr(), v.data_ptr(), cu_dev.data_ptr(),
-                             _cu_host(cu_seqlens), budgets.data_ptr(), k_out.data_ptr(), v_out.data_ptr(),
+                             _cu_host(cu_seqlens), budgets.data_ptr(), _lse(lse, params), k_out.data_ptr(),
+                             v_out.data_ptr(),
                              k_out.shape[0], offsets.data_ptr(), kept_idx.data_ptr(), _ptr(pooled), _ptr(status),
                              workspace.data_ptr(), workspace.numel(), _stream(stream))
     if rc != SLKV_OK:
@@ -206,11 +240,12 @@ def slkv_compress(params: SlkvParams, q_win, k, v, cu_dev, cu_seqlens: Sequence[
 
 def slkv_compress_overlapped(params: SlkvParams, q_win, k, v, cu_dev, cu_seqlens: Sequence[int], budgets, k_out,
                              v_out, offsets, kept_idx, workspace, pooled: Optional[torch.Tensor] = None,
-                             status: Optional[torch.Tensor] = None, stream=None) -> None:
+                             status: Optional[torch.Tensor] = None, stream=None,
+                             lse: Optional[torch.Tensor] = None) -> None:
     """slkv_compress with successive calls overlapped on the GPU; outputs are valid behind slkv_join()."""
     rc = lib().slkv_compress_overlapped(C.byref(params), q_win.data_ptr(), k.data_ptr(), v.data_ptr(),
                                         cu_dev.data_ptr(), _cu_host(cu_seqlens), budgets.data_ptr(),
-                                        k_out.data_ptr(), v_out.data_ptr(), k_out.shape[0], offsets.data_ptr(),
+                                        _lse(lse, params), k_out.data_ptr(), v_out.data_ptr(), k_out.shape[0], offsets.data_ptr(),
                                         kept_idx.data_ptr(), _ptr(pooled), _ptr(status), workspace.data_ptr(),
                                         workspace.numel(), _stream(stream))
     if rc != SLKV_OK:

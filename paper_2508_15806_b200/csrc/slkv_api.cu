@@ -43,7 +43,8 @@ int cuda_fail(cudaError_t e) {
 
 constexpr int kLaySlots = 2 * kPipeMaxLayers + 2;   // overlapped calls: layers in flight at once
 struct Layout {
-  size_t hist_off, tile_off, vote[kLaySlots], pooled, part_m[kLaySlots], part_z[kLaySlots], flags, gather_src[kLaySlots], total;
+  size_t hist_off, tile_off, vote[kLaySlots], pooled, part_m[kLaySlots], part_z[kLaySlots], flags, gather_src[kLaySlots],
+      win_m[kLaySlots], win_z[kLaySlots], total;
 };
 
 // Validates p and cu_seqlens_host and fills the host-known fields of `pb`.
@@ -51,7 +52,9 @@ int describe(const slkv_params* p, const int32_t* cu_host, Problem* pb) {
   if (!p || !cu_host) return SLKV_ERR_NULL_PTR;
   if (p->dtype != SLKV_F32 && p->dtype != SLKV_BF16) return SLKV_ERR_BAD_DTYPE;
   if (p->pool_mode != SLKV_POOL_MAX && p->pool_mode != SLKV_POOL_AVG) return SLKV_ERR_BAD_DTYPE;
-  if (p->softmax_domain != SLKV_HISTORY) return SLKV_ERR_BAD_DTYPE;
+  if (p->softmax_domain != SLKV_HISTORY && p->softmax_domain != SLKV_ALL_CAUSAL) return SLKV_ERR_BAD_DTYPE;
+  if (p->lse_units != SLKV_LSE_LN && p->lse_units != SLKV_LSE_LOG2) return SLKV_ERR_BAD_DTYPE;
+  if (p->reserved != 0) return SLKV_ERR_BAD_DTYPE;
   if (p->score_path < SLKV_PATH_AUTO || p->score_path > SLKV_PATH_TENSOR) return SLKV_ERR_BAD_DTYPE;
   if (p->n_seqs < 1 || p->n_seqs > (1 << 20)) return SLKV_ERR_BAD_SHAPE;
   if (p->n_kv_heads < 1 || p->n_kv_heads > 65535 || p->n_q_heads < p->n_kv_heads ||
@@ -146,6 +149,14 @@ Layout layout_of(const Problem& pb, bool overlapped = false) {
     L.gather_src[i] = i < n_slots ? o : L.gather_src[0];
     if (i < n_slots) o = align_up(o + srcs);
   }
+  // row statistics over the window keys (all-causal softmax domain): [n_seg][R] maxima and sums
+  const size_t wins = (size_t)pb.n_seg * pb.R * sizeof(float);
+  for (int i = 0; i < kLaySlots; ++i) {
+    L.win_m[i] = i < n_slots ? o : L.win_m[0];
+    if (i < n_slots) o = align_up(o + wins);
+    L.win_z[i] = i < n_slots ? o : L.win_z[0];
+    if (i < n_slots) o = align_up(o + wins);
+  }
   L.total = o;
   return L;
 }
@@ -178,6 +189,8 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overla
   pb->part_z = reinterpret_cast<float*>(b + L.part_z[slot]);
   pb->dev_flags = reinterpret_cast<int32_t*>(b + L.flags);
   pb->gather_src = reinterpret_cast<int32_t*>(b + L.gather_src[slot]);
+  pb->win_m = reinterpret_cast<float*>(b + L.win_m[slot]);
+  pb->win_z = reinterpret_cast<float*>(b + L.win_z[slot]);
   pb->chunk_keys = path == SLKV_PATH_TENSOR ? 128 : simt_chunk_keys();
   pb->n_chunks = path == SLKV_PATH_TENSOR ? tensor_slot_stride(*pb)
                                           : (pb->max_hist + pb->chunk_keys - 1) / pb->chunk_keys;
@@ -187,11 +200,23 @@ int bind_workspace(Problem* pb, void* ws, size_t ws_bytes, int path, bool overla
 
 bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
 
-// window votes of every history key (device pointers resolved)
+// The window keys' row statistics, where the softmax runs over all causally visible keys and the caller has not
+// supplied the rows' log-sum-exp (Eq. 3-4 over the prefill attention's own key set).
+int enqueue_window_stats(const Problem& pb, int path, cudaStream_t st, int* launches) {
+  if (pb.lse_opt || pb.p.softmax_domain != SLKV_ALL_CAUSAL) return SLKV_OK;
+  cudaError_t e = launch_window_stats(pb, path == SLKV_PATH_TENSOR && tensor_q_head_inner(pb.p), st, launches);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return SLKV_OK;
+}
+
+// window votes of every history key (device pointers resolved); with the caller's row statistics the vote pass alone
 int enqueue_votes(const Problem& pb, int path, const int32_t* cu_host, int32_t* status, cudaStream_t st,
                   int* launches) {
-  cudaError_t e = path == SLKV_PATH_TENSOR ? launch_score_tensor(pb, cu_host, status, st, launches)
-                                           : launch_score_simt(pb, st, launches);
+  int rc = enqueue_window_stats(pb, path, st, launches);
+  if (rc != SLKV_OK) return rc;
+  const int passes = pb.lse_opt ? 2 : 3;
+  cudaError_t e = path == SLKV_PATH_TENSOR ? launch_score_tensor(pb, cu_host, status, passes, st, launches)
+                                           : launch_score_simt(pb, passes, st, launches);
   if (e != cudaSuccess) return cuda_fail(e);
   return SLKV_OK;
 }
@@ -317,7 +342,7 @@ cudaError_t launch_queue(OverlapState* os, int n, bool finish, int* launches) {
   if (n == 1 && finish && !os->pending.valid) {
     // a single layer and nothing to pair it with: both passes in the single-layer kernel
     const PendingCall& c = os->queue[0];
-    cudaError_t e1 = launch_score_tensor(c.pb, c.cu_host.data(), c.status, c.st, launches);
+    cudaError_t e1 = launch_score_tensor(c.pb, c.cu_host.data(), c.status, c.pb.lse_opt ? 2 : 3, c.st, launches);
     if (e1 == cudaSuccess) e1 = enqueue_tail(os, c, false, true, launches);
     os->queue.clear();
     return e1;
@@ -325,7 +350,11 @@ cudaError_t launch_queue(OverlapState* os, int n, bool finish, int* launches) {
   const TcPlan* plans[kPipeMaxLayers];
   for (int i = 0; i < n; ++i) plans[i] = &os->queue[i].plan;
   cudaStream_t st = n > 0 ? os->queue[0].st : os->pending.st;
-  cudaError_t e = launch_score_pipe(os->pending.valid ? &os->pending.plan : nullptr, plans, n, finish, st, launches);
+  // layers that came with their row statistics need the vote pass only (a queue holds one kind: see compress_impl)
+  const bool votes_only = n > 0 && os->queue[0].pb.lse_opt != nullptr;
+  if (votes_only) finish = true;
+  cudaError_t e = launch_score_pipe(os->pending.valid ? &os->pending.plan : nullptr, plans, n, finish, votes_only, st,
+                                    launches);
   if (e == cudaSuccess && os->pending.valid) e = enqueue_tail(os, os->pending, true, finish, launches);
   os->pending.valid = false;
   const int n_voted = finish ? n : n - 1;
@@ -362,7 +391,8 @@ cudaError_t join_overlapped(cudaStream_t st, int* launches) {
 }
 
 int compress_impl(const slkv_params* p, const void* q_win, const void* k, const void* v, const int32_t* cu_dev,
-                  const int32_t* cu_host, const int32_t* budgets, void* k_out, void* v_out, int64_t capacity,
+                  const int32_t* cu_host, const int32_t* budgets, const float* lse_opt, void* k_out, void* v_out,
+                  int64_t capacity,
                   int32_t* offsets, int32_t* kept_idx, float* pooled_opt, int32_t* status, void* ws,
                   size_t ws_bytes, cudaStream_t st, bool overlapped = false) {
   g_last_launches = 0;
@@ -414,6 +444,7 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
     ++os->seq;
     pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
     pb.tab.cu_ptr = cu_dev;
+    pb.lse_opt = lse_opt;
     // the score kernels leave a few SMs to the selection kernels of the layers before this one
     int sms = 148;
     int dev = 0;
@@ -432,7 +463,10 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
       if (cur.plan.n_cta == 0) pipe = false;                        // no history: nothing to score
     }
     const bool queued = !os->queue.empty() || os->pending.valid;
-    if (queued && (!pipe || (os->queue.empty() ? os->pending.st : os->queue[0].st) != st)) {
+    // a queue holds layers of one kind (both passes, or the vote pass alone) and of one stream
+    const bool other_kind = os->pending.valid ? lse_opt != nullptr
+                                              : (!os->queue.empty() && (os->queue[0].pb.lse_opt != nullptr) != (lse_opt != nullptr));
+    if (queued && (!pipe || other_kind || (os->queue.empty() ? os->pending.st : os->queue[0].st) != st)) {
       e = flush_pending(os, &launches);
       if (e != cudaSuccess) return cuda_fail(e);
     }
@@ -441,6 +475,8 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
     if (pipe) {
       // Queue the layer; the score kernel takes a list of layers per launch (pass 1 of each beside pass 2 of the
       // one before) and goes out when the list is full and one more layer has come, or at a join.
+      rc = enqueue_window_stats(pb, path, st, &launches);
+      if (rc != SLKV_OK) return rc;
       os->queue.push_back(cur);
       if ((int)os->queue.size() > kPipeMaxLayers) {
         e = launch_queue(os, kPipeMaxLayers, false, &launches);
@@ -459,6 +495,7 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
   if (rc != SLKV_OK) return rc;
   pb.cu = cu_dev; pb.q = q_win; pb.k = k; pb.v = v;
   pb.tab.cu_ptr = cu_dev;
+  pb.lse_opt = lse_opt;
   const bool clustered = select_cluster_supported(pb);
   if (!clustered || pb.tab.n_inline == 0) {       // tables in global memory and / or the packed offsets
     e = launch_setup(pb, clustered ? nullptr : budgets, offsets, capacity, status, st, &launches);
@@ -548,7 +585,8 @@ int slkv_profile_collect(float* total_ms, int32_t* launches, int32_t n_kernels) 
 
 const char* slkv_kernel_name(int kernel_id) {
   static const char* names[KID_COUNT] = {"k_setup", "k_score_lse", "k_score_vote", "k_pool", "k_select",
-                                         "k_gather", "k_alloc", "k_score_fused", "k_score_pipe"};
+                                         "k_gather", "k_alloc", "k_score_fused", "k_score_pipe", "k_window_stats",
+                                         "k_merge_lse"};
   return (kernel_id >= 0 && kernel_id < KID_COUNT) ? names[kernel_id] : "";
 }
 
@@ -561,7 +599,12 @@ int slkv_trace_set_buffer(void* dev_buf, size_t bytes) {
 
 int slkv_last_cuda_error(void) { return g_last_cuda_error; }
 int slkv_last_launch_count(void) { return g_last_launches; }
-int slkv_version(void) { return 100; }
+int slkv_version(void) { return 200; }
+
+int slkv_debug_expire_next_wait(int on) {
+  expire_next_wait(on != 0);
+  return SLKV_OK;
+}
 
 int slkv_alloc_budgets(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
                        int32_t* budgets, int32_t* status, void* stream) {
@@ -589,8 +632,8 @@ size_t slkv_workspace_bytes_overlapped(const slkv_params* p, const int32_t* cu_s
 
 int slkv_compress_overlapped(const slkv_params* p, const void* q_win, const void* k, const void* v,
                              const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
-                             void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets,
-                             int32_t* kept_idx, float* pooled_opt, int32_t* status, void* workspace,
+                             const float* lse_opt, void* k_out, void* v_out, int64_t out_capacity_rows,
+                             int32_t* offsets, int32_t* kept_idx, float* pooled_opt, int32_t* status, void* workspace,
                              size_t workspace_bytes, void* stream) {
   {
     Problem pb;                                   // the overlapped layout is the larger one: check it up front
@@ -598,8 +641,9 @@ int slkv_compress_overlapped(const slkv_params* p, const void* q_win, const void
         workspace_bytes < layout_of(pb, true).total)
       return SLKV_ERR_WORKSPACE;
   }
-  return compress_impl(p, q_win, k, v, cu_seqlens_dev, cu_seqlens_host, budgets, k_out, v_out, out_capacity_rows,
-                       offsets, kept_idx, pooled_opt, status, workspace, workspace_bytes, (cudaStream_t)stream, true);
+  return compress_impl(p, q_win, k, v, cu_seqlens_dev, cu_seqlens_host, budgets, lse_opt, k_out, v_out,
+                       out_capacity_rows, offsets, kept_idx, pooled_opt, status, workspace, workspace_bytes,
+                       (cudaStream_t)stream, true);
 }
 
 int slkv_join(void* stream) {
@@ -622,11 +666,13 @@ int64_t slkv_packed_rows_upper_bound(const slkv_params* p, const int32_t* cu_seq
   return (int64_t)pb.p.n_kv_heads * pb.total_tokens;
 }
 
-int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
-               const int32_t* cu_seqlens_host, float* pooled, int32_t* status, void* workspace,
-               size_t workspace_bytes, void* stream) {
+namespace {
+// slkv_score and slkv_row_lse: the votes pooled into `pooled`, or the rows' log-sum-exp into `lse_out`.
+int score_impl(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+               const int32_t* cu_seqlens_host, const float* lse_opt, float* pooled, float* lse_out, int32_t* status,
+               void* workspace, size_t workspace_bytes, void* stream) {
   g_last_launches = 0;
-  if (!q_win || !k || !cu_seqlens_dev || !pooled) return SLKV_ERR_NULL_PTR;
+  if (!q_win || !k || !cu_seqlens_dev || (!pooled && !lse_out)) return SLKV_ERR_NULL_PTR;
   Problem pb;
   int rc = describe(p, cu_seqlens_host, &pb);
   if (rc != SLKV_OK) return rc;
@@ -638,6 +684,7 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
   if (rc != SLKV_OK) return rc;
   pb.cu = cu_seqlens_dev; pb.q = q_win; pb.k = k; pb.v = nullptr;
   pb.tab.cu_ptr = cu_seqlens_dev;
+  pb.lse_opt = lse_opt;
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
   cudaError_t e = join_overlapped(st, &launches);  // the workspace may still serve an overlapped call
@@ -646,6 +693,19 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
     e = launch_setup(pb, nullptr, nullptr, 0, nullptr, st, &launches);
     if (e != cudaSuccess) return cuda_fail(e);
   }
+  if (lse_out) {
+    // row statistics only: pass 1, the window keys' share where the domain has one, then the merge
+    rc = enqueue_window_stats(pb, path, st, &launches);
+    if (rc != SLKV_OK) return rc;
+    e = path == SLKV_PATH_TENSOR ? launch_score_tensor(pb, cu_seqlens_host, status, 1, st, &launches)
+                                 : launch_score_simt(pb, 1, st, &launches);
+    if (e == cudaSuccess)
+      e = path == SLKV_PATH_TENSOR ? launch_merge_lse_tensor(pb, cu_seqlens_host, lse_out, st, &launches)
+                                   : launch_merge_lse_simt(pb, lse_out, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_last_launches = launches;
+    return SLKV_OK;
+  }
   rc = enqueue_votes(pb, path, cu_seqlens_host, status, st, &launches);
   if (rc != SLKV_OK) return rc;
   e = launch_pool(pb, pooled, st, &launches);
@@ -653,13 +713,48 @@ int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int
   g_last_launches = launches;
   return SLKV_OK;
 }
+}  // namespace
+
+int slkv_score(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+               const int32_t* cu_seqlens_host, const float* lse_opt, float* pooled, int32_t* status, void* workspace,
+               size_t workspace_bytes, void* stream) {
+  if (!pooled) return SLKV_ERR_NULL_PTR;
+  return score_impl(p, q_win, k, cu_seqlens_dev, cu_seqlens_host, lse_opt, pooled, nullptr, status, workspace,
+                    workspace_bytes, stream);
+}
+
+int slkv_row_lse(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+                 const int32_t* cu_seqlens_host, float* lse_out, int32_t* status, void* workspace,
+                 size_t workspace_bytes, void* stream) {
+  if (!lse_out) return SLKV_ERR_NULL_PTR;
+  return score_impl(p, q_win, k, cu_seqlens_dev, cu_seqlens_host, nullptr, nullptr, lse_out, status, workspace,
+                    workspace_bytes, stream);
+}
+
+}  // extern "C"
+
+// Host-side validation of slkv_score's arguments without a workspace (for entry points that bring their own).
+int slkv::check_score_args(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+                           const int32_t* cu_seqlens_host, const float* pooled) {
+  if (!q_win || !k || !cu_seqlens_dev || !pooled) return SLKV_ERR_NULL_PTR;
+  Problem pb;
+  int rc = describe(p, cu_seqlens_host, &pb);
+  if (rc != SLKV_OK) return rc;
+  if (!aligned16(q_win) || !aligned16(k)) return SLKV_ERR_BAD_ALIGN;
+  int path = 0;
+  return resolve_path(pb, &path);
+}
+
+extern "C" {
 
 int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const void* v,
                   const int32_t* cu_seqlens_dev, const int32_t* cu_seqlens_host, const int32_t* budgets,
-                  void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets, int32_t* kept_idx,
-                  float* pooled_opt, int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
-  return compress_impl(p, q_win, k, v, cu_seqlens_dev, cu_seqlens_host, budgets, k_out, v_out, out_capacity_rows,
-                       offsets, kept_idx, pooled_opt, status, workspace, workspace_bytes, (cudaStream_t)stream);
+                  const float* lse_opt, void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets,
+                  int32_t* kept_idx, float* pooled_opt, int32_t* status, void* workspace, size_t workspace_bytes,
+                  void* stream) {
+  return compress_impl(p, q_win, k, v, cu_seqlens_dev, cu_seqlens_host, budgets, lse_opt, k_out, v_out,
+                       out_capacity_rows, offsets, kept_idx, pooled_opt, status, workspace, workspace_bytes,
+                       (cudaStream_t)stream);
 }
 
 // ---- host-buffer variant ---------------------------------------------------------------------------
@@ -747,7 +842,7 @@ int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, c
   SLKV_CP(b + A.cu, cu_seqlens_host, (size_t)(p->n_seqs + 1) * 4, cudaMemcpyHostToDevice);
   SLKV_CP(b + A.budgets, budgets, (size_t)p->n_kv_heads * 4, cudaMemcpyHostToDevice);
   rc = compress_impl(p, b + A.q, b + A.k, b + A.v, reinterpret_cast<int32_t*>(b + A.cu), cu_seqlens_host,
-                     reinterpret_cast<int32_t*>(b + A.budgets), b + A.k_out, b + A.v_out, out_capacity_rows,
+                     reinterpret_cast<int32_t*>(b + A.budgets), nullptr, b + A.k_out, b + A.v_out, out_capacity_rows,
                      reinterpret_cast<int32_t*>(b + A.offsets), reinterpret_cast<int32_t*>(b + A.kept), nullptr,
                      nullptr, b + A.ws, arena_bytes - A.ws, st);
   if (rc != SLKV_OK) return rc;

@@ -34,6 +34,25 @@ struct SeqTables {
 #endif
 };
 
+// Where a vote pass takes the window rows' log-sum-exp from when it does not merge the row statistics of the keys
+// it scored itself alone: the caller's array (lse_opt of the public entry points), and / or the statistics of the
+// window keys (softmax over all causally visible keys).  Row r of a segment is query head g*G + hh, window row i with
+// r = i*G + hh (head_inner) or r = hh*window + i.
+struct LseSource {
+  const float* lse_opt;     // [n_seqs][n_q_heads][window], or null
+  const float* win_m;       // [n_seg][R] maxima (log2 units) over the window keys a row sees, or null
+  const float* win_z;       // [n_seg][R] sums of 2^(x - max) over them
+  float to_log2;            // lse_opt * to_log2 is in log2 units
+  int n_q_heads;
+#ifdef __CUDACC__
+  __device__ __forceinline__ float caller_lse(int s, int g, int r, int G, int window, bool head_inner) const {
+    const int hh = head_inner ? r % G : r / window;
+    const int i = head_inner ? r / G : r - hh * window;
+    return lse_opt[((long long)s * n_q_heads + g * G + hh) * window + i] * to_log2;
+  }
+#endif
+};
+
 // Programmatic dependent launch: a kernel may start while its predecessor in the stream drains; it must
 // not touch global memory the predecessor may write before pdl_wait() returns.
 #ifdef __CUDACC__
@@ -93,11 +112,14 @@ struct Problem {
   float* pooled_ws;       // [n_kv_heads * total_hist] used when the caller wants no pooled output
   int32_t* gather_src;    // [n_kv_heads * total_tokens] per packed row: token * n_kv_heads + head of its source
   int32_t* dev_flags;     // [8] scratch words (timeouts etc.)
+  float* win_m;           // [n_seg][R] row statistics over the window keys (SLKV_ALL_CAUSAL without lse_opt)
+  float* win_z;
+  const float* lse_opt;   // the caller's row log-sum-exps, or null
   int max_score_ctas;     // > 0: the score kernels use at most this many CTAs (SMs); 0 = all
 };
 
 // kernel ids for launch accounting / per-kernel timing
-enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_SCORE_PIPE, KID_COUNT };
+enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_SCORE_PIPE, KID_WINDOW_STATS, KID_MERGE_LSE, KID_COUNT };
 
 // Brackets one kernel launch: counts it and, when per-kernel timing is on for this thread, records a
 // CUDA event pair around it on the launch stream.
@@ -107,6 +129,10 @@ struct LaunchScope {
   int kid_; cudaStream_t st_; int slot_;
 };
 
+// slkv_score's host-side argument checks, without a workspace: SLKV_OK or the status slkv_score would return
+int check_score_args(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
+                     const int32_t* cu_seqlens_host, const float* pooled);
+
 // host-side launchers; each returns a cudaError_t and adds to *launches
 cudaError_t launch_alloc(const float* inf, int n_layers, int n_heads, int fixed, long long total, int32_t* budgets,
                          int32_t* status, cudaStream_t st);
@@ -114,12 +140,25 @@ cudaError_t launch_setup(const Problem& pb, const int32_t* budgets, int32_t* off
                          int32_t* status, cudaStream_t st, int* launches);
 int simt_chunk_keys();
 size_t simt_smem_bytes(const Problem& pb);
-cudaError_t launch_score_simt(const Problem& pb, cudaStream_t st, int* launches);
+// passes: 1 = row statistics only, 2 = votes only (the log-sum-exps come from lse_source_of), 3 = both
+cudaError_t launch_score_simt(const Problem& pb, int passes, cudaStream_t st, int* launches);
+// Row statistics of the window keys each window row sees causally (SLKV_ALL_CAUSAL) -> pb.win_m / pb.win_z, rows in
+// the order of the score path (head_inner: r = i*G + hh).
+cudaError_t launch_window_stats(const Problem& pb, bool head_inner, cudaStream_t st, int* launches);
+// Merges the per-chunk (SIMT layout) or per-CTA (tensor layout, schedule in `plan`) row statistics and the window
+// statistics, if any, into lse_out[n_seqs][n_q_heads][window] in the problem's lse_units.
+cudaError_t launch_merge_lse_simt(const Problem& pb, float* lse_out, cudaStream_t st, int* launches);
+cudaError_t launch_merge_lse_tensor(const Problem& pb, const int32_t* cu_host, float* lse_out, cudaStream_t st,
+                                    int* launches);
+LseSource lse_source_of(const Problem& pb);
+float lse_out_scale(const Problem& pb);          // log2 units -> the problem's lse_units
+bool tensor_q_head_inner(const slkv_params& p);
 bool tensor_path_supported(const slkv_params& p);
 int tensor_slot_stride(const Problem& pb);
 void set_tensor_trace(void* dev_buf, size_t bytes);
-cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, cudaStream_t st,
-                                int* launches);
+// passes as launch_score_simt
+cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, int passes,
+                                cudaStream_t st, int* launches);
 cudaError_t launch_pool(const Problem& pb, float* pooled, cudaStream_t st, int* launches);
 cudaError_t launch_select(const Problem& pb, const float* pooled, const int32_t* budgets, const int32_t* offsets,
                           int32_t* kept_idx, int64_t capacity, cudaStream_t st, int* launches);
@@ -140,9 +179,12 @@ struct TcArgs {
   float* part_m;
   float* part_z;
   float* vote;
+  LseSource lse;
   int32_t* status;
   unsigned long long* trace;    // optional timeline buffer: kTraceSlots timestamps (ns) per CTA, or null
   int n_seqs, n_kv_heads, G, window, R, MT, n_stages, slot_stride, tiles_per_cta, total_tiles, barrier_slot;
+  int fresh_inputs;             // vote pass only: no kernel of this library has read Q and K before this launch
+  int barrier_extra;            // 0; 1 makes the grid-wide wait expect an arrival that never comes (diagnostics)
   int q_head_inner, k_head_inner;   // tensor-map dimension order: 1 = the head axis comes before the row axis
   float scale_log2;
 };
@@ -158,13 +200,18 @@ struct TcPlan {
 cudaError_t plan_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, TcPlan* plan);
 // Timeline buffer of this thread (diagnostics), or null: half 0 / 1, kTraceSlots words per CTA.
 unsigned long long* tensor_trace_buffer(int half, int n_cta);
+// Diagnostics: arm / consume the one-shot switch that makes the next inter-CTA wait of this thread's launches run out.
+void expire_next_wait(int on);
+int take_expire_next_wait();
 
 // Several layers per launch, pass 1 of one layer beside pass 2 of the layer before: pass 1 of a[0..n_a), pass 2 of
 // `pending` (pass 1 done by an earlier launch; may be null) and of a[0..n_a-1), or of all of a[] when `finish`.
 // All plans share one shape.  The shapes it takes:
 bool score_pipe_supported(const Problem& pb);
 constexpr int kPipeMaxLayers = 8;
-cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int n_a, bool finish, cudaStream_t st,
-                              int* launches);
+// votes_only: every plan carries the caller's row statistics, so both streams run pass 2 (no pending layer before or
+// after the launch, no CTA waits for another).
+cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int n_a, bool finish, bool votes_only,
+                              cudaStream_t st, int* launches);
 
 }  // namespace slkv

@@ -46,20 +46,20 @@ size_t slkv_noalloc_scratch_bytes(void) { return kScratchBytes; }
 int slkv_noalloc_last_cuda_error(void) { return g_noalloc_cuda_error; }
 
 int slkv_score_noalloc(const slkv_params* p, const void* q_win, const void* k, const int32_t* cu_seqlens_dev,
-                       const int32_t* cu_seqlens_host, float* pooled, int32_t* status, void* stream) {
-  if (!p || !cu_seqlens_host) return SLKV_ERR_NULL_PTR;
+                       const int32_t* cu_seqlens_host, const float* lse_opt, float* pooled, int32_t* status,
+                       void* stream) {
+  // the argument checks of slkv_score first, so that a bad call gets the same status from either entry point
+  int rc = slkv::check_score_args(p, q_win, k, cu_seqlens_dev, cu_seqlens_host, pooled);
+  if (rc != SLKV_OK) return rc;
   const size_t need = slkv_workspace_bytes(p, cu_seqlens_host);
-  if (need == 0) {
-    // let the ordinary entry point name the argument error (it fails before touching the workspace)
-    return slkv_score(p, q_win, k, cu_seqlens_dev, cu_seqlens_host, pooled, status,
-                      reinterpret_cast<void*>(uintptr_t(256)), ~size_t(0), stream);
-  }
-  if (need > kScratchBytes) return SLKV_ERR_WORKSPACE;          // shapes beyond the built-in scratch
+  if (need == 0 || need > kScratchBytes) return SLKV_ERR_WORKSPACE;          // shapes beyond the built-in scratch
   void* scratch = nullptr;
-  int rc = scratch_of_current_device(&scratch, &g_noalloc_cuda_error);
+  g_noalloc_cuda_error = 0;
+  rc = scratch_of_current_device(&scratch, &g_noalloc_cuda_error);
   if (rc != SLKV_OK) return rc;
   // Nothing in the scratch has to start at zero: every kernel writes the part it later reads.
-  return slkv_score(p, q_win, k, cu_seqlens_dev, cu_seqlens_host, pooled, status, scratch, kScratchBytes, stream);
+  return slkv_score(p, q_win, k, cu_seqlens_dev, cu_seqlens_host, lse_opt, pooled, status, scratch, kScratchBytes,
+                    stream);
 }
 
 }  // extern "C"

@@ -58,6 +58,7 @@ struct LayerDesc {
   float* part_m;
   float* part_z;
   float* vote;
+  LseSource lse;               // where pass 2 takes the rows' log-sum-exp from besides this launch's / the last launch's pass 1
   int32_t* status;
   int tile_begin, tile_end;    // the entry's tiles in the layer's tile list; CTA b takes tiles_per_cta of them from
                                // tile_begin + b * tiles_per_cta
@@ -67,6 +68,8 @@ struct PipeArgs {
   LayerDesc lay[kMaxLay];
   int a_first, a_last;         // stream A: pass 1 of layers a_first..a_last (none if a_first > a_last)
   int b_first, b_last;         // stream B: pass 2 of layers b_first..b_last
+  int step;                    // 1; 2 when both streams run pass 2 (the callers supplied the row statistics): stream A
+                               // takes entries a_first, a_first + 2, ..., stream B entries b_first, b_first + 2, ...
   unsigned* counters;          // [kMaxLay] CTAs that have published the layer's row statistics, then [1] CTAs that are done
   unsigned target[kMaxLay];    // value a layer's counter reaches when all CTAs of this launch have published
 };
@@ -87,6 +90,7 @@ struct StreamCtx {
   __device__ __forceinline__ uint32_t acce_bar(int b) const { return bar0 + 8u * (8 + b); }
   __device__ __forceinline__ uint32_t qfull_bar() const { return bar0 + 8u * 10; }
   __device__ __forceinline__ uint32_t qempty_bar() const { return bar0 + 8u * 11; }
+  __device__ __forceinline__ uint32_t drain_bar() const { return bar0 + 8u * 12; }   // used only when a wait ran out
 };
 
 // sum_e 2^(v_e * sc - m) over 32 accumulator values.  All exponentials on the special-function unit: with sixteen
@@ -112,14 +116,14 @@ __device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, %
 // ---- one thread: TMA loads of the stream's Q tiles and K tiles ------------------------------------------
 template <bool VOTE>
 __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, const LayerDesc* lay, int first, int last,
-                                         int new_from) {
+                                         int step, int new_from) {
   int it = 0, run_idx = 0, st = 0;
   uint32_t st_phase = 0;
   bool ok = true;
   // Every K tile is read twice, by pass 1 and a layer later by pass 2, in the same order: pass 1 asks L2 to keep the
   // lines, pass 2 to drop them first, so that about one layer's K is live in L2 and pass 2 need not go to HBM.
   const uint64_t policy = VOTE ? l2_policy_evict_first() : l2_policy_evict_last();
-  for (int j = first; j <= last && ok; ++j) {
+  for (int j = first; j <= last && ok; j += step) {
     if (j == new_from || (j == first && j > new_from)) pdl_wait();   // inputs this launch is the first to read
     if (!VOTE) {
       // Pass 1 stays at most one layer ahead of this CTA's pass 2 (which needs the other CTAs' pass 1 of the layer
@@ -172,7 +176,8 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
 
 // ---- one thread: the stream's MMAs, one 128 x 128 x 128 product per tile into one of two accumulators --------
 template <bool VOTE>
-__device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, const LayerDesc* lay, int first, int last) {
+__device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, const LayerDesc* lay, int first, int last,
+                                       int step) {
   // pass 1: D[row, key] = Q K^T (A = Q, B = K); pass 2: D[key, row] = K Q^T (A = K, B = Q, N = R)
   const uint32_t idesc = VOTE ? instr_desc(kTileKeys, a.R) : instr_desc(128, kTileKeys);
   const uint64_t q_desc0 = smem_desc(c.q_smem), k_desc0 = smem_desc(c.k_smem);
@@ -181,7 +186,7 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, cons
   uint32_t st_phase = 0, b_phase = 0;
   uint64_t k_desc = k_desc0;
   bool ok = true;
-  for (int j = first; j <= last && ok; ++j) {
+  for (int j = first; j <= last && ok; j += step) {
   int begin, end;
   entry_range(a, lay[j], begin, end);
   for (int pos = begin; pos < end && ok;) {
@@ -209,6 +214,12 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, cons
     pos += r.count;
     ++run_idx;
   }
+  }
+  if (!ok) {
+    // gave up: the MMAs this thread has issued must be through before the accumulators are released
+    tc_commit(c.drain_bar());
+    const unsigned long long t0 = now_ns();
+    while (!mbar_try(c.drain_bar(), 0) && now_ns() - t0 < kWaitLimitNs) {}
   }
 }
 
@@ -319,8 +330,10 @@ __device__ __forceinline__ float vote_chunk(const uint32_t (&r)[32], float sc, c
 }
 
 // ---- 256 threads: pass 2, votes (stream B) ---------------------------------------------------------------------
+// `first`, `last`, pa.step: the entries this stream takes; `bar_id`: the named barrier of its 256 threads; `is_b`: the
+// stream pass 1 of the same CTA keeps its distance to.
 __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs& a, const PipeArgs& pa, int et, int warp,
-                                               float* lse2) {
+                                               float* lse2, int first, int last, int bar_id, bool is_b) {
   const int wg = et >> 7, row = et & 127, lane = et & 31;
   const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
   const float sc = a.scale_log2;
@@ -328,9 +341,9 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
   const int R = a.R;
   int it = 0, run_idx = 0;
   bool ok = true;
-  for (int j = pa.b_first; j <= pa.b_last; ++j) {
+  for (int j = first; j <= last; j += pa.step) {
   const LayerDesc& L = pa.lay[j];
-  if (j >= pa.a_first && j <= pa.a_last) {
+  if (pa.step == 1 && j >= pa.a_first && j <= pa.a_last && !L.lse.lse_opt) {
     // the layer's pass 1 is part of this launch: wait until every CTA has published its row statistics (all CTAs
     // are resident, and stream A waits for nothing, so the count gets there; bounded all the same)
     if (et == 0 && ok) {
@@ -343,11 +356,11 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
         __nanosleep(64);
       }
     }
-    named_bar(2);
+    named_bar(bar_id);
     ok = ok && *c.abort_flag == 0;
   }
-  if (et == 0) *c.b_layer = j;
-  if (et == 0 && j < 24) trace_mark(a.trace, 9 + 2 * j);
+  if (et == 0 && is_b) *c.b_layer = j;
+  if (et == 0 && is_b && j < 24) trace_mark(a.trace, 9 + 2 * j);
   int begin, end;
   entry_range(a, L, begin, end);
   for (int pos = begin; pos < end;) {
@@ -356,42 +369,24 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
     const int first_cta = (r.seg_tile0 - L.tile_begin) / a.tiles_per_cta;
     float* lse = lse2 + 128 * (run_idx & 1);
     {
-      // merge the per-CTA partials of this segment into the rows' log-sum-exp (log2 units): two neighbouring
-      // lanes share a row (even / odd slots), all loads in flight before the first use
+      // the rows' log-sum-exp (log2 units): the caller's, or the per-CTA partials of this segment merged (two
+      // neighbouring lanes share a row)
       const int n_slots = (r.seg_tile0 - L.tile_begin + r.tiles_seg - 1) / a.tiles_per_cta - first_cta + 1;
       const int rr = (et >> 1) < R ? (et >> 1) : -1;
       const int half = et & 1;
-      float M = -INFINITY, Z = 0.f;
-      if (rr >= 0) {
-        const float* pm = L.part_m + (long long)seg * a.slot_stride * R + rr;      // [segment][slot][row]
-        const float* pz = L.part_z + (long long)seg * a.slot_stride * R + rr;
-        for (int c0 = half; c0 < n_slots; c0 += 24) {
-          float m12[12], z12[12];
-#pragma unroll
-          for (int u = 0; u < 12; ++u) {
-            const int cc = c0 + u * 2;
-            const bool in = cc < n_slots;
-            m12[u] = in ? __ldcg(pm + (long long)cc * R) : -INFINITY;
-            z12[u] = in ? __ldcg(pz + (long long)cc * R) : 0.f;
-          }
-#pragma unroll
-          for (int u = 0; u < 12; ++u)
-            if (z12[u] > 0.f) {                                       // empty partials carry z = 0
-              const float Mn = fmaxf(M, m12[u]);
-              Z = Z * ex2(M - Mn) + z12[u] * ex2(m12[u] - Mn);      // ex2(-inf) = 0 covers the first term
-              M = Mn;
-            }
-        }
+      float l2;
+      if (L.lse.lse_opt) {
+        l2 = rr >= 0 ? L.lse.caller_lse(r.s, r.g, rr, a.G, a.window, a.q_head_inner != 0) : 0.f;
+      } else {
+        const bool has_win = L.lse.win_m != nullptr && rr >= 0;
+        l2 = merged_row_lse(L.part_m + (long long)seg * a.slot_stride * R, L.part_z + (long long)seg * a.slot_stride * R,
+                            n_slots, R, rr, half, 2, has_win, has_win ? L.lse.win_m[(long long)seg * R + rr] : 0.f,
+                            has_win ? L.lse.win_z[(long long)seg * R + rr] : 0.f);
       }
-      const float M1 = __shfl_xor_sync(0xffffffffu, M, 1), Z1 = __shfl_xor_sync(0xffffffffu, Z, 1);
-      const float Mn = fmaxf(M, M1);
-      float Zt = 0.f;
-      if (M > -INFINITY) Zt += Z * ex2(M - Mn);
-      if (M1 > -INFINITY) Zt += Z1 * ex2(M1 - Mn);
-      if (half == 0 && rr >= 0) lse[rr] = Mn + log2f(Zt);
+      if (half == 0 && rr >= 0) lse[rr] = l2;
     }
-    named_bar(2);
-    if (et == 0 && run_idx == 0) trace_mark(a.trace, 3);
+    named_bar(bar_id);
+    if (et == 0 && is_b && run_idx == 0) trace_mark(a.trace, 3);
     for (int i = 0; i < r.count; ++i, ++it) {
       if ((it & 1) != wg) continue;
       const int b = it & 1;
@@ -431,6 +426,8 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
   }
 }
 
+// DUAL: both streams run pass 2 (every layer of the list came with its row statistics), each on every other entry.
+template <bool DUAL>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 k_score_pipe(const __grid_constant__ PipeArgs pa) {
   // Shared memory, all dynamic and 1024-byte aligned (the swizzled tiles need it):
@@ -482,6 +479,7 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
       for (int b = 0; b < 2; ++b) { mbar_init(c.accf_bar(b), 1); mbar_init(c.acce_bar(b), 4); }
       mbar_init(c.qfull_bar(), 1);
       mbar_init(c.qempty_bar(), 1);
+      mbar_init(c.drain_bar(), 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -507,25 +505,33 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   // which are inputs, and for the pending layer have been read by the launch before: they start at once; its
   // epilogue needs that launch's row statistics and waits.
   if (warp == 0) {
-    if (lane == 0 && has_a) producer<false>(ca, a, pa.lay, pa.a_first, pa.a_last, pa.a_first);
+    if (lane == 0 && has_a) {
+      if (DUAL) producer<true>(ca, a, pa.lay, pa.a_first, pa.a_last, pa.step, pa.a_first);
+      else producer<false>(ca, a, pa.lay, pa.a_first, pa.a_last, 1, pa.a_first);
+    }
   } else if (warp == 1) {
-    if (lane == 0 && has_a) issuer<false>(ca, a, pa.lay, pa.a_first, pa.a_last);
+    if (lane == 0 && has_a) {
+      if (DUAL) issuer<true>(ca, a, pa.lay, pa.a_first, pa.a_last, pa.step);
+      else issuer<false>(ca, a, pa.lay, pa.a_first, pa.a_last, 1);
+    }
   } else if (warp == 2) {
-    if (lane == 0 && has_b) producer<true>(cb, a, pa.lay, pa.b_first, pa.b_last, 1);   // layer 0 was read before
+    // normally entry 0 was read by the launch before; with both streams on pass 2 every entry is new to this launch
+    if (lane == 0 && has_b) producer<true>(cb, a, pa.lay, pa.b_first, pa.b_last, pa.step, DUAL ? pa.b_first : 1);
   } else if (warp == 3) {
-    if (lane == 0 && has_b) issuer<true>(cb, a, pa.lay, pa.b_first, pa.b_last);
+    if (lane == 0 && has_b) issuer<true>(cb, a, pa.lay, pa.b_first, pa.b_last, pa.step);
   } else if (warp < 12) {
     if (has_a) {
       pdl_wait();
       if (tid == 128) trace_mark(a.trace, 1);
-      epilogue_rows(ca, a, pa, tid - 128, warp, stat_m, stat_z);
+      if (DUAL) epilogue_votes(ca, a, pa, tid - 128, warp, stat_m, pa.a_first, pa.a_last, 1, false);
+      else epilogue_rows(ca, a, pa, tid - 128, warp, stat_m, stat_z);
       if (tid == 128) trace_mark(a.trace, 5);
     }
   } else {
     if (has_b) {
       pdl_wait();
       if (tid == 384) trace_mark(a.trace, 7);
-      epilogue_votes(cb, a, pa, tid - 384, warp, lse2);
+      epilogue_votes(cb, a, pa, tid - 384, warp, lse2, pa.b_first, pa.b_last, 2, true);
       if (tid == 384) trace_mark(a.trace, 6);
     }
   }
@@ -560,9 +566,10 @@ bool score_pipe_supported(const Problem& pb) {
 
 // One launch: pass 1 of plans a[0..n_a) beside pass 2 of `pending` (the layer whose pass 1 an earlier launch did;
 // may be null) and of a[0..n_a-1), or of all of a[] when `finish` is set.  The plans share one shape and schedule.
-cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int n_a, bool finish, cudaStream_t st,
-                              int* launches) {
+cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int n_a, bool finish, bool votes_only,
+                              cudaStream_t st, int* launches) {
   if (n_a > kPipeMaxLayers) return cudaErrorInvalidValue;
+  if (votes_only && pending) return cudaErrorInvalidValue;     // nothing stays pending between vote-only launches
   // Without cooperative launches (refused once on this device) no launch may hold both passes of a layer: one layer's
   // pass 1 per launch, beside pass 2 of the layer before.
   static thread_local bool no_coop[64] = {};
@@ -573,14 +580,15 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
   {
     int d = 0;
     if (env_no_coop && cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < 64) no_coop[d] = true;
-    if (cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < 64 && no_coop[d] && (n_a > 1 || (n_a == 1 && finish))) {
+    if (!votes_only && cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < 64 && no_coop[d] &&
+        (n_a > 1 || (n_a == 1 && finish))) {
       const TcPlan* prev = pending;
       for (int i = 0; i < n_a; ++i) {
-        cudaError_t e1 = launch_score_pipe(prev, a + i, 1, false, st, launches);
+        cudaError_t e1 = launch_score_pipe(prev, a + i, 1, false, false, st, launches);
         if (e1 != cudaSuccess) return e1;
         prev = a[i];
       }
-      return finish ? launch_score_pipe(prev, nullptr, 0, true, st, launches) : cudaSuccess;
+      return finish ? launch_score_pipe(prev, nullptr, 0, true, false, st, launches) : cudaSuccess;
     }
   }
   const TcPlan* any = pending && pending->n_cta > 0 ? pending : nullptr;
@@ -593,7 +601,9 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (configured_dev != dev) {
-    e = cudaFuncSetAttribute(k_score_pipe, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem);
+    e = cudaFuncSetAttribute(k_score_pipe<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_score_pipe<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem);
     if (e != cudaSuccess) return e;
     void* sym = nullptr;
     e = cudaGetSymbolAddress(&sym, g_layer_published);
@@ -630,6 +640,7 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
     pa.lay[j].tm_q = p->tm_q; pa.lay[j].tm_k = p->tm_k;
     pa.lay[j].part_m = p->a.part_m; pa.lay[j].part_z = p->a.part_z; pa.lay[j].vote = p->a.vote;
     pa.lay[j].status = p->a.status;
+    pa.lay[j].lse = p->a.lse;
     pa.lay[j].tile_begin = groups == 2 ? group * (total / 2) : 0;
     pa.lay[j].tile_end = groups == 2 ? (group + 1) * (total / 2) : total;
   };
@@ -642,13 +653,20 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
   pa.a_first = 1; pa.a_last = n_live;
   pa.b_first = has_pending ? 0 : 1;
   pa.b_last = finish ? n_live : n_live - 1;
+  pa.step = 1;
+  if (votes_only) {                                   // both streams on pass 2, every other entry each
+    pa.step = 2;
+    pa.b_first = 2;
+    pa.b_last = n_live;
+  }
   if (pa.a_first > pa.a_last && pa.b_first > pa.b_last) return cudaSuccess;
   pa.base.trace = tensor_trace_buffer(0, n_cta);
   // counters of this launch: a slot of the table, zeroed on the stream before the kernel
   static std::atomic<unsigned> launch_seq{0};
   pa.counters = counters_base + (size_t)(launch_seq.fetch_add(1) % kCountSlots) * kCountWords;
-  for (int j = 0; j < kMaxLay; ++j) pa.target[j] = (unsigned)n_cta;
-  const bool waits_inside = pa.b_last >= pa.a_first && pa.a_last >= pa.a_first;   // a layer's two passes in one launch
+  const bool waits_inside = !votes_only && pa.b_last >= pa.a_first && pa.a_last >= pa.a_first;   // a layer's two passes in one launch
+  const unsigned extra = waits_inside && take_expire_next_wait() ? 1u : 0u;       // diagnostics: a wait that runs out
+  for (int j = 0; j < kMaxLay; ++j) pa.target[j] = (unsigned)n_cta + extra;
   // CTAs that wait for one another must all be resident: cooperative launch.  Dependent launch on top where the
   // device takes both (the kernel waits for the launch before it exactly where it needs that launch's results).
   static thread_local int pdl_with_coop[64] = {};     // per device: 0 untried, 1 works, -1 refused
@@ -677,7 +695,7 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
     cudaError_t le;
     {
       LaunchScope scope(KID_SCORE_PIPE, st, launches);
-      le = cudaLaunchKernelEx(&cfg, k_score_pipe, pa);
+      le = votes_only ? cudaLaunchKernelEx(&cfg, k_score_pipe<true>, pa) : cudaLaunchKernelEx(&cfg, k_score_pipe<false>, pa);
     }
     if (le == cudaSuccess) {
       if (waits_inside && with_pdl) pc = 1;
@@ -689,7 +707,7 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
     if (with_pdl && pc != 1) { pc = -1; continue; }   // once more without dependent launch
     // cooperative launches do not work here: the list goes out one layer per launch from now on
     no_coop[dev < 64 ? dev : 0] = true;
-    return launch_score_pipe(pending, a, n_a, finish, st, launches);
+    return launch_score_pipe(pending, a, n_a, finish, votes_only, st, launches);
   }
   return cudaErrorLaunchFailure;
 }

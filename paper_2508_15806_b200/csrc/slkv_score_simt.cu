@@ -49,11 +49,24 @@ __device__ __forceinline__ float dot_row(const T* __restrict__ qrow /*smem*/, co
   return acc0 + acc1;
 }
 
+// Row log-sum-exp (log2 units) from the per-chunk statistics of the SIMT layout [row][chunk], the window keys'
+// statistics folded in when there are any (softmax over all causally visible keys).
+__device__ __forceinline__ float simt_row_lse(const float* pm, const float* pz, int nc, bool has_win, float wm,
+                                              float wz) {
+  float M = -INFINITY;
+  for (int c = 0; c < nc; ++c) M = fmaxf(M, pm[c]);
+  if (has_win) M = fmaxf(M, wm);
+  float Z = 0.f;
+  for (int c = 0; c < nc; ++c) Z = fmaf(pz[c], exp2f(pm[c] - M), Z);      // explicit rounding: the same in every kernel
+  if (has_win) Z = fmaf(wz, exp2f(wm - M), Z);
+  return __fadd_rn(M, log2f(Z));
+}
+
 template <typename T, int D, int PASS>
 __global__ void __launch_bounds__(kThreads)
 k_score_simt(const T* __restrict__ q, const T* __restrict__ k, const __grid_constant__ SeqTables tab,
              float* __restrict__ part_m, float* __restrict__ part_z,
-             float* __restrict__ vote, int n_kv_heads, int G, int window, int n_chunks, long long k_stride_tok,
+             float* __restrict__ vote, const LseSource lse, int n_kv_heads, int G, int window, int n_chunks, long long k_stride_tok,
              long long k_stride_head, long long q_stride_seq, long long q_stride_row, long long q_stride_head,
              float scale_log2) {
   constexpr int VN = Vec<T>::N;
@@ -87,13 +100,15 @@ k_score_simt(const T* __restrict__ q, const T* __restrict__ k, const __grid_cons
   } else {
     const int nc = (n_hist + kThreads * kTilesPerChunk - 1) / (kThreads * kTilesPerChunk);
     for (int r = tid; r < R; r += kThreads) {
+      if (lse.lse_opt) {                                                  // the caller's row statistics
+        run_m[r] = lse.caller_lse(s, g, r, G, window, false);
+        continue;
+      }
       const float* pm = part_m + ((long long)seg * R + r) * n_chunks;
       const float* pz = part_z + ((long long)seg * R + r) * n_chunks;
-      float M = -INFINITY;
-      for (int c = 0; c < nc; ++c) M = fmaxf(M, pm[c]);
-      float Z = 0.f;
-      for (int c = 0; c < nc; ++c) Z += pz[c] * exp2f(pm[c] - M);
-      run_m[r] = M + log2f(Z);
+      const bool has_win = lse.win_m != nullptr;
+      run_m[r] = simt_row_lse(pm, pz, nc, has_win, has_win ? lse.win_m[(long long)seg * R + r] : 0.f,
+                              has_win ? lse.win_z[(long long)seg * R + r] : 0.f);
     }
   }
   __syncthreads();
@@ -162,8 +177,75 @@ k_score_simt(const T* __restrict__ q, const T* __restrict__ k, const __grid_cons
   }
 }
 
+// Row statistics over the window keys a window row sees causally (its own position and the window keys before it):
+// one CTA per segment, one thread per row.  Only the all-causal softmax domain needs them.
 template <typename T, int D>
-cudaError_t launch_both(const Problem& pb, cudaStream_t st, int* launches) {
+__global__ void __launch_bounds__(kThreads)
+k_window_stats(const T* __restrict__ q, const T* __restrict__ k, const __grid_constant__ SeqTables tab,
+               float* __restrict__ win_m, float* __restrict__ win_z, int n_kv_heads, int G, int window, int head_inner,
+               long long k_stride_tok, long long k_stride_head, long long q_stride_seq, long long q_stride_row,
+               long long q_stride_head, float scale_log2) {
+  constexpr int VN = Vec<T>::N;
+  pdl_launch_dependents();
+  pdl_wait();
+  const int seg = blockIdx.x, s = seg / n_kv_heads, g = seg - s * n_kv_heads;
+  const int t0 = tab.cu_at(s);
+  const int n_hist = tab.cu_at(s + 1) - t0 - window;
+  if (n_hist <= 0) return;                                   // no history: nothing is scored
+  const int R = G * window;
+  for (int r = threadIdx.x; r < R; r += kThreads) {
+    const int hh = head_inner ? r % G : r / window;
+    const int i = head_inner ? r / G : r - hh * window;
+    const T* qrow = q + s * q_stride_seq + i * q_stride_row + (long long)(g * G + hh) * q_stride_head;
+    float m = -INFINITY, z = 0.f;
+    for (int j = 0; j <= i; ++j) {                           // window key j is token n_hist + j
+      const T* krow = k + (long long)(t0 + n_hist + j) * k_stride_tok + (long long)g * k_stride_head;
+      float acc0 = 0.f, acc1 = 0.f;
+      for (int c = 0; c < D / VN; ++c) {
+        float fq[VN], fk[VN];
+        unpack(*reinterpret_cast<const uint4*>(qrow + c * VN), fq, T());
+        unpack(*reinterpret_cast<const uint4*>(krow + c * VN), fk, T());
+#pragma unroll
+        for (int e = 0; e < VN; e += 2) {
+          acc0 = fmaf(fq[e], fk[e], acc0);
+          acc1 = fmaf(fq[e + 1], fk[e + 1], acc1);
+        }
+      }
+      const float x = (acc0 + acc1) * scale_log2;
+      const float mn = fmaxf(m, x);
+      z = z * exp2f(m - mn) + exp2f(x - mn);                 // exp2f(-inf) = 0 covers the first key
+      m = mn;
+    }
+    win_m[(long long)seg * R + r] = m;
+    win_z[(long long)seg * R + r] = z;
+  }
+}
+
+// lse_out[s][h][i] from the SIMT layout's per-chunk statistics (and the window statistics, if any).
+__global__ void __launch_bounds__(kThreads)
+k_merge_lse_simt(const float* __restrict__ part_m, const float* __restrict__ part_z, const LseSource lse,
+                 const __grid_constant__ SeqTables tab, float* __restrict__ lse_out, int n_kv_heads, int G, int window,
+                 int n_chunks, int chunk_keys, float out_scale) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int seg = blockIdx.x, s = seg / n_kv_heads, g = seg - s * n_kv_heads;
+  const int n_hist = tab.cu_at(s + 1) - tab.cu_at(s) - window;
+  if (n_hist <= 0) return;
+  const int R = G * window;
+  const int nc = (n_hist + chunk_keys - 1) / chunk_keys;
+  for (int r = threadIdx.x; r < R; r += kThreads) {
+    const float* pm = part_m + ((long long)seg * R + r) * n_chunks;
+    const float* pz = part_z + ((long long)seg * R + r) * n_chunks;
+    const bool has_win = lse.win_m != nullptr;
+    const float l2 = simt_row_lse(pm, pz, nc, has_win, has_win ? lse.win_m[(long long)seg * R + r] : 0.f,
+                                  has_win ? lse.win_z[(long long)seg * R + r] : 0.f);
+    const int hh = r / window, i = r - hh * window;
+    lse_out[((long long)s * lse.n_q_heads + g * G + hh) * window + i] = l2 * out_scale;
+  }
+}
+
+template <typename T, int D>
+cudaError_t launch_passes(const Problem& pb, int passes, cudaStream_t st, int* launches) {
   const size_t smem = simt_smem_bytes(pb);
   static thread_local int configured_dev = -1;
   int dev = 0;
@@ -180,19 +262,31 @@ cudaError_t launch_both(const Problem& pb, cudaStream_t st, int* launches) {
   dim3 grid((pb.max_hist + chunk_keys - 1) / chunk_keys, pb.p.n_kv_heads, pb.p.n_seqs);
   const float scale_log2 = kLog2e / sqrtf((float)pb.p.head_dim);
   const slkv_params& p = pb.p;
-  {
+  const LseSource lse = lse_source_of(pb);
+  if (passes & 1) {
     LaunchScope scope(KID_SCORE_LSE, st, launches);
     e = launch_pdl(k_score_simt<T, D, 1>, grid, dim3(kThreads), smem, st, 1, (const T*)pb.q, (const T*)pb.k, pb.tab,
-                   pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G, p.window, pb.n_chunks,
+                   pb.part_m, pb.part_z, pb.vote, lse, p.n_kv_heads, pb.G, p.window, pb.n_chunks,
                    (long long)p.k_stride_tok, (long long)p.k_stride_head, (long long)p.q_stride_seq,
                    (long long)p.q_stride_row, (long long)p.q_stride_head, scale_log2);
     if (e != cudaSuccess) return e;
   }
+  if (!(passes & 2)) return cudaSuccess;
   LaunchScope scope(KID_SCORE_VOTE, st, launches);
   return launch_pdl(k_score_simt<T, D, 2>, grid, dim3(kThreads), smem, st, 1, (const T*)pb.q, (const T*)pb.k, pb.tab,
-                    pb.part_m, pb.part_z, pb.vote, p.n_kv_heads, pb.G, p.window, pb.n_chunks,
+                    pb.part_m, pb.part_z, pb.vote, lse, p.n_kv_heads, pb.G, p.window, pb.n_chunks,
                     (long long)p.k_stride_tok, (long long)p.k_stride_head, (long long)p.q_stride_seq,
                     (long long)p.q_stride_row, (long long)p.q_stride_head, scale_log2);
+}
+
+template <typename T, int D>
+cudaError_t launch_window(const Problem& pb, bool head_inner, cudaStream_t st, int* launches) {
+  const slkv_params& p = pb.p;
+  LaunchScope scope(KID_WINDOW_STATS, st, launches);
+  return launch_pdl(k_window_stats<T, D>, dim3(pb.n_seg), dim3(kThreads), 0, st, 1, (const T*)pb.q, (const T*)pb.k,
+                    pb.tab, pb.win_m, pb.win_z, p.n_kv_heads, pb.G, p.window, head_inner ? 1 : 0,
+                    (long long)p.k_stride_tok, (long long)p.k_stride_head, (long long)p.q_stride_seq,
+                    (long long)p.q_stride_row, (long long)p.q_stride_head, kLog2e / sqrtf((float)p.head_dim));
 }
 
 }  // namespace
@@ -203,12 +297,42 @@ size_t simt_smem_bytes(const Problem& pb) {
   return (size_t)pb.R * pb.p.head_dim * pb.elem + (size_t)(2 * pb.R + 2 * kRowBatch * 4) * sizeof(float);
 }
 
-cudaError_t launch_score_simt(const Problem& pb, cudaStream_t st, int* launches) {
+cudaError_t launch_score_simt(const Problem& pb, int passes, cudaStream_t st, int* launches) {
   if (pb.max_hist <= 0) return cudaSuccess;
   const bool bf = pb.p.dtype == SLKV_BF16;
   if (pb.p.head_dim == 64)
-    return bf ? launch_both<__nv_bfloat16, 64>(pb, st, launches) : launch_both<float, 64>(pb, st, launches);
-  return bf ? launch_both<__nv_bfloat16, 128>(pb, st, launches) : launch_both<float, 128>(pb, st, launches);
+    return bf ? launch_passes<__nv_bfloat16, 64>(pb, passes, st, launches) : launch_passes<float, 64>(pb, passes, st, launches);
+  return bf ? launch_passes<__nv_bfloat16, 128>(pb, passes, st, launches) : launch_passes<float, 128>(pb, passes, st, launches);
+}
+
+cudaError_t launch_window_stats(const Problem& pb, bool head_inner, cudaStream_t st, int* launches) {
+  if (pb.max_hist <= 0) return cudaSuccess;
+  const bool bf = pb.p.dtype == SLKV_BF16;
+  if (pb.p.head_dim == 64)
+    return bf ? launch_window<__nv_bfloat16, 64>(pb, head_inner, st, launches) : launch_window<float, 64>(pb, head_inner, st, launches);
+  return bf ? launch_window<__nv_bfloat16, 128>(pb, head_inner, st, launches) : launch_window<float, 128>(pb, head_inner, st, launches);
+}
+
+// The row statistics a vote pass (or the merge) uses besides the partials of its own pass 1.
+LseSource lse_source_of(const Problem& pb) {
+  LseSource l;
+  l.lse_opt = pb.lse_opt;
+  const bool win = !pb.lse_opt && pb.p.softmax_domain == SLKV_ALL_CAUSAL;
+  l.win_m = win ? pb.win_m : nullptr;
+  l.win_z = win ? pb.win_z : nullptr;
+  l.to_log2 = pb.p.lse_units == SLKV_LSE_LOG2 ? 1.0f : kLog2e;
+  l.n_q_heads = pb.p.n_q_heads;
+  return l;
+}
+
+float lse_out_scale(const Problem& pb) { return pb.p.lse_units == SLKV_LSE_LOG2 ? 1.0f : 0.6931471805599453f; }
+
+cudaError_t launch_merge_lse_simt(const Problem& pb, float* lse_out, cudaStream_t st, int* launches) {
+  if (pb.max_hist <= 0) return cudaSuccess;
+  LaunchScope scope(KID_MERGE_LSE, st, launches);
+  return launch_pdl(k_merge_lse_simt, dim3(pb.n_seg), dim3(kThreads), 0, st, 1, (const float*)pb.part_m,
+                    (const float*)pb.part_z, lse_source_of(pb), pb.tab, lse_out, pb.p.n_kv_heads, pb.G, pb.p.window,
+                    pb.n_chunks, pb.chunk_keys, lse_out_scale(pb));
 }
 
 }  // namespace slkv

@@ -25,17 +25,20 @@ namespace {
 // Grid-wide barrier of the fused kernel (both passes in one launch): one arrival counter per launch, taken in
 // turn from a small table in the module's globals (zero at load).  atom.inc wraps the counter back to zero with
 // the last arrival, so a waiter -- which has arrived itself, hence has seen the counter above zero -- is done
-// when it reads zero, and the slot is clean for its next user 64 launches later.  The kernel is launched
-// cooperatively (all CTAs resident); the wait is bounded all the same.
+// when it reads zero.  Beside it sits an exit counter: the last CTA to leave the kernel puts both words back to zero,
+// so a launch whose wait ran out (some CTAs never arrived, the arrival counter did not wrap) still leaves the slot
+// clean for its next user 64 launches later.  The kernel is launched cooperatively (all CTAs resident); the wait is
+// bounded all the same.
 constexpr int kBarrierSlots = 64;
-__device__ unsigned g_grid_arrivals[kBarrierSlots];
+__device__ unsigned g_grid_arrivals[2 * kBarrierSlots];
 
-__device__ __forceinline__ bool grid_barrier(unsigned* counter, unsigned n_cta, volatile int* abort_flag) {
+__device__ __forceinline__ bool grid_barrier(unsigned* counter, unsigned n_arrivals, volatile int* abort_flag) {
   // Called by one thread after a CTA-wide barrier: the release on the arrival makes the CTA's earlier writes
-  // visible to whoever acquires the counter afterwards.
+  // visible to whoever acquires the counter afterwards.  n_arrivals = the grid size (a diagnostic launch asks for
+  // one more than will ever come, so that the wait runs out).
   unsigned prev;
-  asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(prev) : "l"(counter), "r"(n_cta - 1) : "memory");
-  if (prev == n_cta - 1) return true;
+  asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;" : "=r"(prev) : "l"(counter), "r"(n_arrivals - 1) : "memory");
+  if (prev == n_arrivals - 1) return true;
   const unsigned long long t0 = now_ns();
   for (unsigned it = 1;; ++it) {
     unsigned c;
@@ -83,6 +86,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   auto accf_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
   auto acce_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 4 + b); };
   const uint32_t qfull_bar = bar0 + 8u * (2 * kStages + 8), qempty_bar = qfull_bar + 8u;
+  auto drain_bar = [&](int issuer) { return bar0 + 8u * (2 * kStages + 10 + issuer); };    // used only when a wait ran out
   volatile int* abort_flag = &abort_sh;
 
   const int begin = blockIdx.x * a.tiles_per_cta;
@@ -98,6 +102,8 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     for (int b = 0; b < 4; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
     mbar_init(qfull_bar, 1);
     mbar_init(qempty_bar, 2);                                 // one arrival per MMA issuer
+    mbar_init(drain_bar(0), 1);
+    mbar_init(drain_bar(1), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // rows of the Q tile beyond R are never written by TMA: keep them zero
@@ -131,7 +137,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       if (zw == 12345.f) abort_sh = 0;                              // keeps the call alive; writes what is there
     }
   }
-  if (MODE != 2 || warp >= 4) pdl_wait();
+  if (MODE != 2 || warp >= 4 || a.fresh_inputs) pdl_wait();
   if (tid == 0) trace_mark(a.trace, 1);
 
   // pass 2 walks the CTA's tiles backwards: the last ones read are likeliest in L2
@@ -246,6 +252,12 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         ++run_idx;
       }
      }
+      if (!ok) {
+        // gave up: the MMAs this thread has issued must be through before the accumulators are released
+        tc_commit(drain_bar(me));
+        const unsigned long long t0 = now_ns();
+        while (!mbar_try(drain_bar(me), 0) && now_ns() - t0 < kWaitLimitNs) {}
+      }
     }
   } else if (warp >= 4) {
     // ---------------- epilogue: two warpgroups, alternating tiles ----------------
@@ -263,7 +275,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       // every CTA's row statistics must be in memory before any row's log-sum-exp is formed
       epi_bar();
       if (et == 0) trace_mark(a.trace, 5);
-      if (et == 0 && ok) grid_barrier(&g_grid_arrivals[a.barrier_slot], gridDim.x, abort_flag);
+      if (et == 0 && ok) grid_barrier(&g_grid_arrivals[2 * a.barrier_slot], gridDim.x + (unsigned)a.barrier_extra, abort_flag);
       if (et == 0) trace_mark(a.trace, 6);
       epi_bar();
       ok = ok && *abort_flag == 0;
@@ -277,43 +289,22 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       if (pass == 2) {
         // merge the per-CTA partials of this segment into the rows' log-sum-exp (log2 units)
         const int n_slots = (r.seg_tile0 + r.tiles_seg - 1) / a.tiles_per_cta - first_cta + 1;
-        // Every thread has all its loads in flight before it uses one.  With R <= 128 two neighbouring lanes
-        // share a row (even / odd slots) and combine through a shuffle.
+        // With R <= 128 two neighbouring lanes share a row (even / odd slots) and combine through a shuffle.
         {
           const int halves = 2 * R <= kEpiThreads ? 2 : 1;
           const int rr = halves == 2 ? ((et >> 1) < R ? (et >> 1) : -1) : (et < R ? et : -1);
           const int half = halves == 2 ? (et & 1) : 0;
-          float M = -INFINITY, Z = 0.f;
-          if (rr >= 0) {
-            const float* pm = a.part_m + (long long)seg * a.slot_stride * R + rr;      // [segment][slot][row]
-            const float* pz = a.part_z + (long long)seg * a.slot_stride * R + rr;
-            for (int c0 = half; c0 < n_slots; c0 += 12 * halves) {
-              float m12[12], z12[12];
-#pragma unroll
-              for (int u = 0; u < 12; ++u) {
-                const int c = c0 + u * halves;
-                const bool in = c < n_slots;
-                m12[u] = in ? __ldcg(pm + (long long)c * R) : -INFINITY;
-                z12[u] = in ? __ldcg(pz + (long long)c * R) : 0.f;
-              }
-#pragma unroll
-              for (int u = 0; u < 12; ++u)
-                if (z12[u] > 0.f) {                                    // empty partials carry z = 0
-                  const float Mn = fmaxf(M, m12[u]);
-                  Z = Z * ex2(M - Mn) + z12[u] * ex2(m12[u] - Mn);      // ex2(-inf) = 0 covers the first term
-                  M = Mn;
-                }
-            }
+          float l2;
+          if (a.lse.lse_opt) {                                            // the caller's row statistics
+            l2 = rr >= 0 ? a.lse.caller_lse(r.s, r.g, rr, a.G, a.window, a.q_head_inner != 0) : 0.f;
+          } else {
+            const bool has_win = a.lse.win_m != nullptr && rr >= 0;
+            l2 = merged_row_lse(a.part_m + (long long)seg * a.slot_stride * R, a.part_z + (long long)seg * a.slot_stride * R,
+                                n_slots, R, rr, half, halves, has_win,
+                                has_win ? a.lse.win_m[(long long)seg * R + rr] : 0.f,
+                                has_win ? a.lse.win_z[(long long)seg * R + rr] : 0.f);
           }
-          if (halves == 2) {                                              // uniform over the warp
-            const float M1 = __shfl_xor_sync(0xffffffffu, M, 1), Z1 = __shfl_xor_sync(0xffffffffu, Z, 1);
-            const float Mn = fmaxf(M, M1);
-            float Zt = 0.f;
-            if (M > -INFINITY) Zt += Z * ex2(M - Mn);
-            if (M1 > -INFINITY) Zt += Z1 * ex2(M1 - Mn);
-            M = Mn; Z = Zt;
-          }
-          if (half == 0 && rr >= 0) lse[rr] = M + log2f(Z);
+          if (half == 0 && rr >= 0) lse[rr] = l2;
         }
         epi_bar();
         if (et == 0 && pass == 2 && pos == first_pos(true)) trace_mark(a.trace, 7);
@@ -436,9 +427,48 @@ k_score_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   if (abort_sh && tid == 0 && a.status) atomicExch(a.status, (int)SLKV_ERR_DEVICE_TIMEOUT);
   if (tid == 0) trace_mark(a.trace, 4);
+  if (MODE == 3 && tid == 0) {
+    // every thread of this CTA is past the grid barrier (the CTA-wide barrier above): the last CTA out cleans the slot
+    unsigned* slot = &g_grid_arrivals[2 * a.barrier_slot];
+    unsigned prev;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(slot + 1) : "memory");
+    if (prev == gridDim.x - 1) {
+      slot[0] = 0;
+      slot[1] = 0;
+      __threadfence();
+    }
+  }
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// lse_out[s][h][i] from the per-CTA statistics pass 1 left (tensor layout), in the units out_scale converts to.
+__global__ void __launch_bounds__(kEpiThreads)
+k_merge_lse_tensor(const __grid_constant__ TcArgs a, float* __restrict__ lse_out, float out_scale) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int seg = blockIdx.x, s = seg / a.n_kv_heads, g = seg - s * a.n_kv_heads;
+  const int n_hist = a.tab.cu_at(s + 1) - a.tab.cu_at(s) - a.window;
+  if (n_hist <= 0) return;
+  const int R = a.R, et = threadIdx.x;
+  const int tiles_seg = a.tab.tile_at(s + 1) - a.tab.tile_at(s);
+  const int seg_tile0 = a.n_kv_heads * a.tab.tile_at(s) + g * tiles_seg;
+  const int first_cta = seg_tile0 / a.tiles_per_cta;
+  const int n_slots = (seg_tile0 + tiles_seg - 1) / a.tiles_per_cta - first_cta + 1;
+  const int halves = 2 * R <= kEpiThreads ? 2 : 1;
+  const int rr = halves == 2 ? ((et >> 1) < R ? (et >> 1) : -1) : (et < R ? et : -1);
+  const int half = halves == 2 ? (et & 1) : 0;
+  const bool has_win = a.lse.win_m != nullptr && rr >= 0;
+  const float l2 = merged_row_lse(a.part_m + (long long)seg * a.slot_stride * R, a.part_z + (long long)seg * a.slot_stride * R,
+                                  n_slots, R, rr, half, halves, has_win,
+                                  has_win ? a.lse.win_m[(long long)seg * R + rr] : 0.f,
+                                  has_win ? a.lse.win_z[(long long)seg * R + rr] : 0.f);
+  if (half == 0 && rr >= 0) {
+    const int hh = a.q_head_inner ? rr % a.G : rr / a.window;
+    const int i = a.q_head_inner ? rr / a.G : rr - hh * a.window;
+    lse_out[((long long)s * a.lse.n_q_heads + g * a.G + hh) * a.window + i] = l2 * out_scale;
   }
 }
 
@@ -471,6 +501,9 @@ int sm_count() {
 }
 
 struct Schedule { int total_tiles, tiles_per_cta, n_cta; };
+
+// One-shot diagnostic: the next launch of this thread whose CTAs wait for one another expects one arrival too many.
+thread_local int g_expire_next_wait = 0;
 
 // Timeline tracing (diagnostics): a caller-owned device buffer, two halves (pass 1, pass 2).
 thread_local unsigned long long* g_trace = nullptr;
@@ -525,6 +558,10 @@ bool tensor_path_supported(const slkv_params& p) {
   return encode_fn() != nullptr;
 }
 
+// Row order inside the Q tile: the query heads of a group next to each other (r = i*G + hh) when the head stride is
+// the smaller one, else the window rows (r = hh*window + i).
+bool tensor_q_head_inner(const slkv_params& p) { return p.q_stride_head <= p.q_stride_row; }
+
 int tensor_slot_stride(const Problem& pb) { return (pb.max_hist + kTileKeys - 1) / kTileKeys + 2; }
 
 cudaError_t plan_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, TcPlan* plan) {
@@ -541,7 +578,7 @@ cudaError_t plan_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t
 
   // Tensor-map dimensions go from the smallest stride to the largest.  The order of the G*w query rows
   // inside the Q tile follows from it (head-fastest or window-row-fastest); the scores do not depend on it.
-  const int q_head_inner = p.q_stride_head <= p.q_stride_row;
+  const int q_head_inner = tensor_q_head_inner(p) ? 1 : 0;
   const int k_head_inner = p.k_stride_head <= p.k_stride_tok;
   {
     cuuint64_t dims[4] = {(cuuint64_t)p.head_dim, (cuuint64_t)p.window, (cuuint64_t)p.n_q_heads, (cuuint64_t)p.n_seqs};
@@ -576,8 +613,11 @@ cudaError_t plan_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t
 
   a.tab = pb.tab;
   a.part_m = pb.part_m; a.part_z = pb.part_z; a.vote = pb.vote; a.status = status;
+  a.lse = lse_source_of(pb);
   a.trace = nullptr;
   a.barrier_slot = 0;
+  a.barrier_extra = 0;
+  a.fresh_inputs = 0;
   a.n_seqs = p.n_seqs; a.n_kv_heads = p.n_kv_heads; a.G = pb.G; a.window = p.window; a.R = pb.R;
   a.MT = (pb.R + 127) / 128;
   a.q_head_inner = q_head_inner; a.k_head_inner = k_head_inner;
@@ -594,8 +634,21 @@ cudaError_t plan_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t
 
 unsigned long long* tensor_trace_buffer(int half, int n_cta) { return trace_buffer(half + 1, n_cta); }
 
-cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, cudaStream_t st,
-                                int* launches) {
+void expire_next_wait(int on) { g_expire_next_wait = on; }
+int take_expire_next_wait() { const int v = g_expire_next_wait; g_expire_next_wait = 0; return v; }
+
+cudaError_t launch_merge_lse_tensor(const Problem& pb, const int32_t* cu_host, float* lse_out, cudaStream_t st,
+                                    int* launches) {
+  TcPlan plan;
+  cudaError_t pe = plan_score_tensor(pb, cu_host, nullptr, &plan);
+  if (pe != cudaSuccess || plan.n_cta == 0) return pe;
+  LaunchScope scope(KID_MERGE_LSE, st, launches);
+  return launch_pdl(k_merge_lse_tensor, dim3(pb.n_seg), dim3(kEpiThreads), 0, st, 1, plan.a, lse_out, lse_out_scale(pb));
+}
+
+
+cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32_t* status, int passes,
+                                cudaStream_t st, int* launches) {
   TcPlan plan;
   cudaError_t pe = plan_score_tensor(pb, cu_host, status, &plan);
   if (pe != cudaSuccess || plan.n_cta == 0) return pe;
@@ -628,7 +681,7 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
       fs = -1;
     else fs = 1;
   }
-  if (fs > 0 && sc.n_cta <= sm_count()) {
+  if (passes == 3 && fs > 0 && sc.n_cta <= sm_count()) {
     for (int attempt = 0; attempt < 2 && fs > 0; ++attempt) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3(sc.n_cta);
@@ -650,6 +703,8 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
       a.trace = trace_buffer(1, sc.n_cta);
       static std::atomic<unsigned> launch_seq{0};
       a.barrier_slot = (int)(launch_seq.fetch_add(1) % kBarrierSlots);
+      a.barrier_extra = g_expire_next_wait ? 1 : 0;
+      g_expire_next_wait = 0;
       cudaError_t le;
       {
         LaunchScope scope(KID_SCORE_FUSED, st, launches);
@@ -661,13 +716,15 @@ cudaError_t launch_score_tensor(const Problem& pb, const int32_t* cu_host, int32
       fs = fs == 1 ? 2 : -1;                          // try without dependent launch, then give up on fusing
     }
   }
-  {
+  if (passes & 1) {
     LaunchScope scope(KID_SCORE_LSE, st, launches);
     a.trace = trace_buffer(1, sc.n_cta);
     e = launch_pdl(k_score_tc<1>, dim3(sc.n_cta), dim3(kThreads), smem, st, 1, tm_q, tm_k, a);
     if (e != cudaSuccess) return e;
   }
+  if (!(passes & 2)) return cudaSuccess;
   LaunchScope scope(KID_SCORE_VOTE, st, launches);
+  a.fresh_inputs = (passes & 1) ? 0 : 1;              // a vote pass on its own is the first to read Q and K
   a.trace = trace_buffer(2, sc.n_cta);
   return launch_pdl(k_score_tc<2>, dim3(sc.n_cta), dim3(kThreads), smem, st, 1, tm_q, tm_k, a);
 }

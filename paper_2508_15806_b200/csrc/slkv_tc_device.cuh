@@ -172,6 +172,52 @@ __device__ __forceinline__ uint32_t instr_desc(int M, int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// Merges the per-CTA partial statistics [slot][row] of one row of a segment (pm / pz point at the segment's first
+// slot) into the row's log-sum-exp in log2 units, the window keys' statistics (wm, wz) folded in when has_win.  With
+// halves == 2 two neighbouring lanes share a row (even / odd slots) and combine through a shuffle, so all 32 lanes
+// of a warp must call it; lanes without a row pass rr < 0.  Every thread has all its loads in flight before it uses
+// one.  One definition for every kernel that merges, so that they agree bit for bit.
+__device__ __forceinline__ float merged_row_lse(const float* pm, const float* pz, int n_slots, int R, int rr, int half,
+                                                int halves, bool has_win, float wm, float wz) {
+  float M = -INFINITY, Z = 0.f;
+  if (rr >= 0) {
+    pm += rr;                                                              // [segment][slot][row]
+    pz += rr;
+    for (int c0 = half; c0 < n_slots; c0 += 12 * halves) {
+      float m12[12], z12[12];
+#pragma unroll
+      for (int u = 0; u < 12; ++u) {
+        const int c = c0 + u * halves;
+        const bool in = c < n_slots;
+        m12[u] = in ? __ldcg(pm + (long long)c * R) : -INFINITY;
+        z12[u] = in ? __ldcg(pz + (long long)c * R) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 12; ++u)
+        if (z12[u] > 0.f) {                                                // empty partials carry z = 0
+          const float Mn = fmaxf(M, m12[u]);
+          Z = fmaf(Z, ex2(M - Mn), __fmul_rn(z12[u], ex2(m12[u] - Mn)));   // ex2(-inf) = 0 covers the first term;
+                                                                           // explicit rounding: the same in every kernel
+          M = Mn;
+        }
+    }
+  }
+  if (halves == 2) {                                                       // uniform over the warp
+    const float M1 = __shfl_xor_sync(0xffffffffu, M, 1), Z1 = __shfl_xor_sync(0xffffffffu, Z, 1);
+    const float Mn = fmaxf(M, M1);
+    float Zt = 0.f;
+    if (M > -INFINITY) Zt = __fmul_rn(Z, ex2(M - Mn));
+    if (M1 > -INFINITY) Zt = __fadd_rn(Zt, __fmul_rn(Z1, ex2(M1 - Mn)));
+    M = Mn; Z = Zt;
+  }
+  if (has_win && wz > 0.f) {
+    const float Mn = fmaxf(M, wm);
+    Z = __fadd_rn(M > -INFINITY ? __fmul_rn(Z, ex2(M - Mn)) : 0.f, __fmul_rn(wz, ex2(wm - Mn)));
+    M = Mn;
+  }
+  return __fadd_rn(M, log2f(Z));
+}
+
 struct Run { int s, g, t0, count, n_hist, seg_tile0, tiles_seg; };
 
 // A run = consecutive tiles of one segment inside the CTA's range [begin, end).  Forward walks (pass 1)

@@ -32,13 +32,24 @@ def to_np_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().to(torch.float32).numpy()
 
 
+def lse_to_dev(lse, units: int = B.SLKV_LSE_LN) -> Optional[torch.Tensor]:
+    """Host row log-sum-exps (natural log, numpy fp64 with NaN where a sequence has no history) -> CUDA fp32 in `units`."""
+    if lse is None:
+        return None
+    a = np.nan_to_num(np.asarray(lse, dtype=np.float64), nan=0.0)
+    if units == B.SLKV_LSE_LOG2:
+        a = a / np.log(2.0)
+    return torch.tensor(a, dtype=torch.float32, device="cuda:0").contiguous()
+
+
 def gpu_compress(q_win, k, v, cu: Sequence[int], budgets_row: Sequence[int], window: int, pool_kernel: int,
                  pool_mode: int = B.SLKV_POOL_MAX, score_path: int = B.SLKV_PATH_AUTO,
-                 capacity: Optional[int] = None, want_pooled: bool = True) -> Dict[str, object]:
+                 capacity: Optional[int] = None, want_pooled: bool = True, domain: int = B.SLKV_HISTORY,
+                 lse=None, lse_units: int = B.SLKV_LSE_LN) -> Dict[str, object]:
     """Runs slkv_compress on cuda:0 with host tensors q_win, k, v; returns host results."""
     dev = torch.device("cuda:0")
     qd, kd, vd = q_win.to(dev), k.to(dev), v.to(dev)
-    params = B.make_params(qd, kd, vd, window, pool_kernel, pool_mode, score_path)
+    params = B.make_params(qd, kd, vd, window, pool_kernel, pool_mode, score_path, domain, lse_units)
     cu = [int(x) for x in cu]
     n_seg = (len(cu) - 1) * k.shape[1]
     cap = B.slkv_packed_rows_upper_bound(params, cu) if capacity is None else capacity
@@ -52,7 +63,8 @@ def gpu_compress(q_win, k, v, cu: Sequence[int], budgets_row: Sequence[int], win
     ws = B.new_workspace(params, cu, dev)
     n_pool = B.slkv_pooled_elems(params, cu)
     pooled = torch.full((max(n_pool, 1),), float("nan"), dtype=torch.float32, device=dev) if want_pooled else None
-    B.slkv_compress(params, qd, kd, vd, cu_dev, cu, bud, k_out, v_out, offsets, kept, ws, pooled, status)
+    B.slkv_compress(params, qd, kd, vd, cu_dev, cu, bud, k_out, v_out, offsets, kept, ws, pooled, status,
+                    lse=lse_to_dev(lse, lse_units))
     launches = B.slkv_last_launch_count()
     torch.cuda.synchronize()
     return {"offsets": offsets.cpu().numpy().astype(np.int64), "kept_idx": kept.cpu().numpy().astype(np.int64),
@@ -61,18 +73,39 @@ def gpu_compress(q_win, k, v, cu: Sequence[int], budgets_row: Sequence[int], win
 
 
 def gpu_score(q_win, k, cu: Sequence[int], window: int, pool_kernel: int, pool_mode: int = B.SLKV_POOL_MAX,
-              score_path: int = B.SLKV_PATH_AUTO) -> np.ndarray:
+              score_path: int = B.SLKV_PATH_AUTO, domain: int = B.SLKV_HISTORY, lse=None,
+              lse_units: int = B.SLKV_LSE_LN) -> np.ndarray:
     dev = torch.device("cuda:0")
     qd, kd = q_win.to(dev), k.to(dev)
-    params = B.make_params(qd, kd, None, window, pool_kernel, pool_mode, score_path)
+    params = B.make_params(qd, kd, None, window, pool_kernel, pool_mode, score_path, domain, lse_units)
     cu = [int(x) for x in cu]
     cu_dev = torch.tensor(cu, dtype=torch.int32, device=dev)
     ws = B.new_workspace(params, cu, dev)
     n_pool = B.slkv_pooled_elems(params, cu)
     pooled = torch.full((max(n_pool, 1),), float("nan"), dtype=torch.float32, device=dev)
-    B.slkv_score(params, qd, kd, cu_dev, cu, pooled, ws)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    lse_dev = lse if isinstance(lse, torch.Tensor) else lse_to_dev(lse, lse_units)
+    B.slkv_score(params, qd, kd, cu_dev, cu, pooled, ws, status, lse=lse_dev)
     torch.cuda.synchronize()
+    assert int(status.item()) == 0
     return pooled[:n_pool].cpu().numpy()
+
+
+def gpu_row_lse(q_win, k, cu: Sequence[int], window: int, score_path: int = B.SLKV_PATH_AUTO,
+                domain: int = B.SLKV_HISTORY, lse_units: int = B.SLKV_LSE_LN) -> torch.Tensor:
+    """slkv_row_lse on cuda:0: CUDA float32 [n_seqs, n_q_heads, window] (rows of sequences without history: NaN)."""
+    dev = torch.device("cuda:0")
+    qd, kd = q_win.to(dev), k.to(dev)
+    params = B.make_params(qd, kd, None, window, 1, B.SLKV_POOL_MAX, score_path, domain, lse_units)
+    cu = [int(x) for x in cu]
+    cu_dev = torch.tensor(cu, dtype=torch.int32, device=dev)
+    ws = B.new_workspace(params, cu, dev)
+    out = torch.full((q_win.shape[0], q_win.shape[2], window), float("nan"), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    B.slkv_row_lse(params, qd, kd, cu_dev, cu, out, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    return out
 
 
 def split_pooled(flat: np.ndarray, cu: Sequence[int], n_kv_heads: int, window: int) -> List[np.ndarray]:
@@ -147,17 +180,20 @@ def assert_selection_valid(gpu: Dict[str, object], oracle_pooled: List[np.ndarra
     return stats
 
 
-def oracle_pooled(q_win, k, cu, window, pool_kernel, pool_mode=B.SLKV_POOL_MAX) -> List[np.ndarray]:
-    votes = O.window_votes(to_np64(q_win), to_np64(k), cu, window)
+def oracle_pooled(q_win, k, cu, window, pool_kernel, pool_mode=B.SLKV_POOL_MAX, domain: int = B.SLKV_HISTORY,
+                  lse=None) -> List[np.ndarray]:
+    votes = O.window_votes(to_np64(q_win), to_np64(k), cu, window,
+                           "all_causal" if domain == B.SLKV_ALL_CAUSAL else "history", lse)
     return [O.pool(vt, pool_kernel, "max" if pool_mode == B.SLKV_POOL_MAX else "avg") for vt in votes]
 
 
 def check_compress(q_win, k, v, cu, budgets_row, window, pool_kernel, pool_mode=B.SLKV_POOL_MAX,
-                   score_path=B.SLKV_PATH_AUTO, pooled_ref=None):
-    """Full parity of one layer: returns (gpu result, stats)."""
-    gpu = gpu_compress(q_win, k, v, cu, budgets_row, window, pool_kernel, pool_mode, score_path)
+                   score_path=B.SLKV_PATH_AUTO, pooled_ref=None, domain: int = B.SLKV_HISTORY, lse=None):
+    """Full parity of one layer: returns (gpu result, stats).  `lse` (natural log, host fp64) goes to both sides."""
+    gpu = gpu_compress(q_win, k, v, cu, budgets_row, window, pool_kernel, pool_mode, score_path, domain=domain, lse=lse)
     assert gpu["status"] == 0
-    ref = pooled_ref if pooled_ref is not None else oracle_pooled(q_win, k, cu, window, pool_kernel, pool_mode)
+    ref = pooled_ref if pooled_ref is not None else oracle_pooled(q_win, k, cu, window, pool_kernel, pool_mode, domain,
+                                                                 lse)
     worst = assert_pooled_close(gpu["pooled"], ref, cu, k.shape[1], window)
     stats = assert_selection_valid(gpu, ref, cu, budgets_row, window, k, v)
     stats["pooled_max_rel_err"] = worst

@@ -35,6 +35,7 @@ def test_exports_every_declared_symbol(L):
 def params(**kw):
     d = dict(n_seqs=1, n_q_heads=8, n_kv_heads=2, head_dim=128, window=16, pool_kernel=5, dtype=B.SLKV_BF16,
              pool_mode=B.SLKV_POOL_MAX, softmax_domain=B.SLKV_HISTORY, score_path=B.SLKV_PATH_AUTO,
+             lse_units=B.SLKV_LSE_LN, reserved=0,
              k_stride_tok=256, k_stride_head=128, v_stride_tok=256, v_stride_head=128,
              q_stride_seq=16 * 8 * 128, q_stride_row=8 * 128, q_stride_head=128)
     d.update(kw)
@@ -62,18 +63,19 @@ def test_bad_enums_and_alignment(L):
     cu = (C.c_int32 * 2)(0, 100)
     fake = C.c_void_p(4096)          # never dereferenced: validation fails first
     for kw, code in [(dict(dtype=7), "BAD_DTYPE"), (dict(pool_mode=3), "BAD_DTYPE"),
-                     (dict(softmax_domain=1), "BAD_DTYPE"), (dict(score_path=9), "BAD_DTYPE"),
+                     (dict(softmax_domain=2), "BAD_DTYPE"), (dict(score_path=9), "BAD_DTYPE"),
+                     (dict(lse_units=2), "BAD_DTYPE"), (dict(reserved=1), "BAD_DTYPE"),
                      (dict(k_stride_tok=257), "BAD_ALIGN")]:
         p = params(**kw)
-        rc = L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, None, fake, 1 << 30, None)
+        rc = L.slkv_score(C.byref(p), fake, fake, fake, cu, None, fake, None, fake, 1 << 30, None)
         assert rc == B.ERR[code], (kw, rc)
     p = params()
-    assert L.slkv_score(C.byref(p), None, fake, fake, cu, fake, None, fake, 1 << 30, None) == B.ERR["NULL_PTR"]
-    assert L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, None, None, 0, None) == B.ERR["WORKSPACE"]
-    assert L.slkv_score(C.byref(p), fake, fake, fake, cu, fake, None, fake, 16, None) == B.ERR["WORKSPACE"]
-    assert L.slkv_score(C.byref(p), C.c_void_p(4100), fake, fake, cu, fake, None, fake, 1 << 30, None) == B.ERR["BAD_ALIGN"]
+    assert L.slkv_score(C.byref(p), None, fake, fake, cu, None, fake, None, fake, 1 << 30, None) == B.ERR["NULL_PTR"]
+    assert L.slkv_score(C.byref(p), fake, fake, fake, cu, None, fake, None, None, 0, None) == B.ERR["WORKSPACE"]
+    assert L.slkv_score(C.byref(p), fake, fake, fake, cu, None, fake, None, fake, 16, None) == B.ERR["WORKSPACE"]
+    assert L.slkv_score(C.byref(p), C.c_void_p(4100), fake, fake, cu, None, fake, None, fake, 1 << 30, None) == B.ERR["BAD_ALIGN"]
     bad_cu = (C.c_int32 * 2)(0, -5)
-    assert L.slkv_score(C.byref(p), fake, fake, fake, bad_cu, fake, None, fake, 1 << 30, None) == B.ERR["BAD_SHAPE"]
+    assert L.slkv_score(C.byref(p), fake, fake, fake, bad_cu, None, fake, None, fake, 1 << 30, None) == B.ERR["BAD_SHAPE"]
 
 
 def test_alloc_argument_errors(L):
@@ -90,10 +92,11 @@ def test_compress_argument_errors(L):
     fake = C.c_void_p(4096)
     cu = (C.c_int32 * 2)(0, 100)
     p = params()
-    args = [C.byref(p), fake, fake, fake, fake, cu, fake, fake, fake, 10, fake, fake, None, None, fake, 1 << 30, None]
+    args = [C.byref(p), fake, fake, fake, fake, cu, fake, None, fake, fake, 10, fake, fake, None, None, fake, 1 << 30,
+            None]
     bad = list(args); bad[6] = None
     assert L.slkv_compress(*bad) == B.ERR["NULL_PTR"]
-    bad = list(args); bad[9] = -1
+    bad = list(args); bad[10] = -1
     assert L.slkv_compress(*bad) == B.ERR["CAPACITY"]
     pt = params(score_path=B.SLKV_PATH_TENSOR, dtype=B.SLKV_F32, k_stride_tok=256, head_dim=64, k_stride_head=64,
                 v_stride_head=64, q_stride_head=64)

@@ -117,6 +117,59 @@ def test_all_causal_matches_masked_full_attention():
     assert np.allclose(got, ref, rtol=1e-12)
 
 
+def brute_lse(q_row, keys, d):
+    """log of Eq. 4's denominator for one query row, pure Python."""
+    tot = 0.0
+    for kj in keys:
+        tot += math.exp(sum(a * b for a, b in zip(q_row, kj)) / math.sqrt(d))
+    return math.log(tot)
+
+
+@pytest.mark.parametrize("domain", ["history", "all_causal"])
+def test_row_lse_matches_brute_force(domain):
+    rng = np.random.default_rng(41)
+    w, Hq, Hkv, d = 3, 4, 2, 6
+    q = rng.normal(size=(2, w, Hq, d))
+    k = rng.normal(size=(11 + 2, Hkv, d))          # second sequence is shorter than the window: no rows
+    got = O.row_lse(q, k, [0, 11, 13], w, domain)
+    assert got.shape == (2, Hq, w) and np.all(np.isnan(got[1]))
+    for h in range(Hq):
+        for i in range(w):
+            n_keys = 8 if domain == "history" else 8 + i + 1
+            ref = brute_lse(q[0, i, h].tolist(), k[:n_keys, h // 2].tolist(), d)
+            assert abs(got[0, h, i] - ref) < 1e-12
+
+
+def test_row_lse_of_equal_keys_is_logit_plus_log_count():
+    rng = np.random.default_rng(42)
+    d = 8
+    q = rng.normal(size=(1, 4, 2, d))
+    k = np.tile(rng.normal(size=(1, 1, d)), (36, 1, 1))
+    got = O.row_lse(q, k, [0, 36], 4)
+    ref = (q[0] @ k[0, 0]) / math.sqrt(d) + math.log(32)         # [w, Hq]
+    assert np.allclose(got[0], ref.T, rtol=0, atol=1e-12)
+    got_c = O.row_lse(q, k, [0, 36], 4, "all_causal")
+    ref_c = (q[0] @ k[0, 0]) / math.sqrt(d) + np.log(32 + 1 + np.arange(4))[:, None]
+    assert np.allclose(got_c[0], ref_c.T, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("domain", ["history", "all_causal"])
+def test_votes_from_supplied_lse(domain):
+    rng = np.random.default_rng(43)
+    q = rng.normal(size=(2, 4, 4, 8))
+    k = rng.normal(size=(30 + 21, 2, 8))
+    cu = [0, 30, 51]
+    lse = O.row_lse(q, k, cu, 4, domain)
+    a = O.window_votes(q, k, cu, 4, domain)
+    b = O.window_votes(q, k, cu, 4, "history", lse=lse)          # the domain only matters for the normaliser
+    for x, y in zip(a, b):
+        assert np.allclose(x, y, rtol=1e-12, atol=0)
+    # a normaliser one unit larger scales every vote of that row by 1/e: the array is used as given
+    lse2 = lse.copy(); lse2[0, :, :] += 1.0
+    c = O.window_votes(q, k, cu, 4, "history", lse=lse2)
+    assert np.allclose(c[0], a[0] / math.e, rtol=1e-12) and np.allclose(c[1], a[1], rtol=1e-12)
+
+
 def test_short_sequences_have_no_history():
     q = np.zeros((2, 4, 1, 2)); k = np.zeros((6, 1, 2))
     v = O.window_votes(q, k, [0, 4, 6], 4)

@@ -14,7 +14,7 @@ import torch
 from paper_2508_15806_b200 import binding as B
 from paper_2508_15806_b200 import build as builder
 
-REL_TOL = 1e-3          # the tolerance of the other parity tests (the two entry points run the same kernels)
+import parity as P      # the parity rules of the other GPU tests: pooled scores within 1e-3 of the oracle
 
 
 def _case(seed, lens, Hq=8, Hkv=2, w=32, dtype=torch.bfloat16, d=128):
@@ -49,14 +49,18 @@ def test_matches_slkv_score_on_two_calls_in_a_row():
         q, k, cu = _case(seed, lens, w=w)
         got, ref = _both(q, k, cu, w, p)
         assert np.all(np.isfinite(got))
-        assert np.all(np.abs(got - ref) <= REL_TOL * np.abs(ref))
+        # the same kernels on the same inputs: the two entry points agree bit for bit ...
+        assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+        # ... and with the oracle within the tolerance of every other parity test
+        P.assert_pooled_close(got, P.oracle_pooled(q, k, cu, w, p), cu, k.shape[1], w)
 
 
 @pytest.mark.gpu
 def test_fp32_path_too():
     q, k, cu = _case(3, [900], Hq=4, Hkv=4, w=16, dtype=torch.float32, d=64)
     got, ref = _both(q, k, cu, 16, 5)
-    assert np.all(np.abs(got - ref) <= REL_TOL * np.abs(ref))
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+    P.assert_pooled_close(got, P.oracle_pooled(q, k, cu, 16, 5), cu, k.shape[1], 16)
 
 
 def test_oversized_shapes_are_rejected_on_the_host():
@@ -66,11 +70,13 @@ def test_oversized_shapes_are_rejected_on_the_host():
     assert B.slkv_noalloc_scratch_bytes() == 8 << 20
     p = B.SlkvParams(n_seqs=1, n_q_heads=32, n_kv_heads=8, head_dim=128, window=32, pool_kernel=7, dtype=B.SLKV_BF16,
                      pool_mode=B.SLKV_POOL_MAX, softmax_domain=B.SLKV_HISTORY, score_path=B.SLKV_PATH_AUTO,
-                     k_stride_tok=1024, k_stride_head=128, v_stride_tok=1024, v_stride_head=128,
+                     lse_units=B.SLKV_LSE_LN, reserved=0, k_stride_tok=1024, k_stride_head=128, v_stride_tok=1024, v_stride_head=128,
                      q_stride_seq=32 * 32 * 128, q_stride_row=32 * 128, q_stride_head=128)
     cu = (C.c_int32 * 2)(0, 131072)
     assert B.slkv_workspace_bytes(p, [0, 131072]) > B.slkv_noalloc_scratch_bytes()
     fake = C.c_void_p(4096)
-    assert L.slkv_score_noalloc(C.byref(p), fake, fake, fake, cu, fake, None, None) == B.ERR["WORKSPACE"]
-    p.head_dim = 96                                        # argument errors keep their own codes
-    assert L.slkv_score_noalloc(C.byref(p), fake, fake, fake, cu, fake, None, None) == B.ERR["BAD_SHAPE"]
+    assert L.slkv_score_noalloc(C.byref(p), fake, fake, fake, cu, None, fake, None, None) == B.ERR["WORKSPACE"]
+    # argument errors keep the codes slkv_score gives them, and come first
+    assert L.slkv_score_noalloc(C.byref(p), None, fake, fake, cu, None, fake, None, None) == B.ERR["NULL_PTR"]
+    p.head_dim = 96
+    assert L.slkv_score_noalloc(C.byref(p), fake, fake, fake, cu, None, fake, None, None) == B.ERR["BAD_SHAPE"]
