@@ -176,6 +176,10 @@ def run_cuda(args):
     params = None
     for l in range(nl):
         x = synth.layer_inputs(wl, l, device=dev)
+        if args.kv_head_major:
+            # the same values, stored [n_kv_heads, tokens, head_dim]: the library takes the layout through the strides
+            x.k = x.k.permute(1, 0, 2).contiguous().permute(1, 0, 2)
+            x.v = x.v.permute(1, 0, 2).contiguous().permute(1, 0, 2)
         if params is None:
             params = B.make_params(x.q_win, x.k, x.v, w, wl.pool_kernel)
         rows = rows_of_layer(wl.seq_lens, budgets_host[l].tolist(), w)
@@ -188,6 +192,13 @@ def run_cuda(args):
     ws = torch.empty(B.slkv_workspace_bytes_overlapped(params, cu), dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
+    # the rows' log-sum-exps, as a prefill attention kernel that keeps its softmax statistics would hand them over
+    # (computed once, outside every timed region; used by the "with_lse" figures only)
+    for L in layers:
+        L["lse"] = torch.zeros(len(wl.seq_lens), wl.n_q_heads, w, dtype=torch.float32, device=dev)
+        B.slkv_row_lse(params, L["q"], L["k"], cu_dev, cu, L["lse"], ws, status)
+    torch.cuda.synchronize()
+    use_lse = [bool(args.with_lse)]
 
     launches_per_step = 0
 
@@ -199,7 +210,7 @@ def run_cuda(args):
         call = B.slkv_compress_overlapped if overlap else B.slkv_compress
         for L in layers:
             call(params, L["q"], L["k"], L["v"], cu_dev, cu, L["bud"], L["k_out"], L["v_out"],
-                 L["offsets"], L["kept"], ws, None, status, stream)
+                 L["offsets"], L["kept"], ws, None, status, stream, L["lse"] if use_lse[0] else None)
             n += B.slkv_last_launch_count()
         B.slkv_join(stream)
         launches_per_step = n + B.slkv_last_launch_count()
@@ -481,6 +492,10 @@ def main():
     ap.add_argument("--no-graph", action="store_true",
                     help="issue the calls of every step (default: capture a step's calls in a CUDA graph once and replay it)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--kv-head-major", action="store_true",
+                    help="store K and V head-major ([n_kv_heads, tokens, head_dim]) instead of token-major; not the headline")
+    ap.add_argument("--with-lse", action="store_true",
+                    help="hand every layer's row log-sum-exps to the calls (vote pass only); not the headline")
     ap.add_argument("--no-overlap", action="store_true", help="one layer at a time (slkv_compress) instead of overlapped calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)

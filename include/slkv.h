@@ -2,6 +2,7 @@
  * slkv.h -- C ABI of the SurfaceLogicKV prefill KV-cache compression library (CUDA, sm_100a).
  *
  * One call per step of the paper's method:
+ *   slkv_behavior_scores Stage 1, SF_sc / LG_sc / INF_sc of attention rows               (Sec. 3.2, Algorithm 1)
  *   slkv_alloc_budgets   Stage 2, per-head KV budgets from the INF_sc table     (Sec. 3.3, Eq. 6, Algorithm 2)
  *   slkv_score           relevance of every history key to the query window     (Sec. 3.4, Eq. 7, Alg. 3 l.4-6)
  *   slkv_compress        score -> top-(C - window) history rows + window, gather (Sec. 3.4, Eq. 8, Algorithm 3)
@@ -98,6 +99,25 @@ const char* slkv_strerror(int status);
 int slkv_last_cuda_error(void);
 
 /*
+ * Stage-1 attention behaviour analysis (Sec. 3.2, Algorithm 1), for a batch of attention rows (one row = the
+ * attention weights of one head for one probe prompt's answering position, over the context).
+ * For each row with needle positions N and top-k positions T (both as sets):
+ *     WO = sum of W over N and T,  WD = sum over T without N,  TNW = sum over N,  WS = max(0, TNW - WO)
+ *     SF_sc = WO / (WO + WD),  LG_sc = WO / (WO + WS),  INF_sc = 2 SF_sc LG_sc / (SF_sc + LG_sc)     (0/0 = 0)
+ *   attn         dev, float: row r starts at attn + r*row_stride and has row_len weights (row_stride 0 shares one row)
+ *   needle_idx   dev, int32: row r's needle positions at needle_idx + r*needle_stride, n_needle entries
+ *                (needle_stride 0: one list for all rows); entries outside [0, row_len) are padding
+ *   topk_idx     dev, int32: likewise the positions of the row's k largest weights (n_topk entries, topk_stride)
+ *   sf_sc, lg_sc, inf_sc   dev, out, float[n_rows]
+ * An index listed twice counts once.  Averaging the per-row scores into the per-(layer, head) INF_sc table that
+ * slkv_alloc_budgets takes is left to the caller (the paper does not print how it aggregates over prompts).
+ * Limits: n_needle, n_topk <= 4096.
+ */
+int slkv_behavior_scores(const float* attn, int64_t n_rows, int32_t row_len, int64_t row_stride,
+                         const int32_t* needle_idx, int32_t n_needle, int64_t needle_stride, const int32_t* topk_idx,
+                         int32_t n_topk, int64_t topk_stride, float* sf_sc, float* lg_sc, float* inf_sc, void* stream);
+
+/*
  * Stage-2 budget allocation (Sec. 3.3, Eq. 6; Algorithm 2).
  *   inf_sc   dev, float[n_layers*n_heads], row-major (layer, head); INF_sc >= 0, finite
  *   fixed    fixed part every head receives (= b_c (1 - 1/beta) in the paper's notation)
@@ -112,6 +132,33 @@ int slkv_last_cuda_error(void);
  */
 int slkv_alloc_budgets(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
                        int32_t* budgets, int32_t* status, void* stream);
+
+/*
+ * The same allocation with the readings Sec. 3.3 leaves open (Eq. 6 and its prose; Algorithm 2's last line).
+ *   head_normaliser  SLKV_NORM_GLOBAL: a head's share S_ij = inf_ij / L_s of the grand sum, as Algorithm 2 prints it;
+ *                    SLKV_NORM_WITHIN_LAYER: inf_ij / L_i of its own layer's sum, as the prose under Eq. 6 describes
+ *                    it (an all-zero layer shares evenly).  Under the second one a layer's total follows
+ *                    (0.01 + L_i/L_s) / (1 + 0.01 n_layers): the 0.01 "minimum layer budget" really is a floor.
+ *   rounding         SLKV_ROUND_SUM_EXACT: normalised weights, largest remainder, sum == total (as slkv_alloc_budgets);
+ *                    SLKV_ROUND_PAPER: Algorithm 2's own C = floor(max(0, fixed + D * weight) + 0.5) per head with
+ *                    D = total - N*fixed; the weights are not normalised, so the sum is whatever it comes to.
+ *   cap              0: none.  > 0: no head gets more than `cap` (say, the sequence length: budget beyond it could
+ *                    never be used).  With SLKV_ROUND_SUM_EXACT what a full head cannot take goes to the others in
+ *                    proportion to their weights, again and again until nobody is above the cap, and the budgets
+ *                    still sum to `total` (needs cap >= fixed and total <= N * cap, else SLKV_ERR_BUDGET_SUM); with
+ *                    SLKV_ROUND_PAPER the budgets are just clipped.  The paper has no cap.
+ * opt == NULL means {SLKV_NORM_GLOBAL, SLKV_ROUND_SUM_EXACT, 0}.  Other arguments, limits and errors as
+ * slkv_alloc_budgets; an unknown enum value gives SLKV_ERR_BAD_DTYPE.  Bit-reproducible like slkv_alloc_budgets.
+ */
+enum { SLKV_NORM_GLOBAL = 0, SLKV_NORM_WITHIN_LAYER = 1 };     /* slkv_alloc_options.head_normaliser */
+enum { SLKV_ROUND_SUM_EXACT = 0, SLKV_ROUND_PAPER = 1 };       /* slkv_alloc_options.rounding */
+typedef struct slkv_alloc_options {
+  int32_t head_normaliser;
+  int32_t rounding;
+  int64_t cap;
+} slkv_alloc_options;
+int slkv_alloc_budgets_ex(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
+                          const slkv_alloc_options* opt, int32_t* budgets, int32_t* status, void* stream);
 
 /* Bytes of workspace slkv_score / slkv_compress need for these shapes (0 on invalid arguments).
  * cu_seqlens_host: host, int32[n_seqs+1]. */

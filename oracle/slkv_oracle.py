@@ -6,10 +6,13 @@ A numpy matmul / stable sort serves as a step where the definition is a matrix p
 there is no blocking, fusion or reordering beyond what the definitions state.
 
 What follows which passage of the paper:
-  alloc_paper_literal   Algorithm 2 (and Eq. 6) exactly as printed, with its line-8 rounding.
-  alloc_budgets         Algorithm 2's weights (0.01 + L_i) * S_ij, normalised so the dynamic parts sum to
-                        the dynamic pool exactly (largest-remainder rounding) -- the paper concedes that its
-                        own formula "does not strictly conform to mathematical normalization" (Sec. 3.3).
+  head_weights          Algorithm 2's weight (0.01 + L_i) * S_ij of every head; S_ij over the grand sum (the
+                        algorithm) or over the layer's sum (the prose under Eq. 6).
+  alloc_paper_literal   Eq. 6 / Algorithm 2 in the paper's parameters (b_c, beta), with its own rounding.
+  alloc_budgets         the same weights, normalised so that the dynamic parts sum to the dynamic pool exactly
+                        (largest-remainder rounding): Sec. 3.3 itself says that the printed formula is not a
+                        normalisation.  Options: the prose's head normaliser, a per-head cap with the excess
+                        handed on (the paper has no cap), Algorithm 2's own rounding.
   row_lse               Eq. 3-4's row normaliser over Eq. 7's key set (the log of the softmax denominator).
   window_votes          Eq. 7 / Algorithm 3 line 6: softmax over the history keys of Q_window H^T / sqrt(d_k)
                         (Eq. 3-4 fix the scale and the softmax axis), then -- the paper does not say how the
@@ -51,42 +54,15 @@ def paper_fixed_and_pool(b_c: float, beta: float, n_layers: int, n_heads: int) -
     return b_c * (1.0 - 1.0 / beta), (b_c / beta) * n_layers * n_heads
 
 
-def alloc_paper_literal(b_c: float, beta: float, inf: np.ndarray, rounded: bool = True) -> np.ndarray:
-    """Algorithm 2 as printed.  inf[i][j] = INF_sc of head j in layer i.  Returns C[i][j]."""
-    inf = np.asarray(inf, dtype=np.float64)
-    L, H = inf.shape
-    b_fixed, B_total = paper_fixed_and_pool(b_c, beta, L, H)
-    L_alpha = [sum(float(inf[i][j]) for j in range(H)) for i in range(L)]        # line 3
-    L_s = sum(L_alpha)                                                           # line 4
-    out = np.zeros((L, H), dtype=np.float64)
-    for i in range(L):
-        L_ih = L_alpha[i] / L_s                                                  # line 5
-        for j in range(H):
-            S_jh = float(inf[i][j]) / L_s                                        # line 5
-            b_dyn = B_total * (LAYER_FLOOR + L_ih) * S_jh                        # line 6
-            b = b_fixed + b_dyn                                                  # line 7
-            out[i][j] = math.floor(max(0.0, b) + 0.5) if rounded else b          # line 8
-    return out.astype(np.int64) if rounded else out
-
-
-def alloc_budgets(inf: np.ndarray, fixed: int, total: int) -> np.ndarray:
-    """Integer budgets C[i][j] >= fixed with sum exactly `total` (Algorithm 2's weights, normalised).
-
-    Every floating-point operation is a separately rounded fp64 operation in the order written, sums run
-    in index order: the CUDA kernel must reproduce the result bit for bit.
-    """
-    inf32 = np.asarray(inf, dtype=np.float32)
-    if inf32.ndim != 2:
-        raise OracleError("BAD_SHAPE", "inf must be [n_layers, n_heads]")
-    L, H = inf32.shape
+def head_weights(inf: np.ndarray, within_layer: bool = False) -> List[float]:
+    """Algorithm 2's dynamic-budget weight of every head, flat in (layer, head) order:
+    (0.01 + L_i / L_s) * S_ij, with L_i the layer's INF_sc sum, L_s the grand sum and S_ij the head's share --
+    of the grand sum as the algorithm prints it (S_ij = inf_ij / L_s), or of its own layer's sum as the prose
+    under Eq. 6 describes it (within_layer: S_ij = inf_ij / L_i; an all-zero layer shares evenly).  All-zero INF_sc
+    gives every head the weight 1.  Separately rounded fp64 operations, sums in index order."""
+    x = np.asarray(inf, dtype=np.float32).astype(np.float64)
+    L, H = x.shape
     N = L * H
-    D = int(total) - N * int(fixed)
-    if fixed < 0 or D < 0:
-        raise OracleError("BUDGET_SUM", "total < n_heads_total * fixed")
-    x = inf32.astype(np.float64)
-    if not np.all(np.isfinite(x)) or np.any(x < 0):
-        raise OracleError("NEG_INF_SC", "INF_sc must be finite and >= 0")
-
     La = [0.0] * L
     for i in range(L):
         acc = 0.0
@@ -96,44 +72,126 @@ def alloc_budgets(inf: np.ndarray, fixed: int, total: int) -> np.ndarray:
     Ls = 0.0
     for i in range(L):
         Ls = Ls + La[i]
+    if not (Ls > 0.0):
+        return [1.0] * N
+    wgt = [0.0] * N
+    for i in range(L):
+        lw = LAYER_FLOOR + La[i] / Ls                            # 0.01 + L_{i,h}
+        for j in range(H):
+            if within_layer:
+                share = float(x[i][j]) / La[i] if La[i] > 0.0 else 1.0 / H
+            else:
+                share = float(x[i][j]) / Ls                      # S_{j,h}
+            wgt[i * H + j] = lw * share
+    return wgt
 
-    wgt = [1.0] * N
-    if Ls > 0.0:
-        for i in range(L):
-            lw = LAYER_FLOOR + La[i] / Ls                    # 0.01 + L_{i,h}
-            for j in range(H):
-                wgt[i * H + j] = lw * (float(x[i][j]) / Ls)  # * S_{j,h}
-    W = 0.0
-    for a in range(N):
-        W = W + wgt[a]
-    if not (W > 0.0):                                        # everything underflowed: uniform
-        wgt = [1.0] * N
-        W = float(N)
 
-    f = [0] * N
-    r = [0.0] * N
-    for a in range(N):
-        q = (float(D) * wgt[a]) / W
+def alloc_paper_literal(b_c: float, beta: float, inf: np.ndarray, rounded: bool = True) -> np.ndarray:
+    """Eq. 6 / Algorithm 2 in the paper's own parameters: C_ij = round-half-up(max(0, b_fixed + B_total * w_ij))
+    with b_fixed = b_c (1 - 1/beta), B_total = (b_c / beta) L H and w_ij = head_weights.  The dynamic parts are
+    not normalised: they sum to B_total (0.01 + sum_i L_i^2), not to B_total."""
+    x = np.asarray(inf, dtype=np.float64)
+    L, H = x.shape
+    b_fixed, B_total = paper_fixed_and_pool(b_c, beta, L, H)
+    b = b_fixed + B_total * np.array(head_weights(x), dtype=np.float64).reshape(L, H)
+    if not rounded:
+        return b
+    return np.floor(np.maximum(0.0, b) + 0.5).astype(np.int64)
+
+
+def alloc_budgets(inf: np.ndarray, fixed: int, total: int, within_layer: bool = False, cap: int = None,
+                  paper_rounding: bool = False) -> np.ndarray:
+    """Integer budgets C[i][j] from the INF_sc table (Sec. 3.3, Eq. 6, Algorithm 2), D = total - N * fixed the
+    dynamic pool.
+
+    Default: C >= fixed with sum exactly `total`: Algorithm 2's weights, normalised by their sum and rounded by
+    largest remainder (ties: lower index).
+    within_layer    the head normaliser of the prose under Eq. 6 instead of the algorithm's (see head_weights).
+    cap             no head gets more than `cap` (say, the sequence length: rows beyond it could never be kept);
+                    what a capped head cannot take goes to the others in proportion to their weights, again and
+                    again until nobody is above the cap (water filling).  total <= N * cap, cap >= fixed.
+    paper_rounding  Algorithm 2's own last line instead of the normalisation: C = floor(max(0, fixed + D * w) + 0.5)
+                    per head, clipped at `cap` if given; the sum is whatever it comes to.
+
+    Every floating-point operation is a separately rounded fp64 operation in the order written, sums run in index
+    order: the CUDA kernel must reproduce the result bit for bit.
+    """
+    inf32 = np.asarray(inf, dtype=np.float32)
+    if inf32.ndim != 2:
+        raise OracleError("BAD_SHAPE", "inf must be [n_layers, n_heads]")
+    L, H = inf32.shape
+    N = L * H
+    D = int(total) - N * int(fixed)
+    if fixed < 0 or D < 0:
+        raise OracleError("BUDGET_SUM", "total < n_heads_total * fixed")
+    if cap is not None and (cap < fixed or (not paper_rounding and int(total) > N * int(cap))):
+        raise OracleError("BUDGET_SUM", "cap below the fixed part, or total above n_heads_total * cap")
+    x = inf32.astype(np.float64)
+    if not np.all(np.isfinite(x)) or np.any(x < 0):
+        raise OracleError("NEG_INF_SC", "INF_sc must be finite and >= 0")
+    wgt = head_weights(inf32, within_layer)
+
+    if paper_rounding:
+        out = [0] * N
+        no_scores = not np.any(x > 0)                        # all-zero INF_sc: the pool in equal parts
+        for a in range(N):
+            b = float(fixed) + float(D) * (1.0 / N if no_scores else wgt[a])
+            c = int(math.floor(max(0.0, b) + 0.5))
+            out[a] = c if cap is None else min(c, int(cap))
+        return np.array(out, dtype=np.int64).reshape(L, H)
+
+    active = [True] * N
+    share = [0] * N                                          # dynamic part of every head
+    d_rem = D
+    room = None if cap is None else int(cap) - int(fixed)    # the most dynamic budget a head can take
+    while True:
+        W = 0.0
+        n_active = 0
+        for a in range(N):
+            if active[a]:
+                W = W + wgt[a]
+                n_active += 1
+        flat = not (W > 0.0)                                 # every weight left underflowed: share evenly
+        if flat:
+            W = float(n_active)
+        if room is None or n_active == 0:
+            break
+        newly = [a for a in range(N) if active[a] and (float(d_rem) * (1.0 if flat else wgt[a])) / W >= float(room)]
+        if not newly:
+            break
+        for a in newly:                                      # these heads are full; the rest share what is left
+            active[a] = False
+            share[a] = room
+            d_rem -= room
+
+    idx = [a for a in range(N) if active[a]]
+    f = {}
+    r = {}
+    for a in idx:
+        q = (float(d_rem) * (1.0 if flat else wgt[a])) / W
         fl = math.floor(q)
         f[a] = int(fl)
         r[a] = q - fl
-    R = D - sum(f)
-    if R >= N:                                               # cannot happen in exact arithmetic
-        for a in range(N):
-            f[a] += R // N
-        R = R % N
+    R = d_rem - sum(f.values())
+    n_act = len(idx)
+    if n_act and R >= n_act:                                 # cannot happen in exact arithmetic
+        for a in idx:
+            f[a] += R // n_act
+        R = R % n_act
     if R > 0:
-        order = sorted(range(N), key=lambda a: (-r[a], a))  # largest remainder, ties -> lower index
+        order = sorted(idx, key=lambda a: (-r[a], a))        # largest remainder, ties -> lower index
         for a in order[:R]:
             f[a] += 1
-    while R < 0:                                             # rounding pushed the floors above D
-        cand = [a for a in range(N) if f[a] > 0]
+    while R < 0:                                             # rounding pushed the floors above the pool
+        cand = [a for a in idx if f[a] > 0]
         order = sorted(cand, key=lambda a: (r[a], -a))       # smallest remainder, ties -> higher index
         take = order[:min(-R, len(order))]
         for a in take:
             f[a] -= 1
         R += len(take)
-    return (np.array(f, dtype=np.int64) + int(fixed)).reshape(L, H)
+    for a in idx:
+        share[a] = f[a]
+    return (np.array(share, dtype=np.int64) + int(fixed)).reshape(L, H)
 
 
 # ----------------------------------------------------------------------------------------------

@@ -32,6 +32,14 @@ class SlkvParams(C.Structure):
                                          "q_stride_seq", "q_stride_row", "q_stride_head")]
 
 
+class SlkvAllocOptions(C.Structure):
+    _fields_ = [("head_normaliser", C.c_int32), ("rounding", C.c_int32), ("cap", C.c_int64)]
+
+
+SLKV_NORM_GLOBAL, SLKV_NORM_WITHIN_LAYER = 0, 1
+SLKV_ROUND_SUM_EXACT, SLKV_ROUND_PAPER = 0, 1
+
+
 class SlkvError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -61,6 +69,10 @@ def lib() -> C.CDLL:
         L.slkv_version.restype = C.c_int
         L.slkv_alloc_budgets.restype = C.c_int
         L.slkv_alloc_budgets.argtypes = [vp, i32, i32, i32, i64, vp, vp, vp]
+        L.slkv_alloc_budgets_ex.restype = C.c_int
+        L.slkv_alloc_budgets_ex.argtypes = [vp, i32, i32, i32, i64, C.POINTER(SlkvAllocOptions), vp, vp, vp]
+        L.slkv_behavior_scores.restype = C.c_int
+        L.slkv_behavior_scores.argtypes = [vp, i64, i32, i64, vp, i32, i64, vp, i32, i64, vp, vp, vp, vp]
         L.slkv_workspace_bytes.restype = sz
         L.slkv_workspace_bytes.argtypes = [pp, i32p]
         L.slkv_pooled_elems.restype = i64
@@ -143,16 +155,42 @@ def slkv_last_launch_count() -> int:
 
 
 def slkv_alloc_budgets(inf_sc: torch.Tensor, fixed: int, total: int, budgets: Optional[torch.Tensor] = None,
-                       status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """inf_sc: CUDA float32 [n_layers, n_heads] -> CUDA int32 budgets of the same shape."""
+                       status: Optional[torch.Tensor] = None, stream=None,
+                       options: Optional[SlkvAllocOptions] = None) -> torch.Tensor:
+    """inf_sc: CUDA float32 [n_layers, n_heads] -> CUDA int32 budgets of the same shape (slkv_alloc_budgets, or
+    slkv_alloc_budgets_ex when `options` is given)."""
     assert inf_sc.is_cuda and inf_sc.dtype == torch.float32 and inf_sc.dim() == 2 and inf_sc.is_contiguous()
     if budgets is None:
         budgets = torch.empty(inf_sc.shape, dtype=torch.int32, device=inf_sc.device)
+    if options is not None:
+        rc = lib().slkv_alloc_budgets_ex(inf_sc.data_ptr(), inf_sc.shape[0], inf_sc.shape[1], int(fixed), int(total),
+                                         C.byref(options), budgets.data_ptr(), _ptr(status), _stream(stream))
+        if rc != SLKV_OK:
+            raise SlkvError(rc, "slkv_alloc_budgets_ex")
+        return budgets
     rc = lib().slkv_alloc_budgets(inf_sc.data_ptr(), inf_sc.shape[0], inf_sc.shape[1], int(fixed), int(total),
                                   budgets.data_ptr(), _ptr(status), _stream(stream))
     if rc != SLKV_OK:
         raise SlkvError(rc, "slkv_alloc_budgets")
     return budgets
+
+
+def slkv_behavior_scores(attn: torch.Tensor, needle_idx: torch.Tensor, topk_idx: torch.Tensor, stream=None):
+    """Algorithm 1 for a batch: attn CUDA float32 [n_rows, row_len]; needle_idx / topk_idx CUDA int32 [n_rows, n] or
+    [n] (one list for all rows), entries < 0 are padding.  Returns (SF_sc, LG_sc, INF_sc), CUDA float32 [n_rows]."""
+    assert attn.is_cuda and attn.dtype == torch.float32 and attn.dim() == 2 and attn.stride(1) == 1
+    n_rows, row_len = attn.shape
+    outs = [torch.empty(n_rows, dtype=torch.float32, device=attn.device) for _ in range(3)]
+
+    def lst(t):
+        assert t.is_cuda and t.dtype == torch.int32 and t.is_contiguous() and t.dim() in (1, 2)
+        return t.data_ptr(), t.shape[-1], (t.shape[-1] if t.dim() == 2 else 0)
+    (np_, nn, ns), (tp, tn, ts) = lst(needle_idx), lst(topk_idx)
+    rc = lib().slkv_behavior_scores(attn.data_ptr(), n_rows, row_len, attn.stride(0), np_, nn, ns, tp, tn, ts,
+                                    outs[0].data_ptr(), outs[1].data_ptr(), outs[2].data_ptr(), _stream(stream))
+    if rc != SLKV_OK:
+        raise SlkvError(rc, "slkv_behavior_scores")
+    return tuple(outs)
 
 
 def slkv_workspace_bytes(params: SlkvParams, cu_seqlens: Sequence[int]) -> int:

@@ -586,7 +586,7 @@ int slkv_profile_collect(float* total_ms, int32_t* launches, int32_t n_kernels) 
 const char* slkv_kernel_name(int kernel_id) {
   static const char* names[KID_COUNT] = {"k_setup", "k_score_lse", "k_score_vote", "k_pool", "k_select",
                                          "k_gather", "k_alloc", "k_score_fused", "k_score_pipe", "k_window_stats",
-                                         "k_merge_lse"};
+                                         "k_merge_lse", "k_behavior"};
   return (kernel_id >= 0 && kernel_id < KID_COUNT) ? names[kernel_id] : "";
 }
 
@@ -606,16 +606,50 @@ int slkv_debug_expire_next_wait(int on) {
   return SLKV_OK;
 }
 
-int slkv_alloc_budgets(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
-                       int32_t* budgets, int32_t* status, void* stream) {
+int slkv_behavior_scores(const float* attn, int64_t n_rows, int32_t row_len, int64_t row_stride,
+                         const int32_t* needle_idx, int32_t n_needle, int64_t needle_stride, const int32_t* topk_idx,
+                         int32_t n_topk, int64_t topk_stride, float* sf_sc, float* lg_sc, float* inf_sc, void* stream) {
+  if (!attn || !needle_idx || !topk_idx || !sf_sc || !lg_sc || !inf_sc) return SLKV_ERR_NULL_PTR;
+  if (n_rows < 0 || n_rows > (1ll << 34) || row_len < 1 || row_stride < 0 || n_needle < 0 || n_needle > 4096 ||
+      n_topk < 0 || n_topk > 4096 || needle_stride < 0 || topk_stride < 0)
+    return SLKV_ERR_BAD_SHAPE;
+  cudaError_t e = launch_behavior(attn, row_stride, row_len, n_rows, needle_idx, n_needle, needle_stride, topk_idx,
+                                  n_topk, topk_stride, sf_sc, lg_sc, inf_sc, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return SLKV_OK;
+}
+
+int slkv_alloc_budgets_ex(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
+                          const slkv_alloc_options* opt, int32_t* budgets, int32_t* status, void* stream) {
   if (!inf_sc || !budgets) return SLKV_ERR_NULL_PTR;
   if (n_layers < 1 || n_heads < 1 || n_layers > 1024 || (int64_t)n_layers * n_heads > 16384)
     return SLKV_ERR_BAD_SHAPE;
-  if (fixed < 0 || total < (int64_t)n_layers * n_heads * fixed) return SLKV_ERR_BUDGET_SUM;
+  const int64_t n = (int64_t)n_layers * n_heads;
+  if (fixed < 0 || total < n * fixed) return SLKV_ERR_BUDGET_SUM;
   if (total > 0x7fffffffll) return SLKV_ERR_BAD_SHAPE;
-  cudaError_t e = launch_alloc(inf_sc, n_layers, n_heads, fixed, total, budgets, status, (cudaStream_t)stream);
+  int within = 0, paper = 0;
+  long long cap = -1;
+  if (opt) {
+    if (opt->head_normaliser != SLKV_NORM_GLOBAL && opt->head_normaliser != SLKV_NORM_WITHIN_LAYER) return SLKV_ERR_BAD_DTYPE;
+    if (opt->rounding != SLKV_ROUND_SUM_EXACT && opt->rounding != SLKV_ROUND_PAPER) return SLKV_ERR_BAD_DTYPE;
+    if (opt->cap < 0 || opt->cap > 0x7fffffffll) return SLKV_ERR_BAD_SHAPE;
+    within = opt->head_normaliser == SLKV_NORM_WITHIN_LAYER;
+    paper = opt->rounding == SLKV_ROUND_PAPER;
+    if (opt->cap > 0) {
+      cap = opt->cap;
+      // a cap below the fixed part, or a total that does not fit under the cap (where the total is to be met)
+      if (cap < fixed || (!paper && total > n * cap)) return SLKV_ERR_BUDGET_SUM;
+    }
+  }
+  cudaError_t e = launch_alloc(inf_sc, n_layers, n_heads, fixed, total, within, paper, cap, budgets, status,
+                               (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e);
   return SLKV_OK;
+}
+
+int slkv_alloc_budgets(const float* inf_sc, int32_t n_layers, int32_t n_heads, int32_t fixed, int64_t total,
+                       int32_t* budgets, int32_t* status, void* stream) {
+  return slkv_alloc_budgets_ex(inf_sc, n_layers, n_heads, fixed, total, nullptr, budgets, status, stream);
 }
 
 size_t slkv_workspace_bytes(const slkv_params* p, const int32_t* cu_seqlens_host) {

@@ -119,7 +119,7 @@ struct Problem {
 };
 
 // kernel ids for launch accounting / per-kernel timing
-enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_SCORE_PIPE, KID_WINDOW_STATS, KID_MERGE_LSE, KID_COUNT };
+enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_SCORE_PIPE, KID_WINDOW_STATS, KID_MERGE_LSE, KID_BEHAVIOR, KID_COUNT };
 
 // Brackets one kernel launch: counts it and, when per-kernel timing is on for this thread, records a
 // CUDA event pair around it on the launch stream.
@@ -134,8 +134,11 @@ int check_score_args(const slkv_params* p, const void* q_win, const void* k, con
                      const int32_t* cu_seqlens_host, const float* pooled);
 
 // host-side launchers; each returns a cudaError_t and adds to *launches
-cudaError_t launch_alloc(const float* inf, int n_layers, int n_heads, int fixed, long long total, int32_t* budgets,
-                         int32_t* status, cudaStream_t st);
+cudaError_t launch_alloc(const float* inf, int n_layers, int n_heads, int fixed, long long total, int within_layer,
+                         int paper_rounding, long long cap, int32_t* budgets, int32_t* status, cudaStream_t st);
+cudaError_t launch_behavior(const float* attn, long long row_stride, int row_len, long long n_rows,
+                            const int32_t* needle_idx, int n_needle, long long needle_stride, const int32_t* topk_idx,
+                            int n_topk, long long topk_stride, float* sf, float* lg, float* inf, cudaStream_t st);
 cudaError_t launch_setup(const Problem& pb, const int32_t* budgets, int32_t* offsets, int64_t capacity,
                          int32_t* status, cudaStream_t st, int* launches);
 int simt_chunk_keys();

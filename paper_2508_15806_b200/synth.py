@@ -273,3 +273,39 @@ def layer_inputs(wl: Workload, layer: int, device="cpu") -> LayerInputs:
             k[cu[s]:cu[s] + wl.n_sinks] += wl.sink_gain * qm.unsqueeze(0)
     dt = wl.torch_dtype
     return LayerInputs(q.to(dt).contiguous(), k.to(dt).contiguous(), v.to(dt).contiguous(), needles)
+
+
+# ---------------------------------------------------------------------------------------------------
+# attention rows for the Stage-1 behaviour analysis (shapes of the paper's needle-in-a-haystack probes)
+# ---------------------------------------------------------------------------------------------------
+TID_ATTN = 9
+
+
+def behavior_rows(n_rows: int, row_len: int, n_needle: int = 12, top_k: int = 16, seed: int = 11, device="cpu"):
+    """Attention-weight rows as a needle-in-a-haystack probe produces them, with their index sets.
+
+    Every row is a probability vector over `row_len` context positions: a heavy first position (attention sink),
+    a contiguous needle span of `n_needle` tokens at a seeded depth that receives a seeded share of the mass
+    (near 0 for heads that ignore the needle, most of it for retrieval heads), a few seeded distractor spikes
+    elsewhere, and a lognormal background.  Returns (attn float32 [n_rows, row_len], needle_idx int32
+    [n_rows, n_needle], topk_idx int32 [n_rows, top_k]); topk_idx are the positions of the row's top_k largest
+    weights (equal weights: lower position first), the input Algorithm 1 calls T.
+    """
+    assert row_len > n_needle + 8 and top_k <= row_len
+    key = stream_key(seed, TID_ATTN)
+    bg = torch.exp(0.7 * normal(key, n_rows * row_len, device)).reshape(n_rows, row_len)
+    u = uniform(stream_key(seed, TID_ATTN, 1), n_rows * 8, device).reshape(n_rows, 8)
+    start = 1 + (u[:, 0] * (row_len - n_needle - 1)).to(torch.int64)                  # needle depth
+    needle = start[:, None] + torch.arange(n_needle, device=device)[None, :]
+    share = u[:, 1] ** 3                                                               # most heads: little mass on it
+    bg = bg / bg.sum(dim=1, keepdim=True) * (1.0 - share)[:, None] * 0.7
+    rows = bg.clone()
+    rows[:, 0] += 0.3 * (1.0 - share)                                                  # the sink
+    w_needle = torch.exp(1.2 * normal(stream_key(seed, TID_ATTN, 2), n_rows * n_needle, device)).reshape(n_rows, n_needle)
+    rows.scatter_add_(1, needle, w_needle / w_needle.sum(dim=1, keepdim=True) * share[:, None])
+    for d in range(3):                                                                 # distractor spikes
+        pos = 1 + (u[:, 2 + d] * (row_len - 1)).to(torch.int64)
+        rows.scatter_add_(1, pos[:, None], (0.05 * u[:, 5 + d] * (1.0 - share))[:, None])
+    rows = (rows / rows.sum(dim=1, keepdim=True)).to(torch.float32)
+    order = torch.sort(rows.to(torch.float64), dim=1, descending=True, stable=True).indices[:, :top_k]
+    return rows.contiguous(), needle.to(torch.int32).contiguous(), order.to(torch.int32).contiguous()

@@ -88,6 +88,22 @@ def test_alloc_argument_errors(L):
     assert f(fake, 2048, 32, 0, 255, fake, None, None) == B.ERR["BAD_SHAPE"]
 
 
+def test_alloc_ex_argument_errors(L):
+    fake = C.c_void_p(4096)
+    f = L.slkv_alloc_budgets_ex
+    opt = B.SlkvAllocOptions(head_normaliser=0, rounding=0, cap=0)
+    assert f(None, 1, 8, 32, 1024, C.byref(opt), fake, None, None) == B.ERR["NULL_PTR"]
+    assert f(fake, 1, 8, 32, 255, None, fake, None, None) == B.ERR["BUDGET_SUM"]
+    for kw, code in [(dict(head_normaliser=2), "BAD_DTYPE"), (dict(rounding=5), "BAD_DTYPE"), (dict(cap=-1), "BAD_SHAPE"),
+                     (dict(cap=31), "BUDGET_SUM"), (dict(cap=100), "BUDGET_SUM")]:
+        o = B.SlkvAllocOptions(head_normaliser=0, rounding=0, cap=0)
+        for k, v in kw.items():
+            setattr(o, k, v)
+        assert f(fake, 1, 8, 32, 1024, C.byref(o), fake, None, None) == B.ERR[code], kw
+    # Algorithm 2's own rounding does not meet a total, so a cap that the total does not fit under is accepted
+    # (the launch itself needs a device, so only the rejections are checked here)
+
+
 def test_compress_argument_errors(L):
     fake = C.c_void_p(4096)
     cu = (C.c_int32 * 2)(0, 100)

@@ -183,6 +183,134 @@ def test_tables_6_8_consistent_with_harmonic_mean():
         assert 0.0 < LG <= 1.0 and sf[head] < inf[head] < LG        # harmonic mean lies between the two
         if head not in lg:
             assert LG < lg10
-        # and the oracle's step 7 reproduces the table value from (SF, LG)
-        W = np.array([1.0])
-        assert abs(2 * sf[head] * LG / (sf[head] + LG) - inf[head]) < 1e-12
+        # an attention row with exactly these SF and LG: one needle token inside the top-k set (weight WO), one
+        # outside it (WS), one top-k token that is no needle (WD); Algorithm 1 on it must print the table's INF_sc
+        WO = 0.3
+        WD, WS = WO * (1 - sf[head]) / sf[head], WO * (1 - LG) / LG
+        W = np.array([WO, WS, WD, 1.0 - WO - WS - WD])
+        got_sf, got_lg, got_inf = O.behavior_scores(W, needle_idx=[0, 1], topk_idx=[0, 2])
+        assert abs(got_sf - sf[head]) < 1e-12 and abs(got_lg - LG) < 1e-12
+        assert abs(got_inf - inf[head]) < 1e-12
+
+
+# ---- variants: head normaliser of the prose under Eq. 6, per-head cap, Algorithm 2's own rounding -----------------
+def waterfill_exact(weights, D, room):
+    """Apportion D seats by exact-rational weights with at most `room` seats per head: heads whose exact quota
+    reaches `room` are filled and removed, the rest share what is left, until none does; then largest remainder
+    (independent of the oracle: Fractions only)."""
+    n = len(weights)
+    active = list(range(n))
+    seats = [0] * n
+    left = D
+    while active:
+        tot = sum(Fraction(weights[a]) for a in active)
+        full = [a for a in active if Fraction(weights[a]) * left / tot >= room]
+        if not full:
+            break
+        for a in full:
+            seats[a] = room
+            left -= room
+            active.remove(a)
+    if active:
+        tot = sum(Fraction(weights[a]) for a in active)
+        quota = {a: Fraction(weights[a]) * left / tot for a in active}
+        for a in active:
+            seats[a] = quota[a].numerator // quota[a].denominator
+        rest = left - sum(seats[a] for a in active)
+        for a in sorted(active, key=lambda a: (-(quota[a] - seats[a]), a))[:rest]:
+            seats[a] += 1
+    return seats
+
+
+def test_within_layer_equals_global_on_one_layer():
+    rng = np.random.default_rng(5)
+    for _ in range(5):
+        inf = rng.lognormal(0, 1.5, size=(1, 9))
+        a = O.alloc_budgets(inf, 16, 16 * 9 + 4000)
+        b = O.alloc_budgets(inf, 16, 16 * 9 + 4000, within_layer=True)
+        assert np.array_equal(a, b)
+
+
+def test_within_layer_hand_example():
+    # inf = [[1,1],[1,7]]: layer sums 2 and 8 of 10, so the layer factors are 0.21 and 0.81.
+    # global head shares [[.1,.1],[.1,.7]]  -> weights [[.021,.021],[.081,.567]], sum .69
+    # layer-wise shares  [[.5,.5],[.125,.875]] -> weights [[.105,.105],[.10125,.70875]], sum 1.02
+    inf = np.array([[1.0, 1.0], [1.0, 7.0]])
+    assert (O.alloc_budgets(inf, 0, 690) == np.array([[21, 21], [81, 567]])).all()
+    # 1020 * w / 1.02 = [[105, 105], [101.25, 708.75]]: the odd seat goes to the larger remainder
+    assert (O.alloc_budgets(inf, 0, 1020, within_layer=True) == np.array([[105, 105], [101, 709]])).all()
+    # fixed parts ride on top
+    assert (O.alloc_budgets(inf, 3, 1020 + 12, within_layer=True) == np.array([[108, 108], [104, 712]])).all()
+
+
+def test_within_layer_makes_the_layer_floor_effective():
+    # a layer with next to no influence keeps ~0.01 / (1 + 0.01 L) of the pool under the layer-wise normaliser
+    # (what Sec. 3.3's "minimum layer budget" is for) and next to nothing under the global one
+    rng = np.random.default_rng(6)
+    L, H, D = 8, 6, 1_000_000
+    inf = rng.lognormal(0, 1.0, size=(L, H))
+    inf[3] = 1e-9
+    g = O.alloc_budgets(inf, 0, D)
+    w = O.alloc_budgets(inf, 0, D, within_layer=True)
+    assert g[3].sum() <= 1
+    assert abs(w[3].sum() - D * 0.01 / (1.0 + 0.01 * L)) <= H
+    # every layer's total follows (0.01 + L_i) / (1 + 0.01 L)
+    Li = inf.sum(axis=1) / inf.sum()
+    assert np.all(np.abs(w.sum(axis=1) - D * (0.01 + Li) / (1.0 + 0.01 * L)) <= H)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_cap_matches_exact_rational_water_filling(seed):
+    rng = np.random.default_rng(300 + seed)
+    while True:
+        H = int(rng.integers(3, 10))
+        inf = rng.integers(1, 40, size=(1, H))
+        inf[0, rng.integers(0, H)] *= 25                   # one head would take most of the pool
+        fixed = int(rng.integers(0, 10))
+        room = int(rng.integers(20, 200))
+        D = int(rng.integers(room, room * H))              # feasible, and at least one head hits the cap
+        # fp64 quotas cannot reproduce exact ties between remainders: draw again when the exact remainders of the
+        # heads that stay below the cap are not all different
+        seats = waterfill_exact([int(v) for v in inf[0]], D, room)
+        open_heads = [a for a in range(H) if seats[a] < room]
+        left = D - room * (H - len(open_heads))
+        tot = sum(int(inf[0, a]) for a in open_heads)
+        rems = [Fraction(int(inf[0, a]) * left, tot) % 1 for a in open_heads]
+        if len(set(rems)) == len(rems):
+            break
+    C = O.alloc_budgets(inf.astype(np.float64), fixed, fixed * H + D, cap=fixed + room)
+    assert (C - fixed).ravel().tolist() == waterfill_exact([int(v) for v in inf[0]], D, room)
+    assert int(C.sum()) == fixed * H + D and C.max() <= fixed + room and C.min() >= fixed
+
+
+def test_cap_edges():
+    inf = np.array([[100.0, 1.0, 1.0]])
+    # no head reaches the cap: same as without
+    assert np.array_equal(O.alloc_budgets(inf, 5, 15 + 30, cap=1000), O.alloc_budgets(inf, 5, 15 + 30))
+    # total == N * cap: everybody is full
+    assert O.alloc_budgets(inf, 5, 3 * 40, cap=40).ravel().tolist() == [40, 40, 40]
+    # the heavy head is filled, the others split the rest evenly (equal weights): 5 + 35, then 20 over two heads
+    assert O.alloc_budgets(inf, 5, 15 + 55, cap=40).ravel().tolist() == [40, 15, 15]
+    # chain: filling one head pushes the next one over the cap as well
+    assert O.alloc_budgets(np.array([[50.0, 30.0, 1.0, 1.0]]), 0, 100, cap=35).ravel().tolist() == [35, 35, 15, 15]
+    for bad in (dict(cap=4), dict(cap=10)):                # cap below fixed; total above N * cap
+        with pytest.raises(O.OracleError) as e:
+            O.alloc_budgets(inf, 5, 15 + 30, **bad)
+        assert e.value.code == "BUDGET_SUM"
+
+
+def test_paper_rounding_agrees_with_the_papers_parameters():
+    # (fixed, total) = (b_c (1 - 1/beta), b_c L H): the same numbers as Eq. 6 in (b_c, beta)
+    rng = np.random.default_rng(7)
+    inf = rng.lognormal(0, 1.5, size=(5, 4))
+    b_c, beta = 128.0, 4.0 / 3.0                           # fixed 32, pool 96 per head
+    a = O.alloc_paper_literal(b_c, beta, inf)
+    b = O.alloc_budgets(inf, 32, 128 * 20, paper_rounding=True)
+    assert np.array_equal(a, b)
+    assert int(b.sum()) != 128 * 20                        # not normalised: the sum is not the total
+    # the hand example of Eq. 6: fixed 50, pool 200
+    assert O.alloc_budgets(np.array([[1.0, 3.0], [2.0, 2.0]]), 50, 400, paper_rounding=True).tolist() == [[63, 88], [76, 76]]
+    # clipped at the cap, nothing handed on
+    assert O.alloc_budgets(np.array([[1.0, 3.0], [2.0, 2.0]]), 50, 400, paper_rounding=True, cap=80).tolist() == [[63, 80], [76, 76]]
+    # all-zero scores: the pool in equal parts
+    assert O.alloc_budgets(np.zeros((2, 2)), 10, 40 + 10, paper_rounding=True).tolist() == [[13, 13], [13, 13]]
