@@ -36,6 +36,54 @@ def test_two_ranks_shard_by_sequence_batch_and_time_by_the_slowest(tmp_path):
     assert abs(r[0]["value"] - 2 * 300 / 15e-3) < 1e-6                        # whole-job tokens/s/layer
 
 
+def _head_shard_main(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from oracle import slkv_oracle as O
+    from paper_2508_15806_b200 import sharding as S
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    # a layer of 5 KV heads over 2 ranks (3 + 2), 3 sequences; the kept counts a rank's compression would report for
+    # its heads come from the oracle's rule here (no GPU in this test): what is checked is the exchange and stitching
+    n_kv, window, lens, budgets = 5, 4, [30, 3, 9], [6, 40, 2, 9, 12]
+    h0, h1 = S.head_range(n_kv, rank, world)
+    kept = torch.tensor([[sum(O.kept_counts(n, budgets[h], window)) for h in range(h0, h1)] for n in lens], dtype=torch.int32)
+    local_offsets = torch.zeros(kept.numel() + 1, dtype=torch.int32)
+    local_offsets[1:] = torch.cumsum(kept.reshape(-1), 0)
+    assert torch.equal(S.local_kept(local_offsets, len(lens), h1 - h0), kept)
+    offsets, bases = S.stitch(S.all_gather_kept(kept))
+    with open(os.path.join(out_dir, f"h{rank}.json"), "w") as f:
+        json.dump({"range": [h0, h1], "offsets": offsets.tolist(), "base": bases[rank].tolist()}, f)
+    dist.destroy_process_group()
+
+
+def test_two_ranks_shard_by_kv_head_and_stitch_offsets(tmp_path):
+    from oracle import slkv_oracle as O
+    world, port = 2, 31000 + os.getpid() % 2000
+    mp.spawn(_head_shard_main, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    r = [json.load(open(tmp_path / f"h{i}.json")) for i in range(world)]
+    assert r[0]["range"] == [0, 3] and r[1]["range"] == [3, 5]
+    n_kv, window, lens, budgets = 5, 4, [30, 3, 9], [6, 40, 2, 9, 12]
+    expect = [0]
+    for n in lens:
+        for h in range(n_kv):
+            expect.append(expect[-1] + sum(O.kept_counts(n, budgets[h], window)))
+    assert r[0]["offsets"] == expect and r[1]["offsets"] == expect            # every rank ends with the same offsets
+    for rank in range(world):
+        h0, h1 = r[rank]["range"]
+        for s in range(len(lens)):
+            assert r[rank]["base"][s] == [expect[s * n_kv + h] for h in range(h0, h1)]
+
+
+def test_head_ranges_cover_all_heads():
+    from paper_2508_15806_b200 import sharding as S
+    for n_kv in (1, 5, 8, 9):
+        for world in (1, 2, 3, 4, 8):
+            rs = [S.head_range(n_kv, r, world) for r in range(world)]
+            assert rs[0][0] == 0 and rs[-1][1] == n_kv and all(a[1] == b[0] for a, b in zip(rs, rs[1:]))
+            assert max(b - a for a, b in rs) - min(b - a for a, b in rs) <= 1
+
+
 def test_reference_arm_only_rank0_works():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
