@@ -32,15 +32,35 @@ METRIC = "context tokens compressed per second per layer"
 UNIT = "tokens/s/layer"
 WORKLOAD_INDEX = 2          # the 32k-context, 32-layer configuration (third of the five workloads)
 TOTAL_INDEX = 1             # average budget 512 per KV head
-# DRAM bytes per key row (256 B of K) of one launch, from an ncu capture of the kernel as it stands; a kernel
-# that has changed since its capture has no entry (traffic is then reported as null)
-DRAM_TRAFFIC_PER_KEY_ROW = {
-    "k_score_fused": {"bytes": 262.6, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch "
-                      "(68.77 MB) / (8 KV heads x 32736 history rows): profiles/k_score_fused_cfg3_4layers.txt"},
-    "k_score_pipe": {"bytes": 442.5, "source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of 8 "
-                     "layers (927.1 MB) / (8 layers x 8 KV heads x 32736 history rows): "
-                     "profiles/k_score_pipe_cfg3_8layers.txt; a launch's traffic is this x the layers it takes"},
-}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic_per_key_row.txt")
+KERNEL_SOURCES = {"k_score_pipe": ["slkv_score_pipe.cu", "slkv_tc_device.cuh"],
+                  "k_score_fused": ["slkv_score_tc.cu", "slkv_tc_device.cuh"]}
+
+
+def source_sha16(kernel: str):
+    """First 16 hex digits of the SHA-256 of the kernel's source files (to tell whether a capture is still current)."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES.get(kernel, []):
+        with open(os.path.join(ROOT, "paper_2508_15806_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def dram_traffic_per_key_row(kernel: str, mode: str):
+    """DRAM bytes per key row (256 B of K) of one launch from the tracked ncu summary, or None when there is no
+    capture of this kernel and mode, or the kernel's sources have changed since the capture was taken."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                t = line.split()
+                if len(t) >= 4 and not line.startswith("#") and t[0] == kernel and t[1] == mode:
+                    if t[3] != source_sha16(kernel):
+                        return None
+                    return {"bytes": float(t[2]), "source": "profiles/" + " ".join(t[4:])}
+    except OSError:
+        pass
+    return None
 
 
 def measured_peaks():
@@ -239,32 +259,46 @@ def run_cuda(args):
     eager_step = step
     eager_us_per_layer = None
     use_graph = overlap and not args.no_graph
-    if use_graph:
-        # The calls of a step are stream-ordered and allocate nothing: capture them once (the side streams of the
-        # overlapped calls fork from and rejoin the captured stream) and replay the graph per step.
+
+    def captured(fn):
+        """fn's calls captured once in a CUDA graph (they are stream-ordered and allocate nothing; the side streams
+        of the overlapped calls fork from and rejoin the captured stream); returns the replaying step."""
+        nonlocal stream
+        cap = torch.cuda.Stream()
+        stream = cap
         try:
-            cap = torch.cuda.Stream()
-            stream = cap
             with torch.cuda.stream(cap):
-                eager_step()
+                fn()
             torch.cuda.synchronize()
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=cap):
-                eager_step()
+                fn()
+        finally:
             stream = torch.cuda.current_stream()
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        return graph.replay
 
-            def step():
-                graph.replay()
-            for _ in range(2):
-                step()
-            torch.cuda.synchronize()
-            assert int(status.item()) == 0
+    def lse_eager_step():
+        use_lse[0] = True
+        try:
+            eager_step()
+        finally:
+            use_lse[0] = bool(args.with_lse)
+
+    lse_step = lse_eager_step
+    if use_graph:
+        try:
+            step = captured(eager_step)
+            lse_step = captured(lse_eager_step)
         except Exception as exc:                       # no capture on this driver: issue the calls every step
             print(f"bench: CUDA graph capture failed ({exc}); timing the calls themselves", file=sys.stderr)
             torch.cuda.synchronize()
             B.slkv_join()
             stream = torch.cuda.current_stream()
-            step = eager_step
+            step, lse_step = eager_step, lse_eager_step
             use_graph = False
     steps = args.steps
     if steps is None:                                   # aim at ~3 s of timed work
@@ -274,23 +308,69 @@ def run_cuda(args):
     sampler = ClockSampler(local)
     sampler.start()
     ms_total = timed(steps, step)
+    sampler.stop()
+    clocks = sampler.summary()
+    ms_per_step = ms_total / steps
+
     if use_graph:
         # the same calls issued every step, right behind the timed run (same clocks and temperature)
         n_eager = max(10, min(steps, 300))
         eager_us_per_layer = timed(n_eager, eager_step) / n_eager * 1e3 / nl
-    # same steps again with an event pair around every kernel: attributes the time to kernels
-    B.slkv_profile_enable(True)
+    # ---- attribution, (1): the score kernels alone bracketed by event pairs, everything else where it normally runs
+    # (selections and gathers on their side streams): the dominant kernel's time in the regime of the timed step,
+    # taken right behind it
+    prof_steps = min(max(steps, 10), 50)
+    B.slkv_profile_enable(2)
     barrier()
-    prof_steps = min(steps, 50)
+    for _ in range(3):
+        eager_step()
+    torch.cuda.synchronize()
+    B.slkv_profile_collect()
+    regime_ms = timed(prof_steps, eager_step) / prof_steps
+    score_kernels = B.slkv_profile_collect()
+    B.slkv_profile_enable(0)
+
+    # ---- the same step with every layer's row log-sum-exps handed over by the caller (vote pass only); not the headline
+    with_lse = None
+    if overlap and not args.with_lse:
+        first = timed(steps, lse_step) / steps                      # as many steps as the headline
+        with_lse = {"us_per_layer": first * 1e3 / nl, "value": whole_job_value(world, T, nl, first),
+                    "what": "lse_opt of slkv_compress_overlapped = the rows' log-sum-exps (from slkv_row_lse, outside "
+                            "the timed region), as a prefill attention kernel that keeps its softmax statistics hands "
+                            "them over: the score kernel runs the vote pass alone"}
+
+    # ---- the same steps for at least two more seconds: the figures the part holds once its power limit has engaged
+    sustained = None
+    if not args.no_sustained:
+        n_sus = max(steps, int(math.ceil(2200.0 / max(ms_per_step, 1e-3))))
+        sus_sampler = ClockSampler(local)
+        sus_sampler.start()
+        sus_ms = timed(n_sus, step) / n_sus
+        sus_sampler.stop()
+        sustained = {"steps": n_sus, "ms_per_step": sus_ms, "us_per_layer": sus_ms * 1e3 / nl,
+                     "value": whole_job_value(world, T, nl, sus_ms), "clocks": sus_sampler.summary()}
+        if with_lse:
+            n_lse = int(math.ceil(1500.0 / max(with_lse["us_per_layer"] * nl * 1e-3, 1e-3)))
+            lse_sampler = ClockSampler(local)
+            lse_sampler.start()
+            held = timed(n_lse, lse_step) / n_lse
+            lse_sampler.stop()
+            with_lse["sustained_us_per_layer"] = held * 1e3 / nl
+            with_lse["sustained_clocks"] = lse_sampler.summary()
+
+    # ---- attribution, (2): every kernel bracketed, on one stream: the other kernels' own times (that step is slower
+    # than the timed one); the score kernels' figures stay those of (1)
+    B.slkv_profile_enable(1)
+    barrier()
     for _ in range(prof_steps):
         eager_step()
     torch.cuda.synchronize()
     per_kernel = B.slkv_profile_collect()
-    B.slkv_profile_enable(False)
-    sampler.stop()
+    B.slkv_profile_enable(0)
+    for name, v in score_kernels.items():
+        per_kernel[name] = v
     assert int(status.item()) == 0
 
-    ms_per_step = ms_total / steps
     t_layer_us = ms_per_step * 1e3 / nl
     value = whole_job_value(world, T, nl, ms_per_step)
 
@@ -351,9 +431,9 @@ def run_cuda(args):
     alg_top = alg[top] * layers_per_launch
     achieved = alg_top / (top_us * 1e-6) / 1e9
     layer_bytes = k_scan + q_bytes + 4 * rows_avg * d * e
-    flops_layer = 2 * 2.0 * wl.n_q_heads * w * n_hist * d           # two softmax passes
-    exps_layer = 2.0 * wl.n_q_heads * w * n_hist
-    clocks = sampler.summary()
+    passes = 1 if args.with_lse else 2                              # row statistics + votes, or votes alone
+    flops_layer = passes * 2.0 * wl.n_q_heads * w * n_hist * d
+    exps_layer = float(passes) * wl.n_q_heads * w * n_hist
     f_sm = (clocks["sm_mhz"] or 1965.0) * 1e6
     ceilings = {"t_hbm_us": layer_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6,
                 "t_tensor_us": flops_layer / (peaks["bf16_tflops"] * 1e12) * 1e6,
@@ -374,10 +454,22 @@ def run_cuda(args):
         roofline["alu"] = {"bound": "alu", "unit": "Gexp/s", "achieved": n_exp / (top_us * 1e-6) / 1e9, "peak": peak_gexp,
                            "frac": n_exp / (top_us * 1e-6) / 1e9 / peak_gexp, "exps_per_launch": n_exp,
                            "peak_source": "148 SMs x 16 ex2.approx per clock x 1965 MHz (nominal unit count and maximum clock)"}
-    tr = DRAM_TRAFFIC_PER_KEY_ROW.get(top)
+    tr = dram_traffic_per_key_row(top, "lse" if args.with_lse else "two_pass")
     if tr:
         roofline["traffic"] = tr["bytes"] * hkv * n_hist * layers_per_launch
         roofline["traffic_source"] = tr["source"]
+    # the dominant kernel's launches of one step, timed in the step's own regime, must fit inside that step
+    roofline["kernel_us_per_step"] = top_us * kern[top]["launches_per_step"]
+    roofline["step_us_in_that_regime"] = regime_ms * 1e3
+    if top in score_kernels:
+        assert roofline["kernel_us_per_step"] <= regime_ms * 1e3 * 1.02, "per-kernel timing exceeds the step it is a share of"
+    if sustained:
+        sustained["layer_frac_of_hbm"] = layer_bytes / (sustained["us_per_layer"] * 1e-6) / 1e9 / peaks["hbm_gbs"]
+    if with_lse:
+        lb = layer_bytes + 4 * len(wl.seq_lens) * wl.n_q_heads * w          # + the log-sum-exps read
+        with_lse["layer_frac_of_hbm"] = lb / (with_lse["us_per_layer"] * 1e-6) / 1e9 / peaks["hbm_gbs"]
+        if "sustained_us_per_layer" in with_lse:
+            with_lse["sustained_layer_frac_of_hbm"] = lb / (with_lse["sustained_us_per_layer"] * 1e-6) / 1e9 / peaks["hbm_gbs"]
 
     # ---- the oracle on the host cores (rank 0, N=1 only): a reported baseline, not a target
     cpu_baseline = None
@@ -388,11 +480,15 @@ def run_cuda(args):
     if rank == 0:
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
                "ms_per_step": ms_per_step, "us_per_layer": t_layer_us, "us_per_layer_without_graph": eager_us_per_layer,
+               "us_per_layer_with_lse": with_lse["us_per_layer"] if with_lse else None,
+               "sustained": sustained, "with_lse": with_lse,
                "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
                "config": {"workload": wl.name, "n_layers": nl, "n_q_heads": wl.n_q_heads, "n_kv_heads": hkv,
                           "head_dim": d, "seq_lens": wl.seq_lens, "window": w, "pool_kernel": wl.pool_kernel,
-                          "avg_budget_per_kv_head": total // (nl * hkv), "fixed": wl.fixed, "parallelism":
+                          "avg_budget_per_kv_head": total // (nl * hkv), "fixed": wl.fixed,
+                          "row_lse": "supplied by the caller (--with-lse)" if args.with_lse else "computed (two passes over K)",
+                          "parallelism":
                           f"dp{world} (one sequence batch per GPU, no collective)",
                           "api": ("slkv_compress_overlapped + slkv_join per step" +
                                   (", captured once in a CUDA graph and replayed" if use_graph else ""))
@@ -498,6 +594,7 @@ def main():
                     help="hand every layer's row log-sum-exps to the calls (vote pass only); not the headline")
     ap.add_argument("--no-overlap", action="store_true", help="one layer at a time (slkv_compress) instead of overlapped calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the two extra seconds of the same step")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--e2e-layers", type=int, default=8, help="distinct layers kept in pinned host memory")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)

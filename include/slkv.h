@@ -329,6 +329,9 @@ int slkv_last_launch_count(void);
  * Per-kernel timing for benchmarks (no counterpart in the paper).  While enabled on the calling thread,
  * every kernel the library enqueues is bracketed by a CUDA event pair on its stream (events are created
  * on demand and reused; this adds host work per launch, so headline timings are taken with it off).
+ * on = 1: every kernel, and the overlapped entry point keeps selections and gathers on the caller's stream so that
+ * the pairs do not overlap (the step is then slower than untimed); on = 2: the score kernels only, everything else
+ * where it normally runs -- the score kernels' times in the regime of an untimed step; on = 0: off.
  * slkv_profile_collect waits for the recorded events, adds each kernel's elapsed milliseconds and launch
  * count into total_ms[id] / launches[id] (arrays of n_kernels entries, overwritten) and forgets the records.
  * Kernel ids run from 0 to slkv_kernel_count()-1; slkv_kernel_name gives their names.
@@ -350,7 +353,7 @@ int slkv_kernel_count(void);
  * stream B, 60 / 61 the SM cycle counter at CTA start / end.  The buffer that is set when a launch is enqueued is
  * the one it writes (the overlapped entry point enqueues a list when it is full and one more layer has come, or at
  * a join).  The buffer must hold 2 * n_cta * 64 * 8 bytes (n_cta <= number of SMs); smaller buffers switch tracing
- * off.  NULL switches it off.  python -m paper_2508_15806_b200.trace_timeline prints a step's timeline from it.
+ * off.  NULL switches it off.
  */
 int slkv_trace_set_buffer(void* dev_buf, size_t bytes);
 

@@ -320,8 +320,9 @@ def slkv_compress_host(params: SlkvParams, q_win, k, v, cu_seqlens: Sequence[int
     return int(rows.value)
 
 
-def slkv_profile_enable(on: bool) -> None:
-    lib().slkv_profile_enable(1 if on else 0)
+def slkv_profile_enable(on) -> None:
+    """False / 0: off; True / 1: every kernel (one stream); 2: the score kernels only, side streams kept."""
+    lib().slkv_profile_enable(int(on))
 
 
 def slkv_profile_collect() -> dict:

@@ -14,7 +14,7 @@ thread_local int g_last_launches = 0;
 
 // ---- per-kernel timing (off by default) -----------------------------------------------------------
 struct TimedLaunch { int kid; cudaEvent_t a, b; };
-thread_local bool g_prof_on = false;
+thread_local int g_prof_on = 0;          // 0 off, 1 every kernel (one stream), 2 the score kernels only (side streams kept)
 thread_local std::vector<TimedLaunch>* g_prof = nullptr;      // records of the current thread
 thread_local std::vector<cudaEvent_t>* g_prof_free = nullptr;
 
@@ -312,7 +312,7 @@ cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pip
   const int slot = c.slot;
   const int si = wide ? slot % kSideStreams : slot % 2;
   cudaStream_t sel = os->side_select[si], gat = os->side_gather[si];
-  if (g_prof_on) sel = gat = c.st;       // per-kernel timing: one stream, so that the event pairs do not overlap
+  if (g_prof_on == 1) sel = gat = c.st;  // timing of every kernel: one stream, so that the event pairs do not overlap
   cudaError_t e = cudaEventRecord(os->scored[slot], c.st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(sel, os->scored[slot], 0);
   if (e == cudaSuccess && os->wait_done[slot]) e = cudaStreamWaitEvent(sel, os->done[slot], 0);
@@ -525,6 +525,8 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
 LaunchScope::LaunchScope(int kid, cudaStream_t st, int* launches) : kid_(kid), st_(st), slot_(-1) {
   ++*launches;
   if (!g_prof_on) return;
+  const bool score_kid = kid == KID_SCORE_LSE || kid == KID_SCORE_VOTE || kid == KID_SCORE_FUSED || kid == KID_SCORE_PIPE;
+  if (g_prof_on == 2 && !score_kid) return;
   if (!g_prof) g_prof = new std::vector<TimedLaunch>();
   TimedLaunch t{kid, prof_event(), prof_event()};
   if (!t.a || !t.b) return;
@@ -560,7 +562,7 @@ const char* slkv_strerror(int status) {
 }
 
 int slkv_profile_enable(int on) {
-  g_prof_on = on != 0;
+  g_prof_on = on < 0 ? 0 : (on > 2 ? 1 : on);
   return SLKV_OK;
 }
 
