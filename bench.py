@@ -333,6 +333,10 @@ def run_cuda(args):
     # ---- the same step with every layer's row log-sum-exps handed over by the caller (vote pass only); not the headline
     with_lse = None
     if overlap and not args.with_lse:
+        torch.cuda.synchronize()
+        time.sleep(1.5)                                             # idle, as before the headline's timed steps
+        for _ in range(warmup):
+            lse_step()
         first = timed(steps, lse_step) / steps                      # as many steps as the headline
         with_lse = {"us_per_layer": first * 1e3 / nl, "value": whole_job_value(world, T, nl, first),
                     "what": "lse_opt of slkv_compress_overlapped = the rows' log-sum-exps (from slkv_row_lse, outside "
