@@ -263,6 +263,7 @@ struct OverlapState {
   unsigned seq = 0;
   std::vector<PendingCall> queue;        // layers whose score kernel is not launched yet (at most kPipeMaxLayers + 1)
   PendingCall pending;                   // pass 1 launched, pass 2 not
+  std::vector<PendingCall> deferred;     // votes launched and `scored` recorded, selection and gather not enqueued yet
   ShapeSig sig;
 };
 constexpr int kMaxDevices = 64;
@@ -298,7 +299,14 @@ cudaError_t overlap_state(OverlapState** out) {
 
 // Before a layer takes a slot: its vote array may still be read by the selection of the layer that had the slot,
 // its source-row list by that layer's gather.
-cudaError_t claim_slot(OverlapState* os, int slot, cudaStream_t st) {
+cudaError_t flush_deferred(OverlapState* os, int* launches);
+cudaError_t claim_slot(OverlapState* os, int slot, cudaStream_t st, int* launches) {
+  for (size_t i = 0; i < os->deferred.size(); ++i)
+    if (os->deferred[i].slot == slot) {                              // its selection is not even enqueued yet
+      cudaError_t e = flush_deferred(os, launches);
+      if (e != cudaSuccess) return e;
+      break;
+    }
   if (!os->in_flight[slot]) return cudaSuccess;
   os->wait_done[slot] = true;
   return cudaStreamWaitEvent(st, os->selected[slot], 0);
@@ -307,13 +315,14 @@ cudaError_t claim_slot(OverlapState* os, int slot, cudaStream_t st) {
 // The votes of layer `c` are enqueued on c.st: selection on a side stream, gather on another.  While more score
 // launches follow, two selections at a time (a selection takes one SM per segment, and a score launch whose CTAs wait
 // for one another starts only when all of them fit beside what is running); `wide`: nothing follows, all side
-// streams.
-cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pipe, bool wide, int* launches) {
+// streams.  `scored_recorded`: the layer's event was recorded when its votes were launched (a deferred tail).
+cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pipe, bool wide, int* launches,
+                         bool scored_recorded = false) {
   const int slot = c.slot;
   const int si = wide ? slot % kSideStreams : slot % 2;
   cudaStream_t sel = os->side_select[si], gat = os->side_gather[si];
   if (g_prof_on == 1) sel = gat = c.st;  // timing of every kernel: one stream, so that the event pairs do not overlap
-  cudaError_t e = cudaEventRecord(os->scored[slot], c.st);
+  cudaError_t e = scored_recorded ? cudaSuccess : cudaEventRecord(os->scored[slot], c.st);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(sel, os->scored[slot], 0);
   if (e == cudaSuccess && os->wait_done[slot]) e = cudaStreamWaitEvent(sel, os->done[slot], 0);
   os->wait_done[slot] = false;
@@ -333,6 +342,16 @@ cudaError_t enqueue_tail(OverlapState* os, const PendingCall& c, bool beside_pip
   return cudaSuccess;
 }
 
+// Selections and gathers that were held back until the score launch after theirs had gone out: the score kernel is
+// then ahead of them in the order the device takes its work in and has its SMs first, and they fill the SMs it leaves.
+cudaError_t flush_deferred(OverlapState* os, int* launches) {
+  cudaError_t e = cudaSuccess;
+  for (size_t i = 0; i < os->deferred.size() && e == cudaSuccess; ++i)
+    e = enqueue_tail(os, os->deferred[i], true, true, launches, true);
+  os->deferred.clear();
+  return e;
+}
+
 // Launches the score kernel for the first n queued layers (pass 1) together with pass 2 of the pending layer and of
 // all but the last of them -- of all of them when `finish` is set -- then the selections and gathers of the
 // layers whose votes that gives.
@@ -343,6 +362,7 @@ cudaError_t launch_queue(OverlapState* os, int n, bool finish, int* launches) {
     // a single layer and nothing to pair it with: both passes in the single-layer kernel
     const PendingCall& c = os->queue[0];
     cudaError_t e1 = launch_score_tensor(c.pb, c.cu_host.data(), c.status, c.pb.lse_opt ? 2 : 3, c.st, launches);
+    if (e1 == cudaSuccess) e1 = flush_deferred(os, launches);
     if (e1 == cudaSuccess) e1 = enqueue_tail(os, c, false, true, launches);
     os->queue.clear();
     return e1;
@@ -352,9 +372,21 @@ cudaError_t launch_queue(OverlapState* os, int n, bool finish, int* launches) {
   cudaStream_t st = n > 0 ? os->queue[0].st : os->pending.st;
   // layers that came with their row statistics need the vote pass only (a queue holds one kind: see compress_impl)
   const bool votes_only = n > 0 && os->queue[0].pb.lse_opt != nullptr;
+  const bool more_follow = !finish;                  // a full list went out because one more layer has come
   if (votes_only) finish = true;
   cudaError_t e = launch_score_pipe(os->pending.valid ? &os->pending.plan : nullptr, plans, n, finish, votes_only, st,
                                     launches);
+  if (votes_only && more_follow) {
+    // An ordinary launch takes the SMs that are free when it starts: selections that became ready at the same moment
+    // would take a third of them for their 26 µs.  So this launch's selections and gathers are held back until the
+    // next score launch is out (or a join), and the ones held back at the launch before go out now, behind this one.
+    for (int i = 0; i < n && e == cudaSuccess; ++i) e = cudaEventRecord(os->scored[os->queue[i].slot], st);
+    if (e == cudaSuccess) e = flush_deferred(os, launches);
+    for (int i = 0; i < n && e == cudaSuccess; ++i) os->deferred.push_back(os->queue[i]);
+    os->queue.erase(os->queue.begin(), os->queue.begin() + n);
+    return e;
+  }
+  if (e == cudaSuccess) e = flush_deferred(os, launches);
   if (e == cudaSuccess && os->pending.valid) e = enqueue_tail(os, os->pending, true, finish, launches);
   os->pending.valid = false;
   const int n_voted = finish ? n : n - 1;
@@ -368,6 +400,7 @@ cudaError_t flush_pending(OverlapState* os, int* launches) {
   while (!os->queue.empty() && (int)os->queue.size() > kPipeMaxLayers && e == cudaSuccess)
     e = launch_queue(os, kPipeMaxLayers, false, launches);
   if (e == cudaSuccess) e = launch_queue(os, (int)os->queue.size(), true, launches);
+  if (e == cudaSuccess) e = flush_deferred(os, launches);
   return e;
 }
 
@@ -470,7 +503,7 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
       e = flush_pending(os, &launches);
       if (e != cudaSuccess) return cuda_fail(e);
     }
-    e = claim_slot(os, slot, st);
+    e = claim_slot(os, slot, st, &launches);
     if (e != cudaSuccess) return cuda_fail(e);
     if (pipe) {
       // Queue the layer; the score kernel takes a list of layers per launch (pass 1 of each beside pass 2 of the

@@ -498,7 +498,10 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   const uint32_t tmem_base = tmem_base_sh;
   ca.tmem0 = tmem_base;
   cb.tmem0 = tmem_base + 256;
-  pdl_launch_dependents();
+  // With both streams on the vote pass the launch behind this one is another of its kind, and none of its CTAs fits
+  // on an SM this launch holds: released now they would only sit on the SMs left to the selection kernels until this
+  // launch ends.  They are released when this CTA is done instead.
+  if (!DUAL) pdl_launch_dependents();
 
   // Stream A reads its layers' Q and K for the first time and overwrites row statistics an earlier launch may still
   // be merging: all its roles wait for the work before this launch.  Stream B's loads and MMAs need only Q and K,
@@ -538,6 +541,7 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
 
   tc_fence_before();
   __syncthreads();
+  if (DUAL) pdl_launch_dependents();
   if (abort_sh && tid == 0)
     for (int j = lay_lo; j <= lay_hi; ++j)
       if (pa.lay[j].status) atomicExch(pa.lay[j].status, (int)SLKV_ERR_DEVICE_TIMEOUT);
@@ -677,8 +681,18 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
     cfg.blockDim = dim3(kPipeThreads);
     cfg.dynamicSmemBytes = kPipeSmem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[3];
     int n = 0;
+    {
+      // ahead of the selections and gathers that become ready at the same moment on the side streams: when SMs
+      // come free, this kernel's CTAs are placed first
+      int least = 0, greatest = 0;
+      if (cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess && greatest != least) {
+        attr[n].id = cudaLaunchAttributePriority;
+        attr[n].val.priority = greatest;
+        ++n;
+      }
+    }
     if (waits_inside) {
       attr[n].id = cudaLaunchAttributeCooperative;
       attr[n].val.cooperative = 1;

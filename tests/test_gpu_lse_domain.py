@@ -127,18 +127,22 @@ def overlapped_layers(xs, cu, buds, w, p, domain=B.SLKV_HISTORY, lses=None, want
     return res
 
 
-@pytest.mark.parametrize("n_layers", [1, 2, 5, 11])
+@pytest.mark.parametrize("n_layers", [1, 2, 5, 11, 43])
 def test_overlapped_calls_with_supplied_lse(n_layers):
-    # every layer comes with its row statistics: the list kernel runs the vote pass on both of its streams
+    # every layer comes with its row statistics: the list kernel runs the vote pass on both of its streams.  The
+    # selections of a full list are held back until the next list is out; 43 layers take every workspace slot more
+    # than twice while some are held back (inputs cycle through 6 cases, the budgets differ per layer).
     w, p, lens = 32, 7, [1500, 700]
-    xs, buds, lses, refs = [], [], [], []
-    for i in range(n_layers):
-        q, k, v, cu = rand_case(8, 2, w, lens, seed=100 + i, scale=1.2)
-        xs.append((q, k, v))
-        buds.append([w + 10 + 17 * i, 300])
-        dom = "all_causal" if i % 2 else "history"
-        lses.append(O.row_lse(P.to_np64(q), P.to_np64(k), cu, w, dom))
-        refs.append(P.oracle_pooled(q, k, cu, w, p, domain=B.SLKV_ALL_CAUSAL if i % 2 else B.SLKV_HISTORY))
+    cases = []
+    for c in range(min(n_layers, 6)):
+        q, k, v, cu = rand_case(8, 2, w, lens, seed=100 + c, scale=1.2)
+        dom = "all_causal" if c % 2 else "history"
+        cases.append((q, k, v, O.row_lse(P.to_np64(q), P.to_np64(k), cu, w, dom),
+                      P.oracle_pooled(q, k, cu, w, p, domain=B.SLKV_ALL_CAUSAL if c % 2 else B.SLKV_HISTORY)))
+    xs = [cases[i % len(cases)][:3] for i in range(n_layers)]
+    lses = [cases[i % len(cases)][3] for i in range(n_layers)]
+    refs = [cases[i % len(cases)][4] for i in range(n_layers)]
+    buds = [[w + 10 + 17 * i, 300 + i] for i in range(n_layers)]
     res = overlapped_layers(xs, cu, buds, w, p, lses=lses)
     for i, gpu in enumerate(res):
         assert gpu["status"] == 0
