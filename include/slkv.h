@@ -244,12 +244,20 @@ int slkv_compress(const slkv_params* p, const void* q_win, const void* k, const 
  *     consume outputs, or free / overwrite any input, output or workspace buffer -- q_win, k, v, cu_seqlens_dev
  *     and budgets included -- only behind it.  cu_seqlens_host is read during the call only.  Any other slkv_*
  *     call that uses a workspace joins by itself first.
+ *   - Streams and host threads: the calls made on one stream form one sequence (queue, workspace slots, events);
+ *     calls made on another stream -- by another host thread or the same one -- form another, and the two do not
+ *     disturb each other as long as each has its own workspace (calls on two streams that share a workspace are
+ *     serialised: the later one waits for what the other stream has in flight).  A join orders its stream behind
+ *     the calls of every stream but settles only its own stream's: each stream that consumes results joins for
+ *     itself.  The entry points may be called from several host threads at once (one lock inside); up to eight
+ *     streams per device keep a sequence each, a ninth takes over the one used longest ago once that one's
+ *     stream has been made to wait for what it had in flight.
  *   - workspace must hold slkv_workspace_bytes_overlapped: votes, source-row lists and row statistics for up to
  *     eighteen layers in flight (77 MB for 8 KV heads x 32k keys; three layers' worth for shapes the list kernel
  *     does not take).  Successive calls share one workspace; a call with another shape or workspace first drains
  *     what is in flight.  q_win, k, v, budgets and the outputs of calls that may be in flight together must not
  *     alias each other's outputs.
- *   - The first call on a device creates eighteen side streams and 54 events (no device memory).
+ *   - The first call on a stream creates eighteen side streams and 54 events for it (no device memory).
  *   - The call sequence is stream-ordered and allocates nothing, so a step's calls plus the join can be captured
  *     in a CUDA graph (the side streams fork from and rejoin `stream`).
  *   - The list kernel takes bf16, head_dim 128, (n_q_heads / n_kv_heads) * window <= 128 and a multiple of 32,

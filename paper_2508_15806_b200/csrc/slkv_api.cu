@@ -266,17 +266,67 @@ struct OverlapState {
   std::vector<PendingCall> deferred;     // votes launched and `scored` recorded, selection and gather not enqueued yet
   ShapeSig sig;
 };
+// One state per (device, caller's stream): calls made on different streams (by different host threads, or by one)
+// never share a queue, a slot or an event, so each stream's calls keep their own order whatever the others do.
 constexpr int kMaxDevices = 64;
-OverlapState g_overlap[kMaxDevices];
+constexpr int kStatesPerDevice = 8;
+struct DeviceStates {
+  OverlapState st[kStatesPerDevice];
+  cudaStream_t owner[kStatesPerDevice] = {};
+  bool used[kStatesPerDevice] = {};
+  unsigned long long last_use[kStatesPerDevice] = {};
+  unsigned long long tick = 0;
+};
+DeviceStates g_overlap[kMaxDevices];
 std::mutex g_overlap_mu;
 constexpr int kSelectSmReserve = 16;              // SMs left to the selection kernels of the layers before
 
-cudaError_t overlap_state(OverlapState** out) {
+cudaError_t flush_pending(OverlapState* os, int* launches);
+
+bool state_idle(const OverlapState& s) {
+  if (!s.queue.empty() || s.pending.valid || !s.deferred.empty()) return false;
+  for (int h = 0; h < kSlots; ++h)
+    if (s.in_flight[h]) return false;
+  return true;
+}
+
+// The state of overlapped calls made on `st` on the current device (g_overlap_mu held).  All eight in use by other
+// streams: the one used longest ago is drained -- its queued layers go out and its own stream waits for what it has
+// in flight, as a join on that stream would -- and handed over.
+cudaError_t overlap_state(cudaStream_t st, OverlapState** out, int* launches) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  OverlapState& s = g_overlap[dev];
+  DeviceStates& d = g_overlap[dev];
+  int idx = -1;
+  for (int i = 0; i < kStatesPerDevice; ++i)
+    if (d.used[i] && d.owner[i] == st) idx = i;
+  if (idx < 0) {
+    for (int i = 0; i < kStatesPerDevice && idx < 0; ++i)
+      if (!d.used[i]) idx = i;
+    if (idx < 0) {
+      int oldest = 0, oldest_idle = -1;
+      for (int i = 0; i < kStatesPerDevice; ++i) {
+        if (d.last_use[i] < d.last_use[oldest]) oldest = i;
+        if (state_idle(d.st[i]) && (oldest_idle < 0 || d.last_use[i] < d.last_use[oldest_idle])) oldest_idle = i;
+      }
+      idx = oldest_idle >= 0 ? oldest_idle : oldest;
+      OverlapState& v = d.st[idx];
+      e = flush_pending(&v, launches);
+      for (int h = 0; h < kSlots && e == cudaSuccess; ++h)
+        if (v.in_flight[h]) {
+          e = cudaStreamWaitEvent(d.owner[idx], v.done[h], 0);
+          v.in_flight[h] = false;
+        }
+      if (e != cudaSuccess) return e;
+      v.sig = ShapeSig();
+    }
+    d.used[idx] = true;
+    d.owner[idx] = st;
+  }
+  d.last_use[idx] = ++d.tick;
+  OverlapState& s = d.st[idx];
   if (!s.side_gather[kSideStreams - 1]) {
     for (int i = 0; i < kSideStreams; ++i) {
       e = cudaStreamCreateWithFlags(&s.side_select[i], cudaStreamNonBlocking);
@@ -404,22 +454,49 @@ cudaError_t flush_pending(OverlapState* os, int* launches) {
   return e;
 }
 
-// Makes `st` wait for every overlapped call still in flight on this device (no host wait).
+// Calls on other streams whose workspace overlaps [ws, ws + bytes): their queued layers go out and `st` waits for what
+// they have in flight, before a call on `st` carves that memory up for itself (g_overlap_mu held).
+cudaError_t drain_states_sharing(const OverlapState* mine, const void* ws, size_t bytes, cudaStream_t st, int* launches) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  DeviceStates& d = g_overlap[dev];
+  const char* lo = static_cast<const char*>(ws);
+  for (int i = 0; i < kStatesPerDevice; ++i) {
+    OverlapState& s = d.st[i];
+    if (!d.used[i] || &s == mine || !s.sig.ws || state_idle(s)) continue;
+    const char* olo = static_cast<const char*>(s.sig.ws);
+    if (olo + s.sig.ws_bytes <= lo || lo + bytes <= olo) continue;
+    e = flush_pending(&s, launches);
+    for (int h = 0; h < kSlots && e == cudaSuccess; ++h)
+      if (s.in_flight[h]) e = cudaStreamWaitEvent(st, s.done[h], 0);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+// Makes `st` wait for every overlapped call still in flight on this device, whatever stream it was made on (no host
+// wait).  Only the calls made on `st` itself are then forgotten: the others stay in flight for a join on their own
+// stream, which still has to be ordered behind them.
 cudaError_t join_overlapped(cudaStream_t st, int* launches) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaSuccess;
   std::lock_guard<std::mutex> lock(g_overlap_mu);
-  OverlapState& s = g_overlap[dev];
-  e = flush_pending(&s, launches);
-  if (e != cudaSuccess) return e;
-  for (int h = 0; h < kSlots; ++h)
-    if (s.in_flight[h]) {
-      e = cudaStreamWaitEvent(st, s.done[h], 0);
-      if (e != cudaSuccess) return e;
-      s.in_flight[h] = false;
-    }
+  DeviceStates& d = g_overlap[dev];
+  for (int i = 0; i < kStatesPerDevice; ++i) {
+    if (!d.used[i]) continue;
+    OverlapState& s = d.st[i];
+    e = flush_pending(&s, launches);
+    if (e != cudaSuccess) return e;
+    for (int h = 0; h < kSlots; ++h)
+      if (s.in_flight[h]) {
+        e = cudaStreamWaitEvent(st, s.done[h], 0);
+        if (e != cudaSuccess) return e;
+        if (d.owner[i] == st) s.in_flight[h] = false;
+      }
+  }
   return cudaSuccess;
 }
 
@@ -455,7 +532,9 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
   if (overlapped) {
     std::lock_guard<std::mutex> lock(g_overlap_mu);
     OverlapState* os = nullptr;
-    e = overlap_state(&os);
+    e = overlap_state(st, &os, &launches);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = drain_states_sharing(os, ws, ws_bytes, st, &launches);
     if (e != cudaSuccess) return cuda_fail(e);
     ShapeSig sig;
     sig.ws = ws; sig.ws_bytes = ws_bytes; sig.n_seqs = pb.p.n_seqs; sig.n_kv_heads = pb.p.n_kv_heads; sig.R = pb.R;
