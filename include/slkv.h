@@ -8,6 +8,7 @@
  *   slkv_compress        score -> top-(C - window) history rows + window, gather (Sec. 3.4, Eq. 8, Algorithm 3)
  *   slkv_compress_host   the same, from/to host buffers (copies included)
  *   slkv_compress_overlapped / slkv_join   the same, successive layers overlapped on the GPU
+ *   slkv_cp_*            the same for one sequence whose keys are split over ranks (context parallel)
  *   slkv_row_lse         the window rows' log-sum-exp over their softmax domain       (Eq. 3-4, Eq. 7)
  *
  * Conventions
@@ -86,7 +87,11 @@ typedef struct slkv_params {
   int32_t softmax_domain;  /* SLKV_HISTORY | SLKV_ALL_CAUSAL: the keys a window row's softmax runs over */
   int32_t score_path;      /* SLKV_PATH_AUTO picks TENSOR when the shape allows it, else SIMT */
   int32_t lse_units;       /* SLKV_LSE_LN | SLKV_LSE_LOG2: units of lse_opt / slkv_row_lse's output */
-  int32_t reserved;        /* must be 0 */
+  int32_t history_only;    /* 0: the last `window` rows of every sequence in K / V are the window rows (never scored);
+                              1: K holds history rows only -- a range of a longer sequence's keys whose window rows
+                              live elsewhere (context-parallel sharding).  n_seqs must be 1; taken by slkv_score,
+                              slkv_row_lse and slkv_score_noalloc, SLKV_ERR_BAD_SHAPE from the compress entry points;
+                              the softmax then runs over the rows given, whatever softmax_domain says */
   int64_t k_stride_tok, k_stride_head;
   int64_t v_stride_tok, v_stride_head;
   int64_t q_stride_seq, q_stride_row, q_stride_head;
@@ -275,6 +280,53 @@ size_t slkv_workspace_bytes_overlapped(const slkv_params* p, const int32_t* cu_s
 /* Enqueues the layers still queued by slkv_compress_overlapped and orders `stream` after every overlapped call made
  * so far on the current device (see above). */
 int slkv_join(void* stream);
+
+/*
+ * Context-parallel compression of ONE long sequence whose history keys are split over ranks (Sec. 3.4, Eq. 7-8;
+ * Algorithm 3; same kept set as slkv_compress on the whole sequence, up to the score tolerance).
+ *
+ * Rank r of n_parts holds K / V rows of a contiguous range of history positions [b_r, e_r) plus up to pool_kernel/2
+ * rows of each neighbour's range on either side (so that pooling needs nothing from the neighbours); the last rank
+ * also holds the `window` rows behind the history.  Every rank holds q_win.  Per layer, on every rank:
+ *   1. slkv_row_lse over the rows it OWNS (history_only = 1 on all ranks but the last, whose range is an ordinary
+ *      sequence tail): the rows' log-sum-exp over this rank's keys.            all-gather over ranks
+ *   2. slkv_cp_merge_lse: log-sum-exp over the ranks = the rows' log-sum-exp over all keys.
+ *   3. slkv_score with lse_opt = that, over the owned rows plus the neighbours' margins: pooled scores.
+ *   4. slkv_cp_select_init once, then for level = 0, 1, 2: slkv_cp_histogram over the owned positions,
+ *      all-reduce (sum) of the histograms over ranks, slkv_cp_descend on the sum.  prefix[] then holds the bit
+ *      pattern of every head's threshold score, need[] how many positions with exactly that score are kept.
+ *   5. slkv_cp_local_ties (from the rank's OWN level-2 histogram): all-gather over ranks; slkv_cp_emit packs the
+ *      rank's kept rows (the ties go to the lowest positions, i.e. in rank order) and its window rows.
+ * The packed cache of head h is the concatenation over ranks of each rank's rows of head h; offsets[] are local.
+ * The collectives (two all-gathers of a few hundred bytes and three all-reduces of n_kv_heads x 2048 int32 per layer)
+ * are the caller's: the library launches no communication.  Everything is enqueued on `stream`; all pointers are
+ * device pointers unless stated.
+ *   lse_parts  [n_parts][n_q_heads][window] in p->lse_units (-inf for a rank without keys); lse_out [n_q_heads][window]
+ *   prefix, need, ties  [n_kv_heads]; hist  [n_kv_heads][2048] int32 (zeroed by slkv_cp_histogram)
+ *   pooled     [n_kv_heads][row_stride]: slkv_score's output for this rank's rows; the owned positions are
+ *              own_begin .. own_begin + own_count - 1 of every row (the margins before and after them are not owned)
+ *   pos0       position in the whole sequence of the first owned row
+ *   rows       rows of k / v on this rank; row j of k / v is position j of pooled; window_rows = 0, or on the last rank
+ *              the number of window rows, which are the last window_rows rows of k / v at positions window_pos0 ..
+ *   ties_all   [n_parts][n_kv_heads]: every rank's slkv_cp_local_ties; part = this rank's index
+ *   offsets    out, int32[n_kv_heads + 1]; kept_idx out, positions in the whole sequence; k_out, v_out as slkv_compress
+ *   status     optional: SLKV_ERR_CAPACITY if offsets[n_kv_heads] > out_capacity_rows
+ */
+int slkv_cp_merge_lse(const slkv_params* p, const float* lse_parts, int32_t n_parts, float* lse_out, void* stream);
+int slkv_cp_select_init(const int32_t* budgets, int32_t n_kv_heads, int32_t window, int64_t seq_len, uint32_t* prefix,
+                        int32_t* need, void* stream);
+int slkv_cp_histogram(const float* pooled, int32_t n_kv_heads, int64_t row_stride, int32_t own_begin, int32_t own_count,
+                      int32_t level, const uint32_t* prefix, int32_t* hist, void* stream);
+int slkv_cp_descend(const int32_t* hist, int32_t n_kv_heads, int32_t level, uint32_t* prefix, int32_t* need,
+                    void* stream);
+int slkv_cp_local_ties(const int32_t* hist_local, const uint32_t* prefix, int32_t n_kv_heads, int32_t* ties,
+                       void* stream);
+size_t slkv_cp_workspace_bytes(int32_t n_kv_heads, int64_t out_capacity_rows);
+int slkv_cp_emit(const slkv_params* p, const void* k, const void* v, int64_t rows, const float* pooled,
+                 int64_t row_stride, int32_t own_begin, int32_t own_count, int64_t pos0, const uint32_t* threshold,
+                 const int32_t* need, const int32_t* ties_all, int32_t n_parts, int32_t part, int32_t window_rows,
+                 int64_t window_pos0, void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets,
+                 int32_t* kept_idx, int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Bytes of device arena slkv_compress_host needs (inputs, outputs and workspace; 0 on invalid arguments). */
 size_t slkv_compress_host_arena_bytes(const slkv_params* p, const int32_t* cu_seqlens_host,

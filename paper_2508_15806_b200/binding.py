@@ -27,7 +27,7 @@ SLKV_PATH_AUTO, SLKV_PATH_SIMT, SLKV_PATH_TENSOR = 0, 1, 2
 class SlkvParams(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_seqs", "n_q_heads", "n_kv_heads", "head_dim", "window", "pool_kernel",
                                          "dtype", "pool_mode", "softmax_domain", "score_path", "lse_units",
-                                         "reserved")] + \
+                                         "history_only")] + \
                [(n, C.c_int64) for n in ("k_stride_tok", "k_stride_head", "v_stride_tok", "v_stride_head",
                                          "q_stride_seq", "q_stride_row", "q_stride_head")]
 
@@ -111,6 +111,22 @@ def lib() -> C.CDLL:
         L.slkv_kernel_count.restype = C.c_int
         L.slkv_trace_set_buffer.restype = C.c_int
         L.slkv_trace_set_buffer.argtypes = [C.c_void_p, C.c_size_t]
+        i32 = C.c_int32
+        L.slkv_cp_merge_lse.restype = C.c_int
+        L.slkv_cp_merge_lse.argtypes = [pp, vp, i32, vp, vp]
+        L.slkv_cp_select_init.restype = C.c_int
+        L.slkv_cp_select_init.argtypes = [vp, i32, i32, i64, vp, vp, vp]
+        L.slkv_cp_histogram.restype = C.c_int
+        L.slkv_cp_histogram.argtypes = [vp, i32, i64, i32, i32, i32, vp, vp, vp]
+        L.slkv_cp_descend.restype = C.c_int
+        L.slkv_cp_descend.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.slkv_cp_local_ties.restype = C.c_int
+        L.slkv_cp_local_ties.argtypes = [vp, vp, i32, vp, vp]
+        L.slkv_cp_workspace_bytes.restype = sz
+        L.slkv_cp_workspace_bytes.argtypes = [i32, i64]
+        L.slkv_cp_emit.restype = C.c_int
+        L.slkv_cp_emit.argtypes = [pp, vp, vp, i64, vp, i64, i32, i32, i64, vp, vp, vp, i32, i32, i32, i64, vp, vp, i64,
+                                   vp, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -140,7 +156,7 @@ def make_params(q_win: torch.Tensor, k: torch.Tensor, v: Optional[torch.Tensor],
     assert q_win.dtype == k.dtype == v.dtype
     return SlkvParams(n_seqs=q_win.shape[0], n_q_heads=q_win.shape[2], n_kv_heads=k.shape[1], head_dim=k.shape[2],
                       window=window, pool_kernel=pool_kernel, dtype=dt, pool_mode=pool_mode,
-                      softmax_domain=softmax_domain, score_path=score_path, lse_units=lse_units, reserved=0,
+                      softmax_domain=softmax_domain, score_path=score_path, lse_units=lse_units, history_only=0,
                       k_stride_tok=k.stride(0), k_stride_head=k.stride(1),
                       v_stride_tok=v.stride(0), v_stride_head=v.stride(1),
                       q_stride_seq=q_win.stride(0), q_stride_row=q_win.stride(1), q_stride_head=q_win.stride(2))
@@ -342,3 +358,57 @@ def slkv_trace_set_buffer(buf: Optional[torch.Tensor]) -> None:
         lib().slkv_trace_set_buffer(None, 0)
     else:
         lib().slkv_trace_set_buffer(buf.data_ptr(), buf.numel() * buf.element_size())
+
+
+# ---- context-parallel selection (one sequence's keys split over ranks): thin wrappers, see include/slkv.h ------------
+def _check(rc: int, what: str) -> None:
+    if rc != SLKV_OK:
+        raise SlkvError(rc, what)
+
+
+def slkv_cp_merge_lse(params: SlkvParams, lse_parts: torch.Tensor, lse_out: torch.Tensor, stream=None) -> torch.Tensor:
+    """lse_parts: CUDA float32 [n_parts, n_q_heads, window] (contiguous); lse_out: [1, n_q_heads, window]."""
+    _check(lib().slkv_cp_merge_lse(C.byref(params), lse_parts.data_ptr(), int(lse_parts.shape[0]), lse_out.data_ptr(),
+                                   _stream(stream)), "slkv_cp_merge_lse")
+    return lse_out
+
+
+def slkv_cp_select_init(budgets: torch.Tensor, window: int, seq_len: int, prefix: torch.Tensor, need: torch.Tensor,
+                        stream=None) -> None:
+    _check(lib().slkv_cp_select_init(budgets.data_ptr(), int(budgets.numel()), int(window), int(seq_len),
+                                     prefix.data_ptr(), need.data_ptr(), _stream(stream)), "slkv_cp_select_init")
+
+
+def slkv_cp_histogram(pooled: torch.Tensor, n_kv_heads: int, row_stride: int, own_begin: int, own_count: int, level: int,
+                      prefix: torch.Tensor, hist: torch.Tensor, stream=None) -> torch.Tensor:
+    _check(lib().slkv_cp_histogram(pooled.data_ptr(), int(n_kv_heads), int(row_stride), int(own_begin), int(own_count),
+                                   int(level), prefix.data_ptr(), hist.data_ptr(), _stream(stream)), "slkv_cp_histogram")
+    return hist
+
+
+def slkv_cp_descend(hist: torch.Tensor, level: int, prefix: torch.Tensor, need: torch.Tensor, stream=None) -> None:
+    _check(lib().slkv_cp_descend(hist.data_ptr(), int(prefix.numel()), int(level), prefix.data_ptr(), need.data_ptr(),
+                                 _stream(stream)), "slkv_cp_descend")
+
+
+def slkv_cp_local_ties(hist_local: torch.Tensor, prefix: torch.Tensor, ties: torch.Tensor, stream=None) -> torch.Tensor:
+    _check(lib().slkv_cp_local_ties(hist_local.data_ptr(), prefix.data_ptr(), int(prefix.numel()), ties.data_ptr(),
+                                    _stream(stream)), "slkv_cp_local_ties")
+    return ties
+
+
+def slkv_cp_workspace_bytes(n_kv_heads: int, capacity_rows: int) -> int:
+    return int(lib().slkv_cp_workspace_bytes(int(n_kv_heads), int(capacity_rows)))
+
+
+def slkv_cp_emit(params: SlkvParams, k: torch.Tensor, v: torch.Tensor, rows: int, pooled: torch.Tensor, row_stride: int,
+                 own_begin: int, own_count: int, pos0: int, threshold: torch.Tensor, need: torch.Tensor,
+                 ties_all: torch.Tensor, part: int, window_rows: int, window_pos0: int, k_out: torch.Tensor,
+                 v_out: torch.Tensor, offsets: torch.Tensor, kept_idx: torch.Tensor, workspace: torch.Tensor,
+                 status: Optional[torch.Tensor] = None, stream=None) -> None:
+    _check(lib().slkv_cp_emit(C.byref(params), k.data_ptr(), v.data_ptr(), int(rows), pooled.data_ptr(), int(row_stride),
+                              int(own_begin), int(own_count), int(pos0), threshold.data_ptr(), need.data_ptr(),
+                              ties_all.data_ptr(), int(ties_all.shape[0]), int(part), int(window_rows), int(window_pos0),
+                              k_out.data_ptr(), v_out.data_ptr(), int(k_out.shape[0]), offsets.data_ptr(),
+                              kept_idx.data_ptr(), _ptr(status), workspace.data_ptr(), workspace.numel(),
+                              _stream(stream)), "slkv_cp_emit")

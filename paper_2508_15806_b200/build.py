@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libslkv.so")
 SOURCES = ["slkv_api.cu", "slkv_alloc.cu", "slkv_score_simt.cu", "slkv_score_tc.cu", "slkv_score_pipe.cu", "slkv_select.cu", "slkv_select_cluster.cu", "slkv_select_cta.cu",
-           "slkv_noalloc.cu", "slkv_behavior.cu"]
+           "slkv_noalloc.cu", "slkv_behavior.cu", "slkv_cp.cu"]
 
 
 def _nvcc() -> str:

@@ -54,7 +54,8 @@ int describe(const slkv_params* p, const int32_t* cu_host, Problem* pb) {
   if (p->pool_mode != SLKV_POOL_MAX && p->pool_mode != SLKV_POOL_AVG) return SLKV_ERR_BAD_DTYPE;
   if (p->softmax_domain != SLKV_HISTORY && p->softmax_domain != SLKV_ALL_CAUSAL) return SLKV_ERR_BAD_DTYPE;
   if (p->lse_units != SLKV_LSE_LN && p->lse_units != SLKV_LSE_LOG2) return SLKV_ERR_BAD_DTYPE;
-  if (p->reserved != 0) return SLKV_ERR_BAD_DTYPE;
+  if (p->history_only != 0 && p->history_only != 1) return SLKV_ERR_BAD_DTYPE;
+  if (p->history_only && p->n_seqs != 1) return SLKV_ERR_BAD_SHAPE;
   if (p->score_path < SLKV_PATH_AUTO || p->score_path > SLKV_PATH_TENSOR) return SLKV_ERR_BAD_DTYPE;
   if (p->n_seqs < 1 || p->n_seqs > (1 << 20)) return SLKV_ERR_BAD_SHAPE;
   if (p->n_kv_heads < 1 || p->n_kv_heads > 65535 || p->n_q_heads < p->n_kv_heads ||
@@ -73,6 +74,13 @@ int describe(const slkv_params* p, const int32_t* cu_host, Problem* pb) {
   for (int64_t s : strides)
     if ((s * elem) % 16 != 0) return SLKV_ERR_BAD_ALIGN;
   if (cu_host[0] != 0) return SLKV_ERR_BAD_SHAPE;
+  // History rows only: the kernels are told about a sequence of rows + window tokens whose last `window` rows they
+  // never read (the window rows are only ever read as keys by the all-causal window statistics, which such a call
+  // does not run); the K tensor map still ends at the rows that exist.
+  const int64_t rows_given = cu_host[p->n_seqs];
+  if (p->history_only && (cu_host[1] < 0 || (int64_t)cu_host[1] + p->window >= (1ll << 31))) return SLKV_ERR_BAD_SHAPE;
+  const int32_t cu_virtual[2] = {0, p->history_only ? cu_host[1] + p->window : 0};
+  if (p->history_only) cu_host = cu_virtual;
   int64_t total_hist = 0;
   int max_hist = 0;
   for (int s = 0; s < p->n_seqs; ++s) {
@@ -90,7 +98,11 @@ int describe(const slkv_params* p, const int32_t* cu_host, Problem* pb) {
   pb->R = pb->G * p->window;
   pb->elem = elem;
   pb->max_hist = max_hist;
-  pb->total_tokens = T;
+  pb->total_tokens = rows_given;
+  if (p->history_only) {
+    pb->p.softmax_domain = SLKV_HISTORY;
+    pb->cu_virtual[0] = cu_virtual[0]; pb->cu_virtual[1] = cu_virtual[1];
+  }
   pb->total_hist = total_hist;
   pb->n_seg = p->n_seqs * p->n_kv_heads;
   if (p->n_seqs <= kInlineSeqs) {
@@ -511,6 +523,7 @@ int compress_impl(const slkv_params* p, const void* q_win, const void* k, const 
   Problem pb;
   int rc = describe(p, cu_host, &pb);
   if (rc != SLKV_OK) return rc;
+  if (p->history_only) return SLKV_ERR_BAD_SHAPE;            // nothing to append behind the selected rows
   if (capacity < 0) return SLKV_ERR_CAPACITY;
   if (!aligned16(q_win) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out))
     return SLKV_ERR_BAD_ALIGN;
@@ -700,7 +713,7 @@ int slkv_profile_collect(float* total_ms, int32_t* launches, int32_t n_kernels) 
 const char* slkv_kernel_name(int kernel_id) {
   static const char* names[KID_COUNT] = {"k_setup", "k_score_lse", "k_score_vote", "k_pool", "k_select",
                                          "k_gather", "k_alloc", "k_score_fused", "k_score_pipe", "k_window_stats",
-                                         "k_merge_lse", "k_behavior"};
+                                         "k_merge_lse", "k_behavior", "k_cp"};
   return (kernel_id >= 0 && kernel_id < KID_COUNT) ? names[kernel_id] : "";
 }
 
@@ -713,7 +726,7 @@ int slkv_trace_set_buffer(void* dev_buf, size_t bytes) {
 
 int slkv_last_cuda_error(void) { return g_last_cuda_error; }
 int slkv_last_launch_count(void) { return g_last_launches; }
-int slkv_version(void) { return 200; }
+int slkv_version(void) { return 300; }
 
 int slkv_debug_expire_next_wait(int on) {
   expire_next_wait(on != 0);
@@ -730,6 +743,106 @@ int slkv_behavior_scores(const float* attn, int64_t n_rows, int32_t row_len, int
   cudaError_t e = launch_behavior(attn, row_stride, row_len, n_rows, needle_idx, n_needle, needle_stride, topk_idx,
                                   n_topk, topk_stride, sf_sc, lg_sc, inf_sc, (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e);
+  return SLKV_OK;
+}
+
+// ---- context-parallel selection (slkv_cp.cu) -----------------------------------------------------------------
+int slkv_cp_merge_lse(const slkv_params* p, const float* lse_parts, int32_t n_parts, float* lse_out, void* stream) {
+  if (!p || !lse_parts || !lse_out) return SLKV_ERR_NULL_PTR;
+  if (n_parts < 1 || n_parts > 4096 || p->n_seqs != 1 || p->n_q_heads < 1 || p->window < 1 || p->window > kMaxWindow)
+    return SLKV_ERR_BAD_SHAPE;
+  if (p->lse_units != SLKV_LSE_LN && p->lse_units != SLKV_LSE_LOG2) return SLKV_ERR_BAD_DTYPE;
+  int launches = 0;
+  const float to_log2 = p->lse_units == SLKV_LSE_LOG2 ? 1.0f : 1.4426950408889634f;
+  cudaError_t e = launch_cp_merge_lse(lse_parts, n_parts, (long long)p->n_q_heads * p->window, to_log2, lse_out,
+                                      (cudaStream_t)stream, &launches);
+  return e == cudaSuccess ? SLKV_OK : cuda_fail(e);
+}
+
+int slkv_cp_select_init(const int32_t* budgets, int32_t n_kv_heads, int32_t window, int64_t seq_len, uint32_t* prefix,
+                        int32_t* need, void* stream) {
+  if (!budgets || !prefix || !need) return SLKV_ERR_NULL_PTR;
+  if (n_kv_heads < 1 || n_kv_heads > 65535 || window < 1 || window > kMaxWindow || seq_len < 0 || seq_len >= (1ll << 31))
+    return SLKV_ERR_BAD_SHAPE;
+  int launches = 0;
+  cudaError_t e = launch_cp_need_init(budgets, n_kv_heads, window, seq_len, prefix, need, (cudaStream_t)stream, &launches);
+  return e == cudaSuccess ? SLKV_OK : cuda_fail(e);
+}
+
+int slkv_cp_histogram(const float* pooled, int32_t n_kv_heads, int64_t row_stride, int32_t own_begin, int32_t own_count,
+                      int32_t level, const uint32_t* prefix, int32_t* hist, void* stream) {
+  if (!pooled || !prefix || !hist) return SLKV_ERR_NULL_PTR;
+  if (n_kv_heads < 1 || n_kv_heads > 65535 || row_stride < 0 || own_begin < 0 || own_count < 0 ||
+      (int64_t)own_begin + own_count > row_stride || level < 0 || level > 2)
+    return SLKV_ERR_BAD_SHAPE;
+  int launches = 0;
+  cudaError_t e = launch_cp_histogram(pooled, n_kv_heads, row_stride, own_begin, own_count, level, prefix, hist,
+                                      (cudaStream_t)stream, &launches);
+  return e == cudaSuccess ? SLKV_OK : cuda_fail(e);
+}
+
+int slkv_cp_descend(const int32_t* hist, int32_t n_kv_heads, int32_t level, uint32_t* prefix, int32_t* need,
+                    void* stream) {
+  if (!hist || !prefix || !need) return SLKV_ERR_NULL_PTR;
+  if (n_kv_heads < 1 || n_kv_heads > 65535 || level < 0 || level > 2) return SLKV_ERR_BAD_SHAPE;
+  int launches = 0;
+  cudaError_t e = launch_cp_descend(hist, n_kv_heads, level, prefix, need, (cudaStream_t)stream, &launches);
+  return e == cudaSuccess ? SLKV_OK : cuda_fail(e);
+}
+
+int slkv_cp_local_ties(const int32_t* hist_local, const uint32_t* prefix, int32_t n_kv_heads, int32_t* ties,
+                       void* stream) {
+  if (!hist_local || !prefix || !ties) return SLKV_ERR_NULL_PTR;
+  if (n_kv_heads < 1 || n_kv_heads > 65535) return SLKV_ERR_BAD_SHAPE;
+  int launches = 0;
+  cudaError_t e = launch_cp_local_ties(hist_local, prefix, n_kv_heads, ties, (cudaStream_t)stream, &launches);
+  return e == cudaSuccess ? SLKV_OK : cuda_fail(e);
+}
+
+size_t slkv_cp_workspace_bytes(int32_t n_kv_heads, int64_t out_capacity_rows) {
+  if (n_kv_heads < 1 || out_capacity_rows < 0) return 0;
+  return align_up((size_t)out_capacity_rows * sizeof(int32_t)) + 2 * align_up((size_t)n_kv_heads * sizeof(int32_t));
+}
+
+int slkv_cp_emit(const slkv_params* p, const void* k, const void* v, int64_t rows, const float* pooled,
+                 int64_t row_stride, int32_t own_begin, int32_t own_count, int64_t pos0, const uint32_t* threshold,
+                 const int32_t* need, const int32_t* ties_all, int32_t n_parts, int32_t part, int32_t window_rows,
+                 int64_t window_pos0, void* k_out, void* v_out, int64_t out_capacity_rows, int32_t* offsets,
+                 int32_t* kept_idx, int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
+  g_last_launches = 0;
+  if (!p || !k || !v || !pooled || !threshold || !need || !ties_all || !k_out || !v_out || !offsets || !kept_idx)
+    return SLKV_ERR_NULL_PTR;
+  const int32_t cu1[2] = {0, (int32_t)(rows < (1ll << 31) && rows >= 0 ? rows : -1)};
+  Problem pb;
+  int rc = describe(p, cu1, &pb);                    // validates dtype, head counts, strides
+  if (rc != SLKV_OK) return rc;
+  if (n_parts < 1 || part < 0 || part >= n_parts || window_rows < 0 || window_rows > p->window || window_rows > rows ||
+      own_begin < 0 || own_count < 0 || (int64_t)own_begin + own_count > rows - window_rows ||
+      (int64_t)own_begin + own_count > row_stride || pos0 < 0 || pos0 + own_count >= (1ll << 31) || window_pos0 < 0 ||
+      window_pos0 + window_rows >= (1ll << 31))
+    return SLKV_ERR_BAD_SHAPE;
+  if (out_capacity_rows < 0) return SLKV_ERR_CAPACITY;
+  if (!aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out)) return SLKV_ERR_BAD_ALIGN;
+  const size_t need_ws = slkv_cp_workspace_bytes(p->n_kv_heads, out_capacity_rows);
+  if (!workspace || workspace_bytes < need_ws || reinterpret_cast<uintptr_t>(workspace) % kAlign != 0)
+    return SLKV_ERR_WORKSPACE;
+  char* w = static_cast<char*>(workspace);
+  int32_t* gather_src = reinterpret_cast<int32_t*>(w);
+  int32_t* rows_h = reinterpret_cast<int32_t*>(w + align_up((size_t)out_capacity_rows * sizeof(int32_t)));
+  int32_t* take_h = rows_h + align_up((size_t)p->n_kv_heads * sizeof(int32_t)) / sizeof(int32_t);
+  cudaStream_t st = (cudaStream_t)stream;
+  int launches = 0;
+  cudaError_t e = launch_cp_emit(pooled, row_stride, own_begin, own_count, pos0, threshold, need, ties_all,
+                                 p->n_kv_heads, part, window_rows, rows - window_rows, window_pos0, out_capacity_rows,
+                                 offsets, kept_idx, gather_src, rows_h, take_h, status, st, &launches);
+  if (e != cudaSuccess) return cuda_fail(e);
+  pb.total_tokens = rows;
+  pb.n_seg = p->n_kv_heads;
+  pb.k = k; pb.v = v;
+  pb.gather_src = gather_src;
+  e = launch_gather(pb, offsets, kept_idx, k_out, v_out, out_capacity_rows, st, &launches, 256);
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_last_launches = launches;
   return SLKV_OK;
 }
 
@@ -833,6 +946,7 @@ int score_impl(const slkv_params* p, const void* q_win, const void* k, const int
   pb.cu = cu_seqlens_dev; pb.q = q_win; pb.k = k; pb.v = nullptr;
   pb.tab.cu_ptr = cu_seqlens_dev;
   pb.lse_opt = lse_opt;
+  if (p->history_only) cu_seqlens_host = pb.cu_virtual;      // one sequence: the tables are inline, cu_seqlens_dev unread
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
   cudaError_t e = join_overlapped(st, &launches);  // the workspace may still serve an overlapped call
@@ -955,7 +1069,7 @@ int slkv_compress_host(const slkv_params* p, const void* q_win, const void* k, c
   Problem pb;
   int rc = describe(p, cu_seqlens_host, &pb);
   if (rc != SLKV_OK) return rc;
-  if (!dense_strides(*p)) return SLKV_ERR_BAD_SHAPE;
+  if (!dense_strides(*p) || p->history_only) return SLKV_ERR_BAD_SHAPE;
   if (out_capacity_rows < 0) return SLKV_ERR_CAPACITY;
   if (reinterpret_cast<uintptr_t>(arena) % kAlign != 0) return SLKV_ERR_BAD_ALIGN;
   HostArena A;

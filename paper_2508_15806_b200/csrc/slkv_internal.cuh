@@ -93,7 +93,8 @@ struct Problem {
   int R;                  // score rows per KV head = G * window
   int elem;               // bytes per element
   int max_hist;           // max_s n_hist_s
-  int64_t total_tokens;
+  int64_t total_tokens;   // rows of K / V that exist (the extent of the K tensor map)
+  int32_t cu_virtual[2];  // history_only: {0, rows + window}, the sequence the kernels are told about
   int64_t total_hist;     // sum_s n_hist_s
   int n_seg;              // n_seqs * n_kv_heads
   const int32_t* cu;      // dev
@@ -119,7 +120,7 @@ struct Problem {
 };
 
 // kernel ids for launch accounting / per-kernel timing
-enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_SCORE_PIPE, KID_WINDOW_STATS, KID_MERGE_LSE, KID_BEHAVIOR, KID_COUNT };
+enum KernelId { KID_SETUP = 0, KID_SCORE_LSE, KID_SCORE_VOTE, KID_POOL, KID_SELECT, KID_GATHER, KID_ALLOC, KID_SCORE_FUSED, KID_SCORE_PIPE, KID_WINDOW_STATS, KID_MERGE_LSE, KID_BEHAVIOR, KID_CP, KID_COUNT };
 
 // Brackets one kernel launch: counts it and, when per-kernel timing is on for this thread, records a
 // CUDA event pair around it on the launch stream.
@@ -139,6 +140,22 @@ cudaError_t launch_alloc(const float* inf, int n_layers, int n_heads, int fixed,
 cudaError_t launch_behavior(const float* attn, long long row_stride, int row_len, long long n_rows,
                             const int32_t* needle_idx, int n_needle, long long needle_stride, const int32_t* topk_idx,
                             int n_topk, long long topk_stride, float* sf, float* lg, float* inf, cudaStream_t st);
+// context-parallel selection (slkv_cp.cu)
+cudaError_t launch_cp_merge_lse(const float* parts, int n_parts, long long n, float to_log2, float* out,
+                                cudaStream_t st, int* launches);
+cudaError_t launch_cp_need_init(const int32_t* budgets, int n_kv_heads, int window, long long seq_len, unsigned* prefix,
+                                int32_t* need, cudaStream_t st, int* launches);
+cudaError_t launch_cp_histogram(const float* pooled, int n_kv_heads, long long row_stride, int own_begin, int own_count,
+                                int level, const unsigned* prefix, int32_t* hist, cudaStream_t st, int* launches);
+cudaError_t launch_cp_descend(const int32_t* hist, int n_kv_heads, int level, unsigned* prefix, int32_t* need,
+                              cudaStream_t st, int* launches);
+cudaError_t launch_cp_local_ties(const int32_t* hist_local, const unsigned* prefix, int n_kv_heads, int32_t* ties,
+                                 cudaStream_t st, int* launches);
+cudaError_t launch_cp_emit(const float* pooled, long long row_stride, int own_begin, int own_count, long long pos0,
+                           const unsigned* threshold, const int32_t* need, const int32_t* ties_all, int n_kv_heads,
+                           int part, int window_rows, long long window_row0, long long window_pos0, long long capacity,
+                           int32_t* offsets, int32_t* kept_idx, int32_t* gather_src, int32_t* rows, int32_t* take,
+                           int32_t* status, cudaStream_t st, int* launches);
 cudaError_t launch_setup(const Problem& pb, const int32_t* budgets, int32_t* offsets, int64_t capacity,
                          int32_t* status, cudaStream_t st, int* launches);
 int simt_chunk_keys();

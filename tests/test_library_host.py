@@ -35,7 +35,7 @@ def test_exports_every_declared_symbol(L):
 def params(**kw):
     d = dict(n_seqs=1, n_q_heads=8, n_kv_heads=2, head_dim=128, window=16, pool_kernel=5, dtype=B.SLKV_BF16,
              pool_mode=B.SLKV_POOL_MAX, softmax_domain=B.SLKV_HISTORY, score_path=B.SLKV_PATH_AUTO,
-             lse_units=B.SLKV_LSE_LN, reserved=0,
+             lse_units=B.SLKV_LSE_LN, history_only=0,
              k_stride_tok=256, k_stride_head=128, v_stride_tok=256, v_stride_head=128,
              q_stride_seq=16 * 8 * 128, q_stride_row=8 * 128, q_stride_head=128)
     d.update(kw)
@@ -64,7 +64,7 @@ def test_bad_enums_and_alignment(L):
     fake = C.c_void_p(4096)          # never dereferenced: validation fails first
     for kw, code in [(dict(dtype=7), "BAD_DTYPE"), (dict(pool_mode=3), "BAD_DTYPE"),
                      (dict(softmax_domain=2), "BAD_DTYPE"), (dict(score_path=9), "BAD_DTYPE"),
-                     (dict(lse_units=2), "BAD_DTYPE"), (dict(reserved=1), "BAD_DTYPE"),
+                     (dict(lse_units=2), "BAD_DTYPE"), (dict(history_only=2), "BAD_DTYPE"),
                      (dict(k_stride_tok=257), "BAD_ALIGN")]:
         p = params(**kw)
         rc = L.slkv_score(C.byref(p), fake, fake, fake, cu, None, fake, None, fake, 1 << 30, None)

@@ -70,7 +70,7 @@ def test_oversized_shapes_are_rejected_on_the_host():
     assert B.slkv_noalloc_scratch_bytes() == 8 << 20
     p = B.SlkvParams(n_seqs=1, n_q_heads=32, n_kv_heads=8, head_dim=128, window=32, pool_kernel=7, dtype=B.SLKV_BF16,
                      pool_mode=B.SLKV_POOL_MAX, softmax_domain=B.SLKV_HISTORY, score_path=B.SLKV_PATH_AUTO,
-                     lse_units=B.SLKV_LSE_LN, reserved=0, k_stride_tok=1024, k_stride_head=128, v_stride_tok=1024, v_stride_head=128,
+                     lse_units=B.SLKV_LSE_LN, history_only=0, k_stride_tok=1024, k_stride_head=128, v_stride_tok=1024, v_stride_head=128,
                      q_stride_seq=32 * 32 * 128, q_stride_row=32 * 128, q_stride_head=128)
     cu = (C.c_int32 * 2)(0, 131072)
     assert B.slkv_workspace_bytes(p, [0, 131072]) > B.slkv_noalloc_scratch_bytes()
