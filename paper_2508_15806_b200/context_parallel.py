@@ -43,9 +43,9 @@ class DistComm:
         self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
 
     def all_gather(self, t: torch.Tensor) -> torch.Tensor:
-        out = torch.empty((self.world,) + tuple(t.shape), dtype=t.dtype, device=t.device)
-        self._dist.all_gather_into_tensor(out, t.contiguous(), group=self._group)
-        return out
+        out = torch.empty(self.world * t.numel(), dtype=t.dtype, device=t.device)
+        self._dist.all_gather_into_tensor(out, t.contiguous().reshape(-1), group=self._group)
+        return out.reshape((self.world,) + tuple(t.shape))
 
     def all_reduce_sum(self, t: torch.Tensor) -> torch.Tensor:
         self._dist.all_reduce(t, op=self._dist.ReduceOp.SUM, group=self._group)

@@ -54,6 +54,25 @@ def test_config5_long_context_heavy_and_fixed_only_layers():
         assert stats["segments"] == 8 and stats["pooled_max_rel_err"] < 1e-3
 
 
+def test_config5_long_context_split_over_four_ranks():
+    # the 131072-token sequence with its history keys split over 4 ranks (emulated on this GPU, one host thread and
+    # stream per rank): the ranks' packed rows together against the oracle on the whole sequence
+    from test_gpu_context_parallel import as_one_layer, run_ranks
+    wl = synth.workloads()[4]
+    budgets = O.alloc_budgets(synth.inf_sc(wl).numpy(), wl.fixed, wl.totals[0])
+    layer = int(np.argmax((budgets > wl.total_tokens).sum(axis=1) * 10**9 + budgets.max(axis=1)))
+    x = synth.layer_inputs(wl, layer, device="cuda")
+    q, k, v = x.q_win.cpu(), x.k.cpu(), x.v.cpu()
+    bud = budgets[layer].tolist()
+    ref = P.oracle_pooled(q, k, wl.cu_seqlens, wl.window, wl.pool_kernel)
+    outs = run_ranks(4, q, k, v, bud, wl.window, wl.pool_kernel)
+    assert all(int(o["status"].item()) == 0 for o in outs)
+    gpu = as_one_layer(outs, 4, wl.total_tokens, wl.window, wl.pool_kernel, wl.n_kv_heads)
+    assert P.assert_pooled_close(gpu["pooled"], ref, wl.cu_seqlens, wl.n_kv_heads, wl.window) < 1e-3
+    stats = P.assert_selection_valid(gpu, ref, wl.cu_seqlens, bud, wl.window, k, v)
+    assert stats["segments"] == 8
+
+
 def test_config3_full_layers_through_the_overlapped_entry_point():
     # the launch configuration bench.py times: layers queued by slkv_compress_overlapped, the score kernel taking
     # them a list at a time (here 10 layers: a full list of 8, then the rest at the join).  Pooled scores and the

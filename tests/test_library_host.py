@@ -118,3 +118,38 @@ def test_compress_argument_errors(L):
                 v_stride_head=64, q_stride_head=64)
     bad = list(args); bad[0] = C.byref(pt)
     assert L.slkv_compress(*bad) == B.ERR["BAD_DTYPE"]      # the tensor path takes bf16 only
+
+
+def test_history_only_and_context_parallel_argument_errors(L):
+    fake = C.c_void_p(4096)
+    cu = (C.c_int32 * 2)(0, 100)
+    ph = params(history_only=1)
+    assert B.slkv_pooled_elems(ph, [0, 100]) == 2 * 100          # every row given is a history row
+    assert B.slkv_pooled_elems(params(), [0, 100]) == 2 * 84
+    assert B.slkv_workspace_bytes(params(history_only=1, n_seqs=2), [0, 50, 100]) == 0      # one sequence only
+    args = [C.byref(ph), fake, fake, fake, fake, cu, fake, None, fake, fake, 10, fake, fake, None, None, fake, 1 << 30,
+            None]
+    assert L.slkv_compress(*args) == B.ERR["BAD_SHAPE"]          # nothing to append behind the selected rows
+    assert L.slkv_compress_overlapped(*args) == B.ERR["BAD_SHAPE"]
+    p = params()
+    assert L.slkv_cp_merge_lse(C.byref(p), None, 2, fake, None) == B.ERR["NULL_PTR"]
+    assert L.slkv_cp_merge_lse(C.byref(p), fake, 0, fake, None) == B.ERR["BAD_SHAPE"]
+    assert L.slkv_cp_select_init(fake, 0, 16, 100, fake, fake, None) == B.ERR["BAD_SHAPE"]
+    assert L.slkv_cp_select_init(fake, 2, 16, 1 << 31, fake, fake, None) == B.ERR["BAD_SHAPE"]
+    assert L.slkv_cp_histogram(fake, 2, 100, 90, 20, 0, fake, fake, None) == B.ERR["BAD_SHAPE"]      # past the row
+    assert L.slkv_cp_histogram(fake, 2, 100, 0, 20, 3, fake, fake, None) == B.ERR["BAD_SHAPE"]
+    assert L.slkv_cp_descend(fake, 2, -1, fake, fake, None) == B.ERR["BAD_SHAPE"]
+    assert L.slkv_cp_local_ties(fake, None, 2, fake, None) == B.ERR["NULL_PTR"]
+    assert L.slkv_cp_workspace_bytes(2, 1000) >= 4000 and L.slkv_cp_workspace_bytes(0, 10) == 0
+    emit = [C.byref(p), fake, fake, 100, fake, 100, 0, 84, 0, fake, fake, fake, 2, 1, 16, 84, fake, fake, 200, fake, fake,
+            None, fake, 1 << 20, None]
+    bad = list(emit); bad[7] = 90                                 # owned rows run into the window rows
+    assert L.slkv_cp_emit(*bad) == B.ERR["BAD_SHAPE"]
+    bad = list(emit); bad[13] = 2                                 # part >= n_parts
+    assert L.slkv_cp_emit(*bad) == B.ERR["BAD_SHAPE"]
+    bad = list(emit); bad[18] = -1
+    assert L.slkv_cp_emit(*bad) == B.ERR["CAPACITY"]
+    bad = list(emit); bad[23] = 16
+    assert L.slkv_cp_emit(*bad) == B.ERR["WORKSPACE"]
+    bad = list(emit); bad[1] = None
+    assert L.slkv_cp_emit(*bad) == B.ERR["NULL_PTR"]
