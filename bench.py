@@ -580,6 +580,83 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+def run_context_parallel(args):
+    """`--context-parallel`: ONE long sequence (the 131072-token workload unless --workload says otherwise) with its
+    history keys split over the ranks; strong scaling.  The per-rank call sequence and its collectives (NCCL) are
+    paper_2508_15806_b200/context_parallel.py's; a step = every layer of the model once.  Not the headline: the
+    headline is the default run (independent sequence batches per rank, no collective)."""
+    import torch.distributed as dist
+    from paper_2508_15806_b200 import binding as B
+    from paper_2508_15806_b200 import context_parallel as CP
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29517")
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    comm = CP.DistComm()
+    wl = synth.workloads()[(args.workload - 1) if args.workload else 4]
+    assert len(wl.seq_lens) == 1, "context parallel splits one sequence"
+    total = wl.totals[0]
+    budgets = B.slkv_alloc_budgets(synth.inf_sc(wl).to(dev), wl.fixed, total)
+    n_distinct = min(args.layers or 4, wl.n_layers)       # distinct layers held; a step cycles through them n_layers times
+    shards = []
+    for l in range(n_distinct):
+        x = synth.layer_inputs(wl, l, device=dev)         # every rank draws the same layer and keeps its own rows
+        sh = CP.shard_of(x.q_win, x.k, x.v, wl.window, wl.pool_kernel, rank, world)
+        sh.k, sh.v = sh.k.clone(), sh.v.clone()
+        shards.append(sh)
+        del x
+    torch.cuda.empty_cache()
+
+    def step():
+        outs = None
+        for l in range(wl.n_layers):
+            outs = CP.compress_rank(shards[l % n_distinct], budgets[l].contiguous(), wl.pool_kernel, comm)
+        return outs
+
+    def barrier():
+        torch.cuda.synchronize()
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        outs = step()
+    torch.cuda.synchronize()
+    assert int(outs["status"].item()) == 0
+    steps = args.steps or 5
+    sampler = ClockSampler(local)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    a.record()
+    for _ in range(steps):
+        step()
+    b.record()
+    barrier()
+    sampler.stop()
+    ms = max_over_ranks(a.elapsed_time(b), dist, dev) / steps
+    if rank == 0:
+        print(json.dumps({
+            "metric": "context tokens compressed per second per layer", "unit": "tokens/s/layer",
+            "value": wl.total_tokens * wl.n_layers / (ms * 1e-3), "n_gpus": world, "steps": steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms, "us_per_layer": ms * 1e3 / wl.n_layers,
+            "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "n_layers": wl.n_layers, "seq_lens": wl.seq_lens, "window": wl.window,
+                       "parallelism": f"cp{world}: one sequence's history keys split over the ranks; per layer one "
+                                      "all-gather of row statistics, three all-reduces of radix histograms, one "
+                                      "all-gather of tie counts (NCCL)",
+                       "api": "context_parallel.compress_rank (slkv_row_lse, slkv_score, slkv_cp_*)",
+                       "l2": f"{n_distinct} distinct layers cycled; a rank's K and V are larger than L2 together"},
+            "clocks": sampler.summary(), "e2e": None, "gpu_launches": None, "roofline": None, "cpu_baseline": None}))
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -602,9 +679,13 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--e2e-layers", type=int, default=8, help="distinct layers kept in pinned host memory")
     ap.add_argument("--cpu-budget-s", type=float, default=20.0)
+    ap.add_argument("--context-parallel", action="store_true",
+                    help="split ONE long sequence's keys over the ranks (strong scaling, NCCL collectives); not the headline")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.context_parallel:
+        run_context_parallel(args)
     else:
         run_cuda(args)
 
