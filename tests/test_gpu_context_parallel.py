@@ -206,3 +206,37 @@ def test_selection_is_exact_on_given_scores_with_many_ties(seed):
         kh, nw = O.kept_counts(L, budgets[h], w)
         want = np.concatenate([O.select_topk(scores[h].astype(np.float64), kh), np.arange(L - nw, L)])
         assert np.array_equal(np.concatenate(kept[h]), want), (h, world, n_hist)
+
+
+@pytest.mark.parametrize("path,dtype,d,w,Hq,Hkv", [(B.SLKV_PATH_TENSOR, torch.bfloat16, 128, 32, 8, 2),
+                                                   (B.SLKV_PATH_SIMT, torch.float32, 64, 16, 8, 8)])
+def test_history_only_rows_score_as_the_history_of_a_longer_sequence(path, dtype, d, w, Hq, Hkv):
+    # K holds history rows only (history_only = 1): same votes, pooled scores and row log-sum-exps as the oracle gives
+    # for a sequence of those rows followed by `w` window rows (which the history-only softmax never reads as keys)
+    n, p = 1777, 5
+    q, k, _ = rand_seq(Hq, Hkv, w, n, seed=3, d=d, dtype=dtype)
+    k_padded = torch.cat([k, torch.zeros(w, Hkv, d, dtype=dtype)])
+    cu_pad = [0, n + w]
+    ref = P.oracle_pooled(q, k_padded, cu_pad, w, p)
+    ref_lse = O.row_lse(P.to_np64(q), P.to_np64(k_padded), cu_pad, w, "history")
+    qd, kd = q.to(DEV), k.to(DEV)
+    prm = B.make_params(qd, kd, None, w, p, B.SLKV_POOL_MAX, path)
+    prm.history_only = 1
+    cu = [0, n]
+    assert B.slkv_pooled_elems(prm, cu) == Hkv * n
+    ws = torch.empty(B.slkv_workspace_bytes(prm, cu), dtype=torch.uint8, device=DEV)
+    cu_dev = torch.tensor(cu, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    pooled = torch.full((Hkv * n,), float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.empty(1, Hq, w, dtype=torch.float32, device=DEV)
+    B.slkv_score(prm, qd, kd, cu_dev, cu, pooled, ws, status)
+    B.slkv_row_lse(prm, qd, kd, cu_dev, cu, lse, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    P.assert_pooled_close(pooled.cpu().numpy(), ref, cu_pad, Hkv, w)
+    assert np.allclose(lse.cpu().numpy().astype(np.float64), np.asarray(ref_lse).reshape(1, Hq, w), rtol=0, atol=2e-4)
+    # the same scores when the caller hands the log-sum-exps over
+    pooled2 = torch.full_like(pooled, float("nan"))
+    B.slkv_score(prm, qd, kd, cu_dev, cu, pooled2, ws, status, lse=lse)
+    torch.cuda.synchronize()
+    P.assert_pooled_close(pooled2.cpu().numpy(), ref, cu_pad, Hkv, w)
