@@ -31,12 +31,14 @@ namespace {
 
 constexpr int kPipeThreads = 640;        // warps 0-3: producer A, issuer A, producer B, issuer B;
                                          // warps 4-11: epilogue of stream A; warps 12-19: epilogue of stream B
+constexpr int kDualWgs = 3;               // vote pass on both streams: warpgroups per stream
+constexpr int kDualThreads = 128 + 2 * kDualWgs * 128;
 constexpr int kLeadEntries = 2;           // entries pass 1 may be ahead of the entry pass 2 has begun
 constexpr unsigned kPollNs = 64;          // pause between two polls of an mbarrier
 constexpr int kStagesA = 3;              // K tiles in flight from HBM
 constexpr int kStagesB = 2;              // K tiles in flight from L2
 constexpr int kQBytes = 2 * kHalfBytes;  // one 128-row Q tile
-constexpr int kBarBytesPerStream = 128;  // up to 16 mbarriers
+constexpr int kBarBytesPerStream = 160;  // up to 20 mbarriers
 constexpr int kPipeTail = 512 + 1024 + 1024;   // mbarriers + flags, stat_m/stat_z of stream A, two log-sum-exp rows of stream B
 constexpr int kPipeSmem = 2 * kQBytes + (kStagesA + kStagesB) * kStageBytes + kPipeTail;
 static_assert(kPipeSmem <= kSmemLimit, "shared memory of the two-stream kernel");
@@ -87,6 +89,9 @@ struct StreamCtx {
   __device__ __forceinline__ uint32_t full_bar(int st) const { return bar0 + 8u * st; }
   __device__ __forceinline__ uint32_t empty_bar(int st) const { return bar0 + 8u * (3 + st); }
   __device__ __forceinline__ uint32_t accf_bar(int b) const { return bar0 + 8u * (6 + b); }
+  // three warpgroups per stream: one barrier per (warpgroup, accumulator), so that a warpgroup sees every phase of the
+  // barriers it waits on (a parity wait tells only adjacent phases apart)
+  __device__ __forceinline__ uint32_t accf_bar_of(int wg, int b) const { return bar0 + 8u * (13 + 2 * wg + b); }
   __device__ __forceinline__ uint32_t acce_bar(int b) const { return bar0 + 8u * (8 + b); }
   __device__ __forceinline__ uint32_t qfull_bar() const { return bar0 + 8u * 10; }
   __device__ __forceinline__ uint32_t qempty_bar() const { return bar0 + 8u * 11; }
@@ -111,7 +116,9 @@ __device__ __forceinline__ void entry_range(const TcArgs& a, const LayerDesc& L,
   begin = min(L.tile_begin + (int)blockIdx.x * a.tiles_per_cta, L.tile_end);
   end = min(begin + a.tiles_per_cta, L.tile_end);
 }
-__device__ __forceinline__ void named_bar(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(kEpiThreads) : "memory"); }
+__device__ __forceinline__ void named_bar(int id, int n_threads = kEpiThreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
 
 // ---- one thread: TMA loads of the stream's Q tiles and K tiles ------------------------------------------
 template <bool VOTE>
@@ -175,7 +182,7 @@ __device__ __forceinline__ void producer(const StreamCtx& c, const TcArgs& a, co
 }
 
 // ---- one thread: the stream's MMAs, one 128 x 128 x 128 product per tile into one of two accumulators --------
-template <bool VOTE>
+template <bool VOTE, int NWG = 2>
 __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, const LayerDesc* lay, int first, int last,
                                        int step) {
   // pass 1: D[row, key] = Q K^T (A = Q, B = K); pass 2: D[key, row] = K Q^T (A = K, B = Q, N = R)
@@ -205,7 +212,7 @@ __device__ __forceinline__ void issuer(const StreamCtx& c, const TcArgs& a, cons
         else tc_mma(d0, q_desc0 + off, k_desc + off, idesc, ks > 0);
       }
       tc_commit(c.empty_bar(st));       // K stage free once these MMAs have read it
-      tc_commit(c.accf_bar(b));         // accumulator ready for the epilogue
+      tc_commit(NWG == 2 ? c.accf_bar(b) : c.accf_bar_of(it % NWG, b));   // accumulator ready for the epilogue
       k_desc += (uint64_t)(kStageBytes >> 4);
       if (++st == c.n_stages) { st = 0; st_phase ^= 1u; k_desc = k_desc0; }
       if (++b == 2) { b = 0; b_phase ^= 1u; }
@@ -329,9 +336,24 @@ __device__ __forceinline__ float vote_chunk(const uint32_t (&r)[32], float sc, c
   return (s0 + s1) + (s2 + s3);
 }
 
+// sum_e 2^(v_e * sc - lse_e) over 16 accumulator values
+__device__ __forceinline__ float vote_chunk16(const uint32_t (&r)[16], float sc, const float* lse) {
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < 16; e += 4) {
+    const float4 l4 = *reinterpret_cast<const float4*>(lse + e);
+    s0 += ex2(fmaf(__uint_as_float(r[e]), sc, -l4.x));
+    s1 += ex2(fmaf(__uint_as_float(r[e + 1]), sc, -l4.y));
+    s2 += ex2(fmaf(__uint_as_float(r[e + 2]), sc, -l4.z));
+    s3 += ex2(fmaf(__uint_as_float(r[e + 3]), sc, -l4.w));
+  }
+  return (s0 + s1) + (s2 + s3);
+}
+
 // ---- 256 threads: pass 2, votes (stream B) ---------------------------------------------------------------------
 // `first`, `last`, pa.step: the entries this stream takes; `bar_id`: the named barrier of its 256 threads; `is_b`: the
 // stream pass 1 of the same CTA keeps its distance to.
+template <int NWG>
 __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs& a, const PipeArgs& pa, int et, int warp,
                                                float* lse2, int first, int last, int bar_id, bool is_b) {
   const int wg = et >> 7, row = et & 127, lane = et & 31;
@@ -340,6 +362,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
   const float inv_g = 1.0f / (float)a.G;
   const int R = a.R;
   int it = 0, run_idx = 0;
+  int own0 = 0, own1 = 0;               // this warpgroup's tiles so far on either accumulator (three warpgroups)
   bool ok = true;
   for (int j = first; j <= last; j += pa.step) {
   const LayerDesc& L = pa.lay[j];
@@ -356,7 +379,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
         __nanosleep(64);
       }
     }
-    named_bar(bar_id);
+    named_bar(bar_id, NWG * 128);
     ok = ok && *c.abort_flag == 0;
   }
   if (et == 0 && is_b) *c.b_layer = j;
@@ -385,18 +408,23 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
       }
       if (half == 0 && rr >= 0) lse[rr] = l2;
     }
-    named_bar(bar_id);
+    named_bar(bar_id, NWG * 128);
     if (et == 0 && is_b && run_idx == 0) trace_mark(a.trace, 3);
     for (int i = 0; i < r.count; ++i, ++it) {
-      if ((it & 1) != wg) continue;
       const int b = it & 1;
-      if (ok) ok = mbar_wait(c.accf_bar(b), (it >> 1) & 1, c.abort_flag, kPollNs);
+      if (NWG == 2) {
+        if ((it & 1) != wg) continue;
+        if (ok) ok = mbar_wait(c.accf_bar(b), (it >> 1) & 1, c.abort_flag, kPollNs);
+      } else {
+        if (it % NWG != wg) continue;
+        const int mine = b ? own1++ : own0++;
+        if (ok) ok = mbar_wait(c.accf_bar_of(wg, b), mine & 1, c.abort_flag, kPollNs);
+      }
       ok = __all_sync(0xffffffffu, ok) != 0;
       if (!ok) continue;
       tc_fence_after();
       const int key0 = (r.t0 + i) * kTileKeys;
       const uint32_t tb = c.tmem0 + lane_sel + (uint32_t)(b * 128);
-      uint32_t ra[32], rb[32];
       float acc = 0.f;
       auto release = [&]() {
         // the accumulator is in registers: hand its TMEM buffer back before the arithmetic and the vote's store
@@ -404,17 +432,33 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
         __syncwarp();
         if (lane == 0) mbar_arrive(c.acce_bar(b));
       };
-      tc_ld32_issue(tb, ra);
+      if (NWG == 2) {
+        uint32_t ra[32], rb[32];
+        tc_ld32_issue(tb, ra);
 #pragma unroll 1
-      for (int c0 = 0; c0 < R; c0 += 64) {
-        tc_ld_wait(ra);
-        if (c0 + 32 < R) tc_ld32_issue(tb + c0 + 32, rb);
-        if (c0 + 32 >= R) release();
-        else if (c0 + 64 >= R) { tc_ld_wait(rb); release(); }
-        acc += vote_chunk(ra, sc, lse + c0);
-        if (c0 + 32 < R) {
-          if (c0 + 64 < R) { tc_ld_wait(rb); tc_ld32_issue(tb + c0 + 64, ra); }
-          acc += vote_chunk(rb, sc, lse + c0 + 32);
+        for (int c0 = 0; c0 < R; c0 += 64) {
+          tc_ld_wait(ra);
+          if (c0 + 32 < R) tc_ld32_issue(tb + c0 + 32, rb);
+          if (c0 + 32 >= R) release();
+          else if (c0 + 64 >= R) { tc_ld_wait(rb); release(); }
+          acc += vote_chunk(ra, sc, lse + c0);
+          if (c0 + 32 < R) {
+            if (c0 + 64 < R) { tc_ld_wait(rb); tc_ld32_issue(tb + c0 + 64, ra); }
+            acc += vote_chunk(rb, sc, lse + c0 + 32);
+          }
+        }
+      } else {
+        // three warpgroups per stream share the register file: rounds of 16 columns (R is a multiple of 32)
+        uint32_t ra[16], rb[16];
+        tc_ld16_issue(tb, ra);
+#pragma unroll 1
+        for (int c0 = 0; c0 < R; c0 += 32) {
+          tc_ld_wait16(ra);
+          tc_ld16_issue(tb + c0 + 16, rb);
+          acc += vote_chunk16(ra, sc, lse + c0);
+          tc_ld_wait16(rb);
+          if (c0 + 32 < R) tc_ld16_issue(tb + c0 + 32, ra); else release();
+          acc += vote_chunk16(rb, sc, lse + c0 + 16);
         }
       }
       const int jk = key0 + row;
@@ -428,7 +472,7 @@ __device__ __forceinline__ void epilogue_votes(const StreamCtx& c, const TcArgs&
 
 // DUAL: both streams run pass 2 (every layer of the list came with its row statistics), each on every other entry.
 template <bool DUAL>
-__global__ void __launch_bounds__(kPipeThreads, 1)
+__global__ void __launch_bounds__(DUAL ? kDualThreads : kPipeThreads, 1)
 k_score_pipe(const __grid_constant__ PipeArgs pa) {
   // Shared memory, all dynamic and 1024-byte aligned (the swizzled tiles need it):
   //   [Q of A 32 KB][Q of B 32 KB][K ring of A 3 x 32 KB][K ring of B 2 x 32 KB][mbarriers, flags 512 B]
@@ -436,9 +480,9 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   extern __shared__ __align__(1024) unsigned char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   unsigned char* tail = smem + 2 * kQBytes + (kStagesA + kStagesB) * kStageBytes;
-  uint32_t& tmem_base_sh = *reinterpret_cast<uint32_t*>(tail + 256);
-  int& abort_sh = *reinterpret_cast<int*>(tail + 260);
-  int& b_layer_sh = *reinterpret_cast<int*>(tail + 264);   // the layer stream B's epilogue has begun
+  uint32_t& tmem_base_sh = *reinterpret_cast<uint32_t*>(tail + 2 * kBarBytesPerStream);
+  int& abort_sh = *reinterpret_cast<int*>(tail + 2 * kBarBytesPerStream + 4);
+  int& b_layer_sh = *reinterpret_cast<int*>(tail + 2 * kBarBytesPerStream + 8);   // the layer stream B's epilogue has begun
   float* stat_m = reinterpret_cast<float*>(tail + 512);
   float* stat_z = stat_m + 128;
   float* lse2 = stat_m + 256;
@@ -477,6 +521,7 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
       const StreamCtx& c = s ? cb : ca;
       for (int st = 0; st < 3; ++st) { mbar_init(c.full_bar(st), 1); mbar_init(c.empty_bar(st), 1); }
       for (int b = 0; b < 2; ++b) { mbar_init(c.accf_bar(b), 1); mbar_init(c.acce_bar(b), 4); }
+      for (int g = 0; g < 6; ++g) mbar_init(c.accf_bar_of(g >> 1, g & 1), 1);
       mbar_init(c.qfull_bar(), 1);
       mbar_init(c.qempty_bar(), 1);
       mbar_init(c.drain_bar(), 1);
@@ -485,7 +530,7 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
   }
   // rows of a Q tile beyond R are never written by TMA: keep them zero
   if (a.R != 128) {
-    for (int i = tid; i < 2 * kQBytes / 16; i += kPipeThreads) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < 2 * kQBytes / 16; i += (int)blockDim.x) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
@@ -514,28 +559,30 @@ k_score_pipe(const __grid_constant__ PipeArgs pa) {
     }
   } else if (warp == 1) {
     if (lane == 0 && has_a) {
-      if (DUAL) issuer<true>(ca, a, pa.lay, pa.a_first, pa.a_last, pa.step);
+      if (DUAL) issuer<true, kDualWgs>(ca, a, pa.lay, pa.a_first, pa.a_last, pa.step);
       else issuer<false>(ca, a, pa.lay, pa.a_first, pa.a_last, 1);
     }
   } else if (warp == 2) {
     // normally entry 0 was read by the launch before; with both streams on pass 2 every entry is new to this launch
     if (lane == 0 && has_b) producer<true>(cb, a, pa.lay, pa.b_first, pa.b_last, pa.step, DUAL ? pa.b_first : 1);
   } else if (warp == 3) {
-    if (lane == 0 && has_b) issuer<true>(cb, a, pa.lay, pa.b_first, pa.b_last, pa.step);
-  } else if (warp < 12) {
+    if (lane == 0 && has_b) { if (DUAL) issuer<true, kDualWgs>(cb, a, pa.lay, pa.b_first, pa.b_last, pa.step); else issuer<true>(cb, a, pa.lay, pa.b_first, pa.b_last, pa.step); }
+  } else if (warp < (DUAL ? 4 + 4 * kDualWgs : 12)) {
     if (has_a) {
       pdl_wait();
       if (tid == 128) trace_mark(a.trace, 1);
-      if (DUAL) epilogue_votes(ca, a, pa, tid - 128, warp, stat_m, pa.a_first, pa.a_last, 1, false);
+      if (DUAL) epilogue_votes<kDualWgs>(ca, a, pa, tid - 128, warp, stat_m, pa.a_first, pa.a_last, 1, false);
       else epilogue_rows(ca, a, pa, tid - 128, warp, stat_m, stat_z);
       if (tid == 128) trace_mark(a.trace, 5);
     }
   } else {
     if (has_b) {
       pdl_wait();
-      if (tid == 384) trace_mark(a.trace, 7);
-      epilogue_votes(cb, a, pa, tid - 384, warp, lse2, pa.b_first, pa.b_last, 2, true);
-      if (tid == 384) trace_mark(a.trace, 6);
+      constexpr int kFirstB = DUAL ? 128 + 128 * kDualWgs : 384;
+      if (tid == kFirstB) trace_mark(a.trace, 7);
+      if (DUAL) epilogue_votes<kDualWgs>(cb, a, pa, tid - kFirstB, warp, lse2, pa.b_first, pa.b_last, 2, true);
+      else epilogue_votes<2>(cb, a, pa, tid - kFirstB, warp, lse2, pa.b_first, pa.b_last, 2, true);
+      if (tid == kFirstB) trace_mark(a.trace, 6);
     }
   }
 
@@ -678,7 +725,7 @@ cudaError_t launch_score_pipe(const TcPlan* pending, const TcPlan* const* a, int
   for (int attempt = 0; attempt < 2; ++attempt) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_cta);
-    cfg.blockDim = dim3(kPipeThreads);
+    cfg.blockDim = dim3(votes_only ? kDualThreads : kPipeThreads);
     cfg.dynamicSmemBytes = kPipeSmem;
     cfg.stream = st;
     cudaLaunchAttribute attr[3];

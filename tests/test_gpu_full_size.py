@@ -100,16 +100,42 @@ def test_config3_full_layers_through_the_overlapped_entry_point():
                      pooled=torch.full((n_pool,), float("nan"), dtype=torch.float32, device=dev),
                      status=torch.zeros(1, dtype=torch.int32, device=dev)) for _ in layers]
 
-    def run(fn, outs):
-        for x, bud, o in zip(xs, buds, outs):
+    def run(fn, outs, lses=None):
+        for i, (x, bud, o) in enumerate(zip(xs, buds, outs)):
             fn(params, x.q_win, x.k, x.v, cu_dev, cu, bud, o["k_out"], o["v_out"], o["offsets"], o["kept"], ws,
-               o["pooled"], o["status"])
+               o["pooled"], o["status"], lse=None if lses is None else lses[i])
         B.slkv_join()
         torch.cuda.synchronize()
 
     a, b = outputs(), outputs()
     run(B.slkv_compress, a)
     run(B.slkv_compress_overlapped, b)
+    # the same layers with their row log-sum-exps handed over (the vote pass alone on both streams of the list kernel,
+    # three epilogue warpgroups per stream): with the library's own log-sum-exps the scores agree with the two-pass
+    # results to rounding (another kernel computed the statistics, in another order) and the selections are valid
+    lses = []
+    for x in xs:
+        lse = torch.empty(1, wl.n_q_heads, wl.window, dtype=torch.float32, device=dev)
+        p2 = B.make_params(x.q_win, x.k, x.v, wl.window, wl.pool_kernel, lse_units=B.SLKV_LSE_LOG2)
+        B.slkv_row_lse(p2, x.q_win, x.k, cu_dev, cu, lse, ws)
+        lses.append(lse)
+    torch.cuda.synchronize()
+    c = outputs()
+    params_log2 = B.make_params(xs[0].q_win, xs[0].k, xs[0].v, wl.window, wl.pool_kernel, lse_units=B.SLKV_LSE_LOG2)
+    for i, (x, bud, o) in enumerate(zip(xs, buds, c)):
+        B.slkv_compress_overlapped(params_log2, x.q_win, x.k, x.v, cu_dev, cu, bud, o["k_out"], o["v_out"], o["offsets"],
+                                   o["kept"], ws, o["pooled"], o["status"], lse=lses[i])
+    B.slkv_join()
+    torch.cuda.synchronize()
+    for i in range(len(layers)):
+        assert int(c[i]["status"].item()) == 0
+        n = int(a[i]["offsets"][-1].item())
+        assert torch.equal(c[i]["offsets"], a[i]["offsets"])
+        assert torch.allclose(c[i]["pooled"], a[i]["pooled"], rtol=2e-5, atol=0)
+        off = a[i]["offsets"].tolist()
+        swapped = sum(len(set(c[i]["kept"][s0:s1].tolist()) ^ set(a[i]["kept"][s0:s1].tolist())) // 2
+                      for s0, s1 in zip(off, off[1:]))
+        assert swapped <= 8                           # positions may swap only inside the rounding band at the threshold
     for i, l in enumerate(layers):
         assert int(b[i]["status"].item()) == 0
         n = int(a[i]["offsets"][-1].item())
@@ -120,7 +146,9 @@ def test_config3_full_layers_through_the_overlapped_entry_point():
         x = xs[i]
         q, k, v = x.q_win.cpu(), x.k.cpu(), x.v.cpu()
         ref = P.oracle_pooled(q, k, cu, wl.window, wl.pool_kernel)
-        gpu = {"offsets": b[i]["offsets"].cpu().numpy().astype(np.int64), "kept_idx": b[i]["kept"].cpu().numpy().astype(np.int64),
-               "k_out": b[i]["k_out"].cpu(), "v_out": b[i]["v_out"].cpu()}
-        P.assert_pooled_close(b[i]["pooled"].cpu().numpy(), ref, cu, wl.n_kv_heads, wl.window)
-        P.assert_selection_valid(gpu, ref, cu, budgets[layers[i]].tolist(), wl.window, k, v)
+        for res in (b, c):                            # two passes, and the vote pass alone
+            gpu = {"offsets": res[i]["offsets"].cpu().numpy().astype(np.int64),
+                   "kept_idx": res[i]["kept"].cpu().numpy().astype(np.int64),
+                   "k_out": res[i]["k_out"].cpu(), "v_out": res[i]["v_out"].cpu()}
+            P.assert_pooled_close(res[i]["pooled"].cpu().numpy(), ref, cu, wl.n_kv_heads, wl.window)
+            P.assert_selection_valid(gpu, ref, cu, budgets[layers[i]].tolist(), wl.window, k, v)
