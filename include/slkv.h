@@ -321,7 +321,7 @@ int slkv_cp_descend(const int32_t* hist, int32_t n_kv_heads, int32_t level, uint
                     void* stream);
 int slkv_cp_local_ties(const int32_t* hist_local, const uint32_t* prefix, int32_t n_kv_heads, int32_t* ties,
                        void* stream);
-size_t slkv_cp_workspace_bytes(int32_t n_kv_heads, int64_t out_capacity_rows);
+size_t slkv_cp_workspace_bytes(int32_t n_kv_heads, int32_t own_count, int64_t out_capacity_rows);
 int slkv_cp_emit(const slkv_params* p, const void* k, const void* v, int64_t rows, const float* pooled,
                  int64_t row_stride, int32_t own_begin, int32_t own_count, int64_t pos0, const uint32_t* threshold,
                  const int32_t* need, const int32_t* ties_all, int32_t n_parts, int32_t part, int32_t window_rows,

@@ -123,7 +123,7 @@ def lib() -> C.CDLL:
         L.slkv_cp_local_ties.restype = C.c_int
         L.slkv_cp_local_ties.argtypes = [vp, vp, i32, vp, vp]
         L.slkv_cp_workspace_bytes.restype = sz
-        L.slkv_cp_workspace_bytes.argtypes = [i32, i64]
+        L.slkv_cp_workspace_bytes.argtypes = [i32, i32, i64]
         L.slkv_cp_emit.restype = C.c_int
         L.slkv_cp_emit.argtypes = [pp, vp, vp, i64, vp, i64, i32, i32, i64, vp, vp, vp, i32, i32, i32, i64, vp, vp, i64,
                                    vp, vp, vp, vp, sz, vp]
@@ -397,8 +397,8 @@ def slkv_cp_local_ties(hist_local: torch.Tensor, prefix: torch.Tensor, ties: tor
     return ties
 
 
-def slkv_cp_workspace_bytes(n_kv_heads: int, capacity_rows: int) -> int:
-    return int(lib().slkv_cp_workspace_bytes(int(n_kv_heads), int(capacity_rows)))
+def slkv_cp_workspace_bytes(n_kv_heads: int, own_count: int, capacity_rows: int) -> int:
+    return int(lib().slkv_cp_workspace_bytes(int(n_kv_heads), int(own_count), int(capacity_rows)))
 
 
 def slkv_cp_emit(params: SlkvParams, k: torch.Tensor, v: torch.Tensor, rows: int, pooled: torch.Tensor, row_stride: int,

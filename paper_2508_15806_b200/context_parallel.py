@@ -148,7 +148,7 @@ def compress_rank(shard: RankShard, budgets_row: torch.Tensor, pool_kernel: int,
                v_out=torch.zeros(max(cap, 1), d, dtype=sh.k.dtype, device=dev),
                offsets=torch.zeros(hkv + 1, **i32), kept_idx=torch.full((max(cap, 1),), -1, **i32), status=status,
                pooled=pooled, lse=lse, capacity=cap)
-    ws = torch.empty(max(B.slkv_cp_workspace_bytes(hkv, max(cap, 1)), 256), dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(B.slkv_cp_workspace_bytes(hkv, sh.own, max(cap, 1)), 256), dtype=torch.uint8, device=dev)
     B.slkv_cp_emit(p_any, sh.k, sh.v, sh.k.shape[0], pooled, max(n_ext, 1), sh.margin_left, sh.own, sh.begin, prefix,
                    need, ties_all, sh.rank, n_win, sh.seq_len - n_win, out["k_out"], out["v_out"], out["offsets"],
                    out["kept_idx"], ws, status, stream)

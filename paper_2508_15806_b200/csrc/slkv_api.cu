@@ -799,9 +799,12 @@ int slkv_cp_local_ties(const int32_t* hist_local, const uint32_t* prefix, int32_
   return e == cudaSuccess ? SLKV_OK : cuda_fail(e);
 }
 
-size_t slkv_cp_workspace_bytes(int32_t n_kv_heads, int64_t out_capacity_rows) {
-  if (n_kv_heads < 1 || out_capacity_rows < 0) return 0;
-  return align_up((size_t)out_capacity_rows * sizeof(int32_t)) + 2 * align_up((size_t)n_kv_heads * sizeof(int32_t));
+size_t slkv_cp_workspace_bytes(int32_t n_kv_heads, int32_t own_count, int64_t out_capacity_rows) {
+  if (n_kv_heads < 1 || own_count < 0 || out_capacity_rows < 0) return 0;
+  // source rows of the packed rows; rows and tie shares per head; two counts per slice of the owned range and head
+  const size_t slices = (size_t)cp_slices(own_count) * (size_t)n_kv_heads;
+  return align_up((size_t)out_capacity_rows * sizeof(int32_t)) + 2 * align_up((size_t)n_kv_heads * sizeof(int32_t)) +
+         2 * align_up(slices * sizeof(int32_t));
 }
 
 int slkv_cp_emit(const slkv_params* p, const void* k, const void* v, int64_t rows, const float* pooled,
@@ -823,18 +826,20 @@ int slkv_cp_emit(const slkv_params* p, const void* k, const void* v, int64_t row
     return SLKV_ERR_BAD_SHAPE;
   if (out_capacity_rows < 0) return SLKV_ERR_CAPACITY;
   if (!aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out)) return SLKV_ERR_BAD_ALIGN;
-  const size_t need_ws = slkv_cp_workspace_bytes(p->n_kv_heads, out_capacity_rows);
+  const size_t need_ws = slkv_cp_workspace_bytes(p->n_kv_heads, own_count, out_capacity_rows);
   if (!workspace || workspace_bytes < need_ws || reinterpret_cast<uintptr_t>(workspace) % kAlign != 0)
     return SLKV_ERR_WORKSPACE;
   char* w = static_cast<char*>(workspace);
   int32_t* gather_src = reinterpret_cast<int32_t*>(w);
   int32_t* rows_h = reinterpret_cast<int32_t*>(w + align_up((size_t)out_capacity_rows * sizeof(int32_t)));
   int32_t* take_h = rows_h + align_up((size_t)p->n_kv_heads * sizeof(int32_t)) / sizeof(int32_t);
+  int32_t* cnt_gt = take_h + align_up((size_t)p->n_kv_heads * sizeof(int32_t)) / sizeof(int32_t);
+  int32_t* cnt_eq = cnt_gt + align_up((size_t)cp_slices(own_count) * p->n_kv_heads * sizeof(int32_t)) / sizeof(int32_t);
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
   cudaError_t e = launch_cp_emit(pooled, row_stride, own_begin, own_count, pos0, threshold, need, ties_all,
                                  p->n_kv_heads, part, window_rows, rows - window_rows, window_pos0, out_capacity_rows,
-                                 offsets, kept_idx, gather_src, rows_h, take_h, status, st, &launches);
+                                 offsets, kept_idx, gather_src, rows_h, take_h, cnt_gt, cnt_eq, status, st, &launches);
   if (e != cudaSuccess) return cuda_fail(e);
   pb.total_tokens = rows;
   pb.n_seg = p->n_kv_heads;

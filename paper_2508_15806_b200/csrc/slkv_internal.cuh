@@ -155,7 +155,8 @@ cudaError_t launch_cp_emit(const float* pooled, long long row_stride, int own_be
                            const unsigned* threshold, const int32_t* need, const int32_t* ties_all, int n_kv_heads,
                            int part, int window_rows, long long window_row0, long long window_pos0, long long capacity,
                            int32_t* offsets, int32_t* kept_idx, int32_t* gather_src, int32_t* rows, int32_t* take,
-                           int32_t* status, cudaStream_t st, int* launches);
+                           int32_t* cnt_gt, int32_t* cnt_eq, int32_t* status, cudaStream_t st, int* launches);
+int cp_slices(int own_count);            // CTAs per head of the counting and packing kernels
 cudaError_t launch_setup(const Problem& pb, const int32_t* budgets, int32_t* offsets, int64_t capacity,
                          int32_t* status, cudaStream_t st, int* launches);
 int simt_chunk_keys();

@@ -191,7 +191,7 @@ def test_selection_is_exact_on_given_scores_with_many_ties(seed):
         cap = n_kv * (s["e"] - s["b"] + (w if last else 0))
         o = dict(k=torch.zeros(max(cap, 1), d, device=DEV), v=torch.zeros(max(cap, 1), d, device=DEV),
                  off=torch.zeros(n_kv + 1, **i32), idx=torch.full((max(cap, 1),), -1, **i32), status=torch.zeros(1, **i32))
-        ws = torch.empty(max(B.slkv_cp_workspace_bytes(n_kv, max(cap, 1)), 256), dtype=torch.uint8, device=DEV)
+        ws = torch.empty(max(B.slkv_cp_workspace_bytes(n_kv, s["e"] - s["b"], max(cap, 1)), 256), dtype=torch.uint8, device=DEV)
         B.slkv_cp_emit(p, kr, vr, kr.shape[0], s["pooled"], s["pooled"].shape[1], s["ml"], s["e"] - s["b"], s["b"],
                        s["prefix"], s["need"], ties_all, r, w if last else 0, L - w, o["k"], o["v"], o["off"], o["idx"],
                        ws, o["status"])

@@ -140,7 +140,7 @@ def test_history_only_and_context_parallel_argument_errors(L):
     assert L.slkv_cp_histogram(fake, 2, 100, 0, 20, 3, fake, fake, None) == B.ERR["BAD_SHAPE"]
     assert L.slkv_cp_descend(fake, 2, -1, fake, fake, None) == B.ERR["BAD_SHAPE"]
     assert L.slkv_cp_local_ties(fake, None, 2, fake, None) == B.ERR["NULL_PTR"]
-    assert L.slkv_cp_workspace_bytes(2, 1000) >= 4000 and L.slkv_cp_workspace_bytes(0, 10) == 0
+    assert L.slkv_cp_workspace_bytes(2, 500, 1000) >= 4000 and L.slkv_cp_workspace_bytes(0, 5, 10) == 0
     emit = [C.byref(p), fake, fake, 100, fake, 100, 0, 84, 0, fake, fake, fake, 2, 1, 16, 84, fake, fake, 200, fake, fake,
             None, fake, 1 << 20, None]
     bad = list(emit); bad[7] = 90                                 # owned rows run into the window rows
