@@ -70,7 +70,7 @@ class Job:
 
 
 def test_two_host_threads_each_on_its_own_stream():
-    # 21 and 13 layers of different shapes (more than a list, more than the slots of a workspace), three rounds each,
+    # 21 and 13 layers of different shapes (more than a list, more than the slots of a workspace), three times each,
     # the two threads free-running against each other; one of them hands its layers' log-sum-exps over
     jobs = [Job([6000], 21, 300, 0), Job([2500, 1200], 13, 200, 5, with_lse=True)]
     refs = [j.reference() for j in jobs]
@@ -157,7 +157,7 @@ def test_more_streams_than_the_library_keeps_states_for():
     job = Job([2000], 3, 150, 4)
     ref = job.reference()
     streams = [torch.cuda.Stream() for _ in range(10)]
-    for st in streams:                                 # first round: every stream joins for itself
+    for st in streams:                                 # first sweep over the streams: every stream joins for itself
         outs = job.outputs()
         torch.cuda.synchronize()
         for l in range(3):
@@ -166,7 +166,7 @@ def test_more_streams_than_the_library_keeps_states_for():
         torch.cuda.synchronize()
         job.assert_equal(outs, ref)
     alive = []
-    for st in streams:                                 # second round: left in flight; the library drains the state it
+    for st in streams:                                 # second sweep: left in flight; the library drains the state it
         outs = job.outputs()                           # hands on, and the last join covers the rest
         torch.cuda.synchronize()
         for l in range(3):
