@@ -35,8 +35,9 @@ constexpr int kDualWgs = 3;               // vote pass on both streams: warpgrou
 constexpr int kDualThreads = 128 + 2 * kDualWgs * 128;
 constexpr int kLeadEntries = 2;           // entries pass 1 may be ahead of the entry pass 2 has begun
 constexpr unsigned kPollNs = 64;          // pause between two polls of an mbarrier
-constexpr int kStagesA = 3;              // K tiles in flight from HBM
-constexpr int kStagesB = 2;              // K tiles in flight from L2
+constexpr int kStagesA = 2;              // K tiles in flight for stream A (pass 1: first read of a layer's K)
+constexpr int kStagesB = 3;              // ... for stream B (pass 2: ~70 % of its re-reads come from HBM again, and
+                                         // its tiles take longer; measured 1.7 % faster than 3 + 2)
 constexpr int kQBytes = 2 * kHalfBytes;  // one 128-row Q tile
 constexpr int kBarBytesPerStream = 160;  // up to 20 mbarriers
 constexpr int kPipeTail = 512 + 1024 + 1024;   // mbarriers + flags, stat_m/stat_z of stream A, two log-sum-exp rows of stream B
@@ -475,7 +476,7 @@ template <bool DUAL>
 __global__ void __launch_bounds__(DUAL ? kDualThreads : kPipeThreads, 1)
 k_score_pipe(const __grid_constant__ PipeArgs pa) {
   // Shared memory, all dynamic and 1024-byte aligned (the swizzled tiles need it):
-  //   [Q of A 32 KB][Q of B 32 KB][K ring of A 3 x 32 KB][K ring of B 2 x 32 KB][mbarriers, flags 512 B]
+  //   [Q of A 32 KB][Q of B 32 KB][K ring of A 2 x 32 KB][K ring of B 3 x 32 KB][mbarriers, flags 512 B]
   //   [stat_m, stat_z of A 1 KB][log-sum-exp rows of B 2 x 512 B]
   extern __shared__ __align__(1024) unsigned char smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
